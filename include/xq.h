@@ -1,0 +1,189 @@
+/* xq.h -- C ABI of the XQuant KV-cache library for NVIDIA B200 (sm_100a).
+ *
+ * The library keeps, for every transformer layer, a KV cache made of
+ *   - a quantized region: 1- or 2-bit integer codes plus one fp16 scale and one
+ *     fp16 zero-point per group (keys: one group per channel and run of
+ *     `group_size` tokens; values: one group per token and run of `group_size`
+ *     channels) -- the min-max group quantizer of Section 3.1 (Eq. 1-3) with
+ *     the data-free calibration of Section 3.2 (Eq. 12);
+ *   - a 16-bit residual window holding the most recent tokens unquantized
+ *     (Section 4.1, residual length);
+ * and, for each adjacent layer pair (2p, 2p+1) at or above the sharing start,
+ * stores the integer codes once, in layer 2p, while both layers keep their own
+ * scale and zero-point (Section 3.3.3 / 3.3.4 with group size G = 2 and dominant
+ * layer k = 0; Algorithms 1 and 2).
+ *
+ * Two operations form the hot path: xq_append_kv (window append, and
+ * quantize-and-pack of every window block that fills) and xq_decode_attention
+ * (one query per head against the packed cache plus the window).
+ *
+ * Conventions that hold for every entry point:
+ *   - "device" pointers are CUDA device addresses valid on the device that was
+ *     current when xq_create ran; "host" pointers are ordinary host addresses.
+ *   - The caller owns every device byte (inputs, outputs, the workspace) and the
+ *     stream.  The library never allocates or frees device memory and never
+ *     synchronizes the device, except where a function says otherwise.  All
+ *     kernels are launched asynchronously on the given stream
+ *     (a cudaStream_t passed as void*; NULL is the default stream).
+ *   - Every function returns XQ_OK (0) or a negative XQ_ERR_* code; a failing
+ *     call leaves the cache unchanged.  Nothing is thrown across the boundary.
+ *   - A cache handle is not thread-safe; use one host thread per handle.
+ *   - 16-bit inputs and outputs are bfloat16 (io_dtype XQ_BF16).
+ */
+#ifndef XQ_H_
+#define XQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define XQ_OK 0
+#define XQ_ERR_CONFIG (-1)   /* invalid xq_config                                        */
+#define XQ_ERR_ARG (-2)      /* null / misaligned pointer, layer or token count invalid   */
+#define XQ_ERR_CAPACITY (-3) /* would exceed max_seq, or the workspace is too small       */
+#define XQ_ERR_ORDER (-4)    /* a code-borrowing layer is ahead of the layer owning codes */
+#define XQ_ERR_CUDA (-5)     /* a CUDA call failed; xq_last_cuda_error gives the code     */
+#define XQ_ERR_NOMEM (-6)    /* host allocation failed                                    */
+
+#define XQ_BF16 0
+
+#define XQ_KERNEL_AUTO 0    /* tensor-core kernel when the shape allows it, else generic   */
+#define XQ_KERNEL_GENERIC 1 /* scalar kernel: any supported shape, slow, used as cross-check */
+#define XQ_KERNEL_MMA 2     /* tensor-core kernel: head_dim 128, group of <= 8 query heads  */
+
+#define XQ_MEM_DEVICE 0
+#define XQ_MEM_HOST 1
+
+/* Problem statement of Algorithm 1 (inputs kq, vq, km, vm, eta[2]) plus the
+ * group size and residual length of Section 4.1 and the tensor shapes. */
+typedef struct xq_config {
+  int32_t n_layers;     /* L >= 1                                                         */
+  int32_t batch;        /* sequences, all of the same length                              */
+  int32_t n_q_heads;    /* query heads; a multiple of n_kv_heads (GQA; equal = MHA)       */
+  int32_t n_kv_heads;   /* KV heads; query head h reads KV head h / (n_q_heads/n_kv_heads) */
+  int32_t head_dim;     /* D: 64 or 128                                                   */
+  int32_t max_seq;      /* capacity in tokens per sequence                                */
+  int32_t group_size;   /* g: tokens per key group, channels per value group; 32 or 64   */
+  int32_t residual_len; /* R: window capacity; a multiple of g and of 32                  */
+  int32_t kq, vq;       /* key / value layers [0,kq) / [0,vq) use 2 bits, the rest 1 bit
+                           (Appendix E)                                                   */
+  int32_t km, vm;       /* from layer km / vm on, odd layer l reads the codes of l-1
+                           (Algorithm 1, dequantize loop); km = vm = n_layers: no sharing.
+                           The two layers of a sharing pair must have equal bit-width.    */
+  float eta1, eta2;     /* calibration parameter eta_B for B = 1, 2, in [0, 0.5] (Eq. 5)  */
+  float sm_scale;       /* softmax scale; 0 selects 1/sqrt(head_dim)                      */
+  int32_t n_splits;     /* sequence splits per (sequence, KV head) in decode; 0 = library
+                           chooses; at most XQ_MAX_SPLITS                                 */
+  int32_t io_dtype;     /* XQ_BF16                                                        */
+  int32_t kernel;       /* XQ_KERNEL_*                                                    */
+} xq_config;
+
+#define XQ_MAX_SPLITS 256
+
+typedef struct xq_cache xq_cache; /* opaque; owns host memory only */
+
+/* Validates a configuration (rules above; head_dim % group_size == 0; with
+ * head_dim 64 and a 1-bit layer, residual_len % 64 == 0).  XQ_OK or XQ_ERR_CONFIG. */
+int xq_config_check(const xq_config* cfg);
+
+/* Device bytes xq_create needs for `cfg`: windows, scale / zero-point, codes of
+ * code-owning layers, split-K partials and the host-staging area.  0 if invalid. */
+size_t xq_workspace_bytes(const xq_config* cfg);
+
+/* Creates a cache over the caller's device buffer `dev_workspace` (256-byte
+ * aligned, at least xq_workspace_bytes(cfg) bytes, contents arbitrary).  The
+ * buffer must outlive the handle and must not be written by the caller while
+ * the handle lives.  Uses the current CUDA device.  All layers start empty. */
+int xq_create(const xq_config* cfg, void* dev_workspace, size_t bytes, xq_cache** out);
+
+/* Frees the host-side handle (and its timing events).  Device memory is the caller's. */
+int xq_destroy(xq_cache* c);
+
+/* All layers back to length 0.  No device work. */
+int xq_reset(xq_cache* c);
+
+/* Appends n_tokens >= 1 tokens to `layer` (Algorithm 1, quantize loop, with the
+ * residual window of Section 4.1).  K, V: device, [batch, n_kv_heads, n_tokens,
+ * head_dim] contiguous bfloat16, 16-byte aligned, read-only, must stay valid
+ * until the stream has run the call.  Tokens enter the window; when the window
+ * already holds R tokens and a further token arrives, that block of R tokens is
+ * quantized (Eq. 1, 2, 12): scale and zero-point always, integer codes only if
+ * the layer owns codes (Quantize), not if it borrows them (PseudoQuantize).
+ * After S tokens the window holds ((S-1) mod R)+1 tokens.
+ * Errors: XQ_ERR_ARG, XQ_ERR_CAPACITY (S would exceed max_seq), XQ_ERR_CUDA. */
+int xq_append_kv(xq_cache* c, int layer, const void* K, const void* V, int n_tokens, void* stream);
+
+/* One decode query per head against everything cached in `layer` (Algorithm 1,
+ * dequantize loop, followed by softmax attention): K_hat = codes * s_hat + z_hat
+ * (Eq. 3 with the calibrated parameters of `layer`, codes of the pair's owning
+ * layer), logits = sm_scale * q . K_hat over quantized then window tokens,
+ * out = softmax(logits) . V_hat.  No mask.  q, out: device, [batch, n_q_heads,
+ * head_dim] bfloat16, 16-byte aligned.  fp32 accumulation.
+ * Errors: XQ_ERR_ARG (also: empty layer), XQ_ERR_ORDER (the owning layer holds
+ * fewer quantized tokens than `layer`), XQ_ERR_CUDA. */
+int xq_decode_attention(xq_cache* c, int layer, const void* q, void* out, void* stream);
+
+/* Same as xq_decode_attention with out: device float32 [batch, n_q_heads,
+ * head_dim] (the accumulator before the final rounding to bfloat16). */
+int xq_decode_attention_f32(xq_cache* c, int layer, const void* q, float* out, void* stream);
+
+/* One decode step of a whole model: for each layer l in ascending order, append
+ * one token and run decode attention.  K_new, V_new: [n_layers, batch,
+ * n_kv_heads, 1, head_dim]; q, out: [n_layers, batch, n_q_heads, head_dim];
+ * bfloat16.  mem = XQ_MEM_DEVICE: device pointers, used in place.
+ * mem = XQ_MEM_HOST: host pointers (pinned memory for the copies to be
+ * asynchronous); inputs are copied to the workspace's staging area on `stream`,
+ * the result is copied back to `out` on `stream`; the caller synchronizes the
+ * stream before reading `out` or reusing the host buffers. */
+int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void* q, void* out,
+                   int mem, void* stream);
+
+/* Equivalent bit-width of Appendix C: stored code bits per cached element,
+ * averaged over layers and over keys and values; scale / zero-point excluded,
+ * a code-borrowing layer counts zero.  Negative if cfg is invalid. */
+double xq_equiv_bits(const xq_config* cfg);
+
+/* Tokens cached in `layer` (negative error code on bad arguments). */
+int xq_seq_len(const xq_cache* c, int layer);
+/* Of those, tokens in the quantized region (a multiple of residual_len). */
+int xq_quantized_len(const xq_cache* c, int layer);
+/* Splits (quantized-region, window) the next decode call on `layer` would use. */
+int xq_split_plan(const xq_cache* c, int layer, int* n_splits_quantized, int* n_splits_window);
+
+/* Where a layer's data lives inside the workspace, for tests and snapshots.
+ * which: 0 key codes, 1 value codes (of the layer that owns them), 2 key
+ * scale/zero, 3 value scale/zero, 4 key window, 5 value window.  Returns byte
+ * offset from the workspace start and the byte stride between consecutive
+ * (sequence, kv head) streams.
+ * Layouts (all little-endian, one stream per (sequence, kv head)):
+ *   codes: tiles of 128 uint32; see DESIGN notes in xq_layout.cuh for the bit map;
+ *   key scale/zero: per token group [2][head_dim] fp16 (scale block, zero block),
+ *     permuted within the block; value scale/zero: per 16 tokens
+ *     [2][16*head_dim/group_size] fp16; windows: [R][head_dim] bfloat16. */
+int xq_region(const xq_cache* c, int layer, int which, size_t* offset, size_t* stream_stride);
+
+/* Kernel launches issued through this handle since creation (all kinds). */
+long long xq_launch_count(const xq_cache* c);
+
+/* Optional per-kernel timing with CUDA events recorded on the launching stream
+ * around each kernel.  xq_timing_enable(c, 1) allocates an event pool (host
+ * call, not on the hot path) and clears the records; (c, 0) stops recording.
+ * xq_timing_read synchronizes on the recorded events and returns, per kind
+ * (0 decode split kernel, 1 merge kernel, 2 quantize-and-pack kernel, 3 window
+ * append kernel), the launch count and total milliseconds. */
+int xq_timing_enable(xq_cache* c, int on);
+int xq_timing_read(xq_cache* c, int kind, int* launches, double* total_ms);
+
+/* CUDA error code (cudaError_t) of the last XQ_ERR_CUDA on this handle, else 0. */
+int xq_last_cuda_error(const xq_cache* c);
+
+/* Static text for an XQ_* code. */
+const char* xq_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XQ_H_ */

@@ -1,0 +1,494 @@
+// Host side of the library: configuration checks, workspace carving, the
+// per-layer sequence counters (Algorithm 1's bookkeeping), split planning and
+// the C entry points.  No device memory is allocated here.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/xq.h"
+#include "xq_internal.h"
+
+using namespace xq;
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline int layer_bits(int l, int q) { return l < q ? 2 : 1; }
+inline bool owns_codes(int l, int m) { return l < m || (l % 2) == 0; }
+
+struct LayerRegions {
+  size_t win_k, win_v, k_meta, v_meta, k_codes, v_codes;  // byte offsets; codes: of the owning layer
+  size_t stride[6];                                       // per (sequence, kv head) stream, bytes
+};
+
+struct Plan {
+  Dims dm;
+  std::vector<LayerRegions> layers;
+  size_t part_acc, part_ml, staging, total;
+  size_t staging_kv_bytes, staging_q_bytes;
+};
+
+bool check(const xq_config* c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1) return false;
+  if (c->n_q_heads % c->n_kv_heads) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->group_size != 32 && c->group_size != 64) return false;
+  if (c->head_dim % c->group_size) return false;
+  if (c->residual_len < 32 || c->residual_len % c->group_size || c->residual_len % 32) return false;
+  if (c->residual_len > 4096) return false;
+  if (c->max_seq < 1) return false;
+  if (c->kq < 0 || c->kq > c->n_layers || c->vq < 0 || c->vq > c->n_layers) return false;
+  if (c->km < 0 || c->km > c->n_layers || c->vm < 0 || c->vm > c->n_layers) return false;
+  if (!(c->eta1 >= 0.f && c->eta1 <= 0.5f) || !(c->eta2 >= 0.f && c->eta2 <= 0.5f)) return false;
+  if (!(c->sm_scale >= 0.f) || isinf(c->sm_scale)) return false;
+  if (c->n_splits < 0 || c->n_splits > XQ_MAX_SPLITS) return false;
+  if (c->io_dtype != XQ_BF16) return false;
+  if (c->kernel < XQ_KERNEL_AUTO || c->kernel > XQ_KERNEL_MMA) return false;
+  bool any_1bit = c->kq < c->n_layers || c->vq < c->n_layers;
+  if (c->head_dim == 64 && any_1bit && c->residual_len % 64) return false;
+  // both layers of a sharing pair must have the same bit-width
+  for (int l = 1; l < c->n_layers; l += 2) {
+    if (!owns_codes(l, c->km) && layer_bits(l, c->kq) != layer_bits(l - 1, c->kq)) return false;
+    if (!owns_codes(l, c->vm) && layer_bits(l, c->vq) != layer_bits(l - 1, c->vq)) return false;
+  }
+  return true;
+}
+
+void make_plan(const xq_config* c, Plan& pl) {
+  Dims& dm = pl.dm;
+  dm.B = c->batch; dm.Hq = c->n_q_heads; dm.Hkv = c->n_kv_heads; dm.G = dm.Hq / dm.Hkv;
+  dm.D = c->head_dim; dm.g = c->group_size; dm.R = c->residual_len; dm.NG = dm.D / dm.g;
+  dm.nq_cap = c->max_seq > 1 ? ((c->max_seq - 1) / dm.R) * dm.R : 0;
+  const size_t BH = (size_t)dm.B * dm.Hkv;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  pl.layers.resize(c->n_layers);
+  for (int l = 0; l < c->n_layers; ++l) {
+    LayerRegions& r = pl.layers[l];
+    int bk = layer_bits(l, c->kq), bv = layer_bits(l, c->vq);
+    r.stride[4] = r.stride[5] = (size_t)dm.R * dm.D * 2;
+    r.win_k = take(BH * r.stride[4]);
+    r.win_v = take(BH * r.stride[5]);
+    r.stride[2] = (size_t)(dm.nq_cap / dm.g) * 2 * dm.D * 2;
+    r.stride[3] = (size_t)(dm.nq_cap / 16) * 2 * 16 * dm.NG * 2;
+    r.k_meta = take(BH * r.stride[2]);
+    r.v_meta = take(BH * r.stride[3]);
+    r.stride[0] = (size_t)dm.nq_cap * dm.D * bk / 8;
+    r.stride[1] = (size_t)dm.nq_cap * dm.D * bv / 8;
+    if (owns_codes(l, c->km)) r.k_codes = take(BH * r.stride[0]); else r.k_codes = pl.layers[l - 1].k_codes;
+    if (owns_codes(l, c->vm)) r.v_codes = take(BH * r.stride[1]); else r.v_codes = pl.layers[l - 1].v_codes;
+  }
+  pl.part_acc = take((size_t)dm.B * dm.Hq * XQ_MAX_SPLITS * dm.D * 4);
+  pl.part_ml = take((size_t)dm.B * dm.Hq * XQ_MAX_SPLITS * 2 * 4);
+  pl.staging_kv_bytes = (size_t)c->n_layers * BH * dm.D * 2;
+  pl.staging_q_bytes = (size_t)c->n_layers * dm.B * dm.Hq * dm.D * 2;
+  pl.staging = take(2 * align_up(pl.staging_kv_bytes, 256) + 2 * align_up(pl.staging_q_bytes, 256));
+  pl.total = off;
+}
+
+constexpr int N_KINDS = 4;
+constexpr int TIMING_POOL = 1 << 15;
+
+struct EventPair { cudaEvent_t a, b; int kind; };
+
+}  // namespace
+
+struct xq_cache {
+  xq_config cfg;
+  Plan plan;
+  uint8_t* ws;
+  std::vector<int> seq;  // tokens cached per layer
+  long long launches;
+  int last_cuda;
+  float scale;
+  int sm_count;
+  // timing
+  bool timing;
+  std::vector<EventPair> pool;
+  size_t used;
+};
+
+namespace {
+
+inline int residual_count(int S, int R) { return S > 0 ? ((S - 1) % R) + 1 : 0; }
+
+LayerPtrs layer_ptrs(const xq_cache* c, int l) {
+  const LayerRegions& r = c->plan.layers[l];
+  LayerPtrs p;
+  p.win_k = (uint16_t*)(c->ws + r.win_k);
+  p.win_v = (uint16_t*)(c->ws + r.win_v);
+  p.k_meta = (uint16_t*)(c->ws + r.k_meta);
+  p.v_meta = (uint16_t*)(c->ws + r.v_meta);
+  p.k_codes = (uint32_t*)(c->ws + r.k_codes);
+  p.v_codes = (uint32_t*)(c->ws + r.v_codes);
+  p.bk = layer_bits(l, c->cfg.kq);
+  p.bv = layer_bits(l, c->cfg.vq);
+  return p;
+}
+
+// Bytes one quantized token / one window token costs a (sequence, kv head) stream.
+void token_bytes(const xq_cache* c, int l, double& q_bytes, double& w_bytes) {
+  const Dims& dm = c->plan.dm;
+  int bk = layer_bits(l, c->cfg.kq), bv = layer_bits(l, c->cfg.vq);
+  q_bytes = dm.D * (bk + bv) / 8.0 + 4.0 * dm.D / dm.g + 4.0 * dm.NG;
+  w_bytes = 4.0 * dm.D;
+}
+
+void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w) {
+  const Dims& dm = c->plan.dm;
+  int S = c->seq[l];
+  int r = residual_count(S, dm.R), nq = S - r;
+  int units = nq / 32, tiles = (r + 15) / 16;
+  double qb, wb;
+  token_bytes(c, l, qb, wb);
+  double bytes_q = qb * nq, bytes_w = wb * r;
+  int total;
+  if (c->cfg.n_splits > 0) {
+    total = c->cfg.n_splits;
+  } else {
+    // aim for ~48 KB of cache per CTA, then round the grid to whole waves of 2 CTAs per SM
+    double per_stream = bytes_q + bytes_w;
+    int streams = dm.B * dm.Hkv;
+    int want = (int)ceil(per_stream / 49152.0);
+    if (want < 1) want = 1;
+    long long ctas = (long long)want * streams;
+    long long wave = 2LL * c->sm_count;
+    if (ctas > wave) {
+      long long waves = (ctas + wave / 2) / wave;
+      if (waves < 1) waves = 1;
+      want = (int)((waves * wave) / streams);
+      if (want < 1) want = 1;
+    }
+    total = want;
+  }
+  if (total > XQ_MAX_SPLITS) total = XQ_MAX_SPLITS;
+  if (units == 0) {
+    ns_q = 0;
+    ns_w = total < tiles ? total : tiles;
+    if (ns_w < 1) ns_w = 1;
+    return;
+  }
+  if (tiles == 0) {  // not reachable with S > 0, kept for safety
+    ns_w = 0;
+    ns_q = total < units ? total : units;
+    return;
+  }
+  int w = (int)floor(total * bytes_w / (bytes_q + bytes_w) + 0.5);
+  if (w < 1) w = 1;
+  if (w > tiles) w = tiles;
+  int q = total - w;
+  if (q < 1) q = 1;
+  if (q > units) q = units;
+  ns_q = q;
+  ns_w = w;
+}
+
+struct Timer {
+  xq_cache* c; cudaStream_t st; EventPair* ev;
+  Timer(xq_cache* c_, cudaStream_t st_, int kind) : c(c_), st(st_), ev(nullptr) {
+    if (c->timing && c->used < c->pool.size()) {
+      ev = &c->pool[c->used++];
+      ev->kind = kind;
+      cudaEventRecord(ev->a, st);
+    }
+  }
+  ~Timer() { if (ev) cudaEventRecord(ev->b, st); }
+};
+
+int fail_cuda(xq_cache* c, cudaError_t e) { c->last_cuda = (int)e; return XQ_ERR_CUDA; }
+
+int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, cudaStream_t st) {
+  if (!c || !q || !out) return XQ_ERR_ARG;
+  if (layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
+  if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return XQ_ERR_ARG;
+  const Dims& dm = c->plan.dm;
+  int S = c->seq[layer];
+  if (S < 1) return XQ_ERR_ARG;
+  int r = residual_count(S, dm.R), nq = S - r;
+  // a code-borrowing layer needs the owning layer's codes for all of its quantized tokens
+  bool bor_k = !owns_codes(layer, c->cfg.km), bor_v = !owns_codes(layer, c->cfg.vm);
+  if (bor_k || bor_v) {
+    int So = c->seq[layer - 1];
+    int nqo = So - residual_count(So, dm.R);
+    if (nqo < nq) return XQ_ERR_ORDER;
+  }
+  DecodeParams p;
+  p.dm = dm;
+  p.L = layer_ptrs(c, layer);
+  p.q = (const uint16_t*)q;
+  p.n_q = nq;
+  p.r = r;
+  plan_splits(c, layer, p.ns_q, p.ns_w);
+  p.scale = c->scale;
+  p.part_acc = (float*)(c->ws + c->plan.part_acc);
+  p.part_ml = (float*)(c->ws + c->plan.part_ml);
+  bool use_mma = c->cfg.kernel != XQ_KERNEL_GENERIC && decode_mma_supported(dm, p.L.bk, p.L.bv);
+  if (c->cfg.kernel == XQ_KERNEL_MMA && !use_mma) return XQ_ERR_CONFIG;
+  cudaError_t e;
+  {
+    Timer t(c, st, 0);
+    e = use_mma ? launch_decode_mma(p, st) : launch_decode_generic(p, st);
+  }
+  c->launches++;
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  MergeParams m;
+  m.dm = dm;
+  m.ns = p.ns_q + p.ns_w;
+  m.part_acc = p.part_acc;
+  m.part_ml = p.part_ml;
+  m.out = out;
+  m.out_f32 = out_f32;
+  {
+    Timer t(c, st, 1);
+    e = launch_merge(m, st);
+  }
+  c->launches++;
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  return XQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int xq_config_check(const xq_config* cfg) { return check(cfg) ? XQ_OK : XQ_ERR_CONFIG; }
+
+size_t xq_workspace_bytes(const xq_config* cfg) {
+  if (!check(cfg)) return 0;
+  Plan pl;
+  make_plan(cfg, pl);
+  return pl.total;
+}
+
+int xq_create(const xq_config* cfg, void* dev_workspace, size_t bytes, xq_cache** out) {
+  if (!out) return XQ_ERR_ARG;
+  *out = nullptr;
+  if (!check(cfg)) return XQ_ERR_CONFIG;
+  if (!dev_workspace || ((uintptr_t)dev_workspace & 255)) return XQ_ERR_ARG;
+  xq_cache* c = new (std::nothrow) xq_cache();
+  if (!c) return XQ_ERR_NOMEM;
+  c->cfg = *cfg;
+  make_plan(cfg, c->plan);
+  if (bytes < c->plan.total) { delete c; return XQ_ERR_CAPACITY; }
+  c->ws = (uint8_t*)dev_workspace;
+  c->seq.assign(cfg->n_layers, 0);
+  c->launches = 0;
+  c->last_cuda = 0;
+  c->scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.0f / sqrtf((float)cfg->head_dim);
+  c->timing = false;
+  c->used = 0;
+  c->sm_count = 148;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess &&
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+    c->sm_count = sms;
+  else
+    cudaGetLastError();  // no device (host-only use of the handle): keep the default
+  *out = c;
+  return XQ_OK;
+}
+
+int xq_destroy(xq_cache* c) {
+  if (!c) return XQ_ERR_ARG;
+  for (auto& e : c->pool) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+  delete c;
+  return XQ_OK;
+}
+
+int xq_reset(xq_cache* c) {
+  if (!c) return XQ_ERR_ARG;
+  for (auto& s : c->seq) s = 0;
+  return XQ_OK;
+}
+
+int xq_append_kv(xq_cache* c, int layer, const void* K, const void* V, int n_tokens, void* stream) {
+  if (!c || !K || !V) return XQ_ERR_ARG;
+  if (layer < 0 || layer >= c->cfg.n_layers || n_tokens < 1) return XQ_ERR_ARG;
+  if (((uintptr_t)K & 15) || ((uintptr_t)V & 15)) return XQ_ERR_ARG;
+  const Dims& dm = c->plan.dm;
+  cudaStream_t st = (cudaStream_t)stream;
+  int s_old = c->seq[layer];
+  if ((long long)s_old + n_tokens > c->cfg.max_seq) return XQ_ERR_CAPACITY;
+  int s_new = s_old + n_tokens;
+  int nq_old = s_old - residual_count(s_old, dm.R);
+  int nq_new = s_new - residual_count(s_new, dm.R);
+  int n_blocks = (nq_new - nq_old) / dm.R;
+  LayerPtrs L = layer_ptrs(c, layer);
+  if (n_blocks > 0) {
+    PackParams p;
+    p.dm = dm; p.L = L;
+    p.K_in = (const uint16_t*)K; p.V_in = (const uint16_t*)V;
+    p.n_in = n_tokens; p.s_old = s_old; p.nq_old = nq_old; p.n_blocks = n_blocks;
+    p.own_k = owns_codes(layer, c->cfg.km); p.own_v = owns_codes(layer, c->cfg.vm);
+    p.eta_k = L.bk == 1 ? c->cfg.eta1 : c->cfg.eta2;
+    p.eta_v = L.bv == 1 ? c->cfg.eta1 : c->cfg.eta2;
+    p.tb = (dm.R % 64 == 0) ? 64 : 32;  // g = 64 implies R % 64 == 0
+    cudaError_t e;
+    {
+      Timer t(c, st, 2);
+      e = launch_pack(p, st);
+    }
+    c->launches++;
+    if (e != cudaSuccess) return fail_cuda(c, e);
+  }
+  {
+    WindowParams w;
+    w.dm = dm; w.L = L;
+    w.K_in = (const uint16_t*)K; w.V_in = (const uint16_t*)V;
+    w.n_in = n_tokens; w.s_old = s_old;
+    w.first = s_old > nq_new ? s_old : nq_new;
+    w.count = s_new - w.first;
+    w.nq_new = nq_new;
+    cudaError_t e;
+    {
+      Timer t(c, st, 3);
+      e = launch_window_append(w, st);
+    }
+    c->launches++;
+    if (e != cudaSuccess) return fail_cuda(c, e);
+  }
+  c->seq[layer] = s_new;
+  return XQ_OK;
+}
+
+int xq_decode_attention(xq_cache* c, int layer, const void* q, void* out, void* stream) {
+  return decode_impl(c, layer, q, out, 0, (cudaStream_t)stream);
+}
+
+int xq_decode_attention_f32(xq_cache* c, int layer, const void* q, float* out, void* stream) {
+  return decode_impl(c, layer, q, out, 1, (cudaStream_t)stream);
+}
+
+int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void* q, void* out, int mem,
+                   void* stream) {
+  if (!c || !K_new || !V_new || !q || !out) return XQ_ERR_ARG;
+  if (mem != XQ_MEM_DEVICE && mem != XQ_MEM_HOST) return XQ_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const Dims& dm = c->plan.dm;
+  const int L = c->cfg.n_layers;
+  for (int l = 0; l < L; ++l)
+    if (c->seq[l] + 1 > c->cfg.max_seq) return XQ_ERR_CAPACITY;
+  const size_t kv_layer = (size_t)dm.B * dm.Hkv * dm.D * 2;
+  const size_t q_layer = (size_t)dm.B * dm.Hq * dm.D * 2;
+  const uint8_t *dk = (const uint8_t*)K_new, *dv = (const uint8_t*)V_new, *dq = (const uint8_t*)q;
+  uint8_t* dout = (uint8_t*)out;
+  if (mem == XQ_MEM_HOST) {
+    uint8_t* s = c->ws + c->plan.staging;
+    size_t kvb = align_up(c->plan.staging_kv_bytes, 256), qb = align_up(c->plan.staging_q_bytes, 256);
+    uint8_t *sk = s, *sv = s + kvb, *sq = s + 2 * kvb, *so = s + 2 * kvb + qb;
+    cudaError_t e = cudaMemcpyAsync(sk, K_new, c->plan.staging_kv_bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(sv, V_new, c->plan.staging_kv_bytes, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(sq, q, c->plan.staging_q_bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return fail_cuda(c, e);
+    dk = sk; dv = sv; dq = sq; dout = so;
+  }
+  for (int l = 0; l < L; ++l) {
+    int rc = xq_append_kv(c, l, dk + l * kv_layer, dv + l * kv_layer, 1, stream);
+    if (rc != XQ_OK) return rc;
+    rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st);
+    if (rc != XQ_OK) return rc;
+  }
+  if (mem == XQ_MEM_HOST) {
+    cudaError_t e = cudaMemcpyAsync(out, dout, c->plan.staging_q_bytes, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return fail_cuda(c, e);
+  }
+  return XQ_OK;
+}
+
+double xq_equiv_bits(const xq_config* cfg) {
+  if (!check(cfg)) return -1.0;
+  long long k = 0, v = 0;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    if (owns_codes(l, cfg->km)) k += layer_bits(l, cfg->kq);
+    if (owns_codes(l, cfg->vm)) v += layer_bits(l, cfg->vq);
+  }
+  return 0.5 * ((double)k + (double)v) / (double)cfg->n_layers;
+}
+
+int xq_seq_len(const xq_cache* c, int layer) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
+  return c->seq[layer];
+}
+
+int xq_quantized_len(const xq_cache* c, int layer) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
+  int S = c->seq[layer];
+  return S - residual_count(S, c->plan.dm.R);
+}
+
+int xq_split_plan(const xq_cache* c, int layer, int* nsq, int* nsw) {
+  if (!c || !nsq || !nsw || layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
+  if (c->seq[layer] < 1) return XQ_ERR_ARG;
+  plan_splits(c, layer, *nsq, *nsw);
+  return XQ_OK;
+}
+
+int xq_region(const xq_cache* c, int layer, int which, size_t* offset, size_t* stream_stride) {
+  if (!c || !offset || !stream_stride || layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
+  if (which < 0 || which > 5) return XQ_ERR_ARG;
+  const LayerRegions& r = c->plan.layers[layer];
+  const size_t offs[6] = {r.k_codes, r.v_codes, r.k_meta, r.v_meta, r.win_k, r.win_v};
+  *offset = offs[which];
+  *stream_stride = r.stride[which];
+  return XQ_OK;
+}
+
+long long xq_launch_count(const xq_cache* c) { return c ? c->launches : 0; }
+
+int xq_timing_enable(xq_cache* c, int on) {
+  if (!c) return XQ_ERR_ARG;
+  if (on && c->pool.empty()) {
+    c->pool.reserve(TIMING_POOL);
+    for (int i = 0; i < TIMING_POOL; ++i) {
+      EventPair e;
+      if (cudaEventCreate(&e.a) != cudaSuccess || cudaEventCreate(&e.b) != cudaSuccess)
+        return fail_cuda(c, cudaGetLastError());
+      e.kind = -1;
+      c->pool.push_back(e);
+    }
+  }
+  c->timing = on != 0;
+  if (on) c->used = 0;
+  return XQ_OK;
+}
+
+int xq_timing_read(xq_cache* c, int kind, int* launches, double* total_ms) {
+  if (!c || !launches || !total_ms || kind < 0 || kind >= N_KINDS) return XQ_ERR_ARG;
+  int n = 0;
+  double tot = 0.0;
+  for (size_t i = 0; i < c->used; ++i) {
+    EventPair& e = c->pool[i];
+    if (e.kind != kind) continue;
+    cudaError_t err = cudaEventSynchronize(e.b);
+    float ms = 0.f;
+    if (err == cudaSuccess) err = cudaEventElapsedTime(&ms, e.a, e.b);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+    tot += ms;
+    ++n;
+  }
+  *launches = n;
+  *total_ms = tot;
+  return XQ_OK;
+}
+
+int xq_last_cuda_error(const xq_cache* c) { return c ? c->last_cuda : 0; }
+
+const char* xq_strerror(int code) {
+  switch (code) {
+    case XQ_OK: return "ok";
+    case XQ_ERR_CONFIG: return "invalid configuration";
+    case XQ_ERR_ARG: return "invalid argument";
+    case XQ_ERR_CAPACITY: return "capacity exceeded";
+    case XQ_ERR_ORDER: return "code-owning layer is behind the layer that borrows its codes";
+    case XQ_ERR_CUDA: return "CUDA error (see xq_last_cuda_error)";
+    case XQ_ERR_NOMEM: return "out of host memory";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

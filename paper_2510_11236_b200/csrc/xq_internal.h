@@ -1,0 +1,78 @@
+// Internal declarations shared by the host state machine and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace xq {
+
+struct Dims {
+  int B, Hq, Hkv, G, D, g, R, NG;
+  int nq_cap;  // capacity of the quantized region in tokens (multiple of R)
+};
+
+// Device addresses of one layer's regions (codes: of the layer that owns them).
+struct LayerPtrs {
+  uint16_t* win_k;   // [B,Hkv,R,D] bf16
+  uint16_t* win_v;
+  uint16_t* k_meta;  // [B,Hkv,nq_cap/g,2,D] fp16
+  uint16_t* v_meta;  // [B,Hkv,nq_cap/16,2,16*NG] fp16
+  uint32_t* k_codes; // [B,Hkv,nq_cap*D*bk/32]
+  uint32_t* v_codes;
+  int bk, bv;
+};
+
+struct PackParams {
+  Dims dm;
+  LayerPtrs L;
+  const uint16_t* K_in;  // [B,Hkv,n_in,D] new tokens (absolute positions s_old ..)
+  const uint16_t* V_in;
+  int n_in;
+  int s_old;     // tokens cached before this append
+  int nq_old;    // quantized tokens before this append
+  int n_blocks;  // R-token blocks to quantize, starting at absolute token nq_old
+  int own_k, own_v;
+  float eta_k, eta_v;
+  int tb;        // tokens per CTA tile (32 or 64)
+};
+
+struct WindowParams {
+  Dims dm;
+  LayerPtrs L;
+  const uint16_t* K_in;
+  const uint16_t* V_in;
+  int n_in;
+  int s_old;
+  int first;   // first absolute token to copy
+  int count;   // tokens to copy
+  int nq_new;  // window slot = absolute token - nq_new
+};
+
+struct DecodeParams {
+  Dims dm;
+  LayerPtrs L;
+  const uint16_t* q;  // [B,Hq,D] bf16
+  int n_q;            // quantized tokens
+  int r;              // window tokens
+  int ns_q, ns_w;     // splits over the quantized region / over the window
+  float scale;
+  float* part_acc;    // [B,Hq,ns,D]
+  float* part_ml;     // [B,Hq,ns,2]  (running max in log2 units, sum)
+};
+
+struct MergeParams {
+  Dims dm;
+  int ns;
+  const float* part_acc;
+  const float* part_ml;
+  void* out;
+  int out_f32;
+};
+
+cudaError_t launch_pack(const PackParams& p, cudaStream_t st);
+cudaError_t launch_window_append(const WindowParams& p, cudaStream_t st);
+cudaError_t launch_decode_generic(const DecodeParams& p, cudaStream_t st);
+cudaError_t launch_decode_mma(const DecodeParams& p, cudaStream_t st);
+bool decode_mma_supported(const Dims& dm, int bk, int bv);
+cudaError_t launch_merge(const MergeParams& p, cudaStream_t st);
+
+}  // namespace xq

@@ -1,0 +1,185 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2510_11236_b200 as xq
+from paper_2510_11236_b200 import workloads as W
+from tests import util
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+KERNELS = [xq.XQ_KERNEL_GENERIC, xq.XQ_KERNEL_AUTO]
+
+
+def _fill(cache, w, layers, S, step=None):
+    """Append tokens [0, S) of the synthetic workload to `layers`; returns {layer: (K, V)}."""
+    kv = {}
+    for pair in sorted({l // 2 for l in layers}):
+        k0, v0, k1, v1 = W.pair_tokens(w, pair, 0, S, DEV)
+        if 2 * pair in layers:
+            kv[2 * pair] = (k0, v0)
+        if 2 * pair + 1 in layers:
+            kv[2 * pair + 1] = (k1, v1)
+    for l in sorted(layers):
+        K, V = kv[l]
+        if step is None:
+            cache.append_kv(l, K, V)
+        else:
+            for lo in range(0, S, step):
+                hi = min(S, lo + step)
+                cache.append_kv(l, K[:, :, lo:hi].contiguous(), V[:, :, lo:hi].contiguous())
+    torch.cuda.synchronize()
+    return kv
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("etas", [(0.0, 0.0), (1 / 6, 0.045)])
+def test_config0_full(kernel, etas):
+    w = W.CONFIGS["c0"]
+    cfg = W.make_xq_config(w, eta1=etas[0], eta2=etas[1], kernel=kernel)
+    cache = xq.Cache(cfg, DEV)
+    kv = _fill(cache, w, [0, 1], w["seq"])
+    assert cache.seq_len(0) == 512 and cache.quantized_len(1) == 480
+    worst = 0.0
+    for l in (0, 1):
+        q = W.queries(w, l, 0, DEV)
+        o32 = cache.decode_attention(l, q, f32=True)
+        o16 = cache.decode_attention(l, q)
+        torch.cuda.synchronize()
+        for hk in range(w["n_kv_heads"]):
+            oc = util.oracle_for_stream(cfg, [0, 1], 0, hk, kv)
+            util.compare_regions(cache, oc, l, 0, hk)
+            worst = max(worst, util.check_attention(cache, oc, l, q, 0, hk, o32, o16))
+    assert xq.xq_equiv_bits(cfg) == 1.0
+    print("config 0 worst fp32 attention error", worst)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("shape", [
+    # (L, B, Hq, Hkv, D, g, R, kq, vq, km, vm, S)
+    (4, 2, 8, 2, 128, 32, 64, 2, 0, 2, 0, 200),    # GQA 4, 2-bit and 1-bit layers, keys shared only from layer 2
+    (2, 1, 8, 1, 128, 64, 64, 2, 2, 0, 0, 331),    # group 64, GQA 8
+    (2, 2, 2, 2, 128, 32, 128, 0, 0, 0, 0, 700),   # MHA, all 1-bit
+    (2, 1, 6, 2, 64, 32, 64, 0, 2, 0, 2, 260),     # head_dim 64, 1-bit keys, values not shared, GQA 3
+    (2, 1, 12, 1, 128, 32, 32, 2, 2, 2, 2, 100),   # GQA 12 (> 8 heads per group), no sharing
+])
+def test_mixed_shapes(kernel, shape):
+    L, B, Hq, Hkv, D, g, R, kq, vq, km, vm, S = shape
+    w = dict(n_layers=L, batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, seq=S, residual_len=R,
+             group_size=g, kq=kq, vq=vq, km=km, vm=vm, n_outliers=3, outlier_scale=10.0, seed=11, n_splits=0)
+    cfg = W.make_xq_config(w, kernel=kernel)
+    assert xq.xq_config_check(cfg) == 0
+    cache = xq.Cache(cfg, DEV)
+    layers = list(range(L))
+    kv = _fill(cache, w, layers, S, step=97)
+    for l in layers:
+        q = W.queries(w, l, 0, DEV)
+        o32 = cache.decode_attention(l, q, f32=True)
+        o16 = cache.decode_attention(l, q)
+        torch.cuda.synchronize()
+        for b in range(B):
+            for hk in range(Hkv):
+                oc = util.oracle_for_stream(cfg, layers, b, hk, kv)
+                util.compare_regions(cache, oc, l, b, hk)
+                util.check_attention(cache, oc, l, q, b, hk, o32, o16)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("S", [1, 5, 16, 31, 32, 33, 64, 65])
+def test_short_sequences(kernel, S):
+    # S <= R: nothing is quantized and the result is plain 16-bit attention; S = R + 1: first flush
+    w = dict(W.CONFIGS["c0"], seq=S)
+    cfg = W.make_xq_config(w, kernel=kernel)
+    cache = xq.Cache(cfg, DEV)
+    kv = _fill(cache, w, [0, 1], S)
+    r = ((S - 1) % 32) + 1
+    assert cache.quantized_len(0) == S - r
+    q = W.queries(w, 1, 0, DEV)
+    o32 = cache.decode_attention(1, q, f32=True)
+    torch.cuda.synchronize()
+    for hk in range(4):
+        oc = util.oracle_for_stream(cfg, [0, 1], 0, hk, kv)
+        util.compare_regions(cache, oc, 1, 0, hk)
+        util.check_attention(cache, oc, 1, q, 0, hk, o32)
+    if S <= 32:
+        # exact 16-bit attention (fp64 on the raw inputs)
+        K, V = kv[1]
+        ref = torch.softmax((q[0].double()[:, None, :] * K[0].double()).sum(-1) / 8.0, dim=-1)
+        ref = (ref[:, :, None] * V[0].double()).sum(1)
+        assert (o32[0].double() - ref).abs().max().item() <= 2e-3
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_append_granularity_and_split_invariance(kernel):
+    w = dict(W.CONFIGS["c0"], seq=300, n_kv_heads=2, n_q_heads=4)
+    outs = []
+    regions = []
+    for step, ns in ((None, 0), (1, 1), (37, 7), (128, 64)):
+        cfg = W.make_xq_config(w, kernel=kernel, n_splits=ns)
+        cache = xq.Cache(cfg, DEV)
+        _fill(cache, w, [0, 1], 300, step=step)
+        q = W.queries(w, 1, 3, DEV)
+        outs.append(cache.decode_attention(1, q, f32=True).clone())
+        nq = cache.quantized_len(1)
+        regions.append([cache.region(1, k).clone() for k in range(6)])
+        torch.cuda.synchronize()
+    for o in outs[1:]:
+        assert (o - outs[0]).abs().max().item() <= 2e-5
+    D = 64
+    used = {0: 288 * D * 2 // 8, 1: 288 * D * 2 // 8, 2: (288 // 32) * 2 * D * 2, 3: (288 // 16) * 2 * 16 * 2 * 2,
+            4: 12 * D * 2, 5: 12 * D * 2}
+    for rg in regions[1:]:
+        for k in range(6):
+            assert torch.equal(rg[k][:, : used[k]], regions[0][k][:, : used[k]])
+
+
+def test_error_paths():
+    w = dict(W.CONFIGS["c0"], seq=100)
+    cfg = W.make_xq_config(w, max_seq=100)
+    cache = xq.Cache(cfg, DEV)
+    k0, v0, k1, v1 = W.pair_tokens(w, 0, 0, 100, DEV)
+    q = W.queries(w, 0, 0, DEV)
+    out = torch.empty_like(q)
+    s = torch.cuda.current_stream().cuda_stream
+    assert xq.xq_decode_attention(cache.handle, 0, q, out, s) == xq.XQ_ERR_ARG  # empty layer
+    assert xq.xq_append_kv(cache.handle, 1, k1, v1, 100, s) == 0
+    # layer 1 borrows layer 0's codes, and layer 0 is still empty
+    assert xq.xq_decode_attention(cache.handle, 1, q, out, s) == xq.XQ_ERR_ORDER
+    assert xq.xq_append_kv(cache.handle, 0, k0, v0, 100, s) == 0
+    assert xq.xq_decode_attention(cache.handle, 1, q, out, s) == 0
+    assert xq.xq_append_kv(cache.handle, 0, k0, v0, 1, s) == xq.XQ_ERR_CAPACITY
+    assert xq.xq_seq_len(cache.handle, 0) == 100
+    assert xq.xq_append_kv(cache.handle, 5, k0, v0, 1, s) == xq.XQ_ERR_ARG
+    assert xq.xq_append_kv(cache.handle, 0, k0, v0, 0, s) == xq.XQ_ERR_ARG
+    assert xq.xq_append_kv(cache.handle, 0, None, v0, 1, s) == xq.XQ_ERR_ARG
+    assert xq.xq_append_kv(cache.handle, 0, k0.data_ptr() + 2, v0, 1, s) == xq.XQ_ERR_ARG
+    torch.cuda.synchronize()
+    assert xq.xq_reset(cache.handle) == 0 and xq.xq_seq_len(cache.handle, 0) == 0
+
+
+def test_decode_step_device_and_host():
+    w = dict(W.CONFIGS["c0"], seq=64)
+    cfg = W.make_xq_config(w, max_seq=128)
+    a, b = xq.Cache(cfg, DEV), xq.Cache(cfg, DEV)
+    _fill(a, w, [0, 1], 64)
+    _fill(b, w, [0, 1], 64)
+    L, B, Hq, Hkv, D = 2, 1, 4, 4, 64
+    for step in range(3):  # the first step flushes the full window
+        kn = torch.randn(L, B, Hkv, 1, D, device=DEV).to(torch.bfloat16)
+        vn = torch.randn(L, B, Hkv, 1, D, device=DEV).to(torch.bfloat16)
+        q = torch.randn(L, B, Hq, D, device=DEV).to(torch.bfloat16)
+        out_d = torch.empty_like(q)
+        a.decode_step(kn, vn, q, out_d)
+        kh, vh, qh = kn.cpu().pin_memory(), vn.cpu().pin_memory(), q.cpu().pin_memory()
+        out_h = torch.empty(L, B, Hq, D, dtype=torch.bfloat16).pin_memory()
+        b.decode_step(kh, vh, qh, out_h, mem=xq.XQ_MEM_HOST)
+        torch.cuda.synchronize()
+        assert torch.equal(out_d.cpu(), out_h)
+        # and equal to the per-layer calls
+        for l in range(L):
+            assert a.seq_len(l) == 65 + step
+            ref = a.decode_attention(l, q[l])
+            assert torch.equal(ref, out_d[l])
+    assert xq.xq_launch_count(a.handle) > 0
