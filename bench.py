@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of the hot path: decode steps over an XQuant KV cache at 32k context.
+
+One step = one generated token of a whole model: for each of the 32 layers,
+append the token's K,V (window append; quantize-and-pack whenever a window block
+fills) and run decode attention over the packed cache plus the window.  The
+metric is decode-attention GB/s: the bytes the method itself must move per
+layer call (packed codes, fp16 scale / zero-point, 16-bit window, q, out)
+divided by time.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config c2] [--impl ours|reference]
+
+With N > 1 (launched by torchrun) every rank runs the same workload on its own
+GPU -- sequences are independent, so the path shards by batch with no
+collective -- and the aggregate is reported (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode-attention GB/s at 32k ctx"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while a region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        clocks, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                clocks.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if clocks:
+            out["sm_mhz"] = statistics.median(clocks)
+            out["sm_max_mhz"] = max(mx)
+            out["samples"] = len(clocks)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+class OracleSample:
+    """The CPU oracle, as it stands, on a bounded sample of the workload: decode
+    attention of one layer for `n_streams` (sequence, kv head) streams at the full
+    context (dequantize the stream's packed region in fp64, then attention for
+    its query heads).  Building the streams' caches is set-up, not timed."""
+
+    def __init__(self, w, n_streams, eta1, eta2):
+        import numpy as np
+        import torch
+        from oracle import xq_oracle as O
+        from paper_2510_11236_b200 import workloads as W
+        from tests import util
+        S = w["seq"]
+        G = w["n_q_heads"] // w["n_kv_heads"]
+        self.n_streams = n_streams
+        k0, v0, _, _ = W.pair_tokens(dict(w, batch=1, n_kv_heads=n_streams), 0, 0, S, "cpu")
+        self.caches = []
+        for s in range(n_streams):
+            oc = O.OracleCache(1, 1, G, 1, w["head_dim"], w["group_size"], w["residual_len"],
+                               1 if w["kq"] > 0 else 0, 1 if w["vq"] > 0 else 0, 1, 1,
+                               np.float32(eta1), np.float32(eta2))
+            oc.append(0, util.bits_of(k0[:, s:s + 1]), util.bits_of(v0[:, s:s + 1]))
+            self.caches.append(oc)
+        gen = torch.Generator().manual_seed(5)
+        self.q = util.bits_of(torch.randn(1, G, w["head_dim"], generator=gen).to(torch.bfloat16))
+        self.bytes = n_streams * W.algorithmic_bytes(dict(w, batch=1, n_kv_heads=1, n_q_heads=G), S, 0)
+        self.cores = 1
+
+    def run(self):
+        """Seconds for one pass over the sample, single-threaded."""
+        try:
+            from threadpoolctl import threadpool_limits
+        except Exception:  # pragma: no cover
+            threadpool_limits = None
+        t0 = time.perf_counter()
+        if threadpool_limits is not None:
+            with threadpool_limits(limits=1):
+                for oc in self.caches:
+                    oc.decode(0, self.q)
+        else:
+            for oc in self.caches:
+                oc.decode(0, self.q)
+        return time.perf_counter() - t0
+
+
+def run_reference(args, w):
+    """The reference arm: the CPU oracle timed on this machine's host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_streams = 2
+    smp = OracleSample(w, n_streams, args.eta1, args.eta2)
+    times = []
+    for i in range(args.warmup + args.steps):
+        dt = smp.run()
+        if i >= args.warmup:
+            times.append(dt)
+    T = sum(times) / len(times)
+    val = smp.bytes / T / 1e9
+    sample = (f"decode attention of one layer for {n_streams} of {w['batch'] * w['n_kv_heads']} (sequence, kv head) "
+              f"streams at S={w['seq']} per step (dequantize + attention, fp64 numpy)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": T * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.config, **{k: w[k] for k in ("n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "seq", "residual_len", "group_size", "kq", "vq", "km", "vm")}},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="c2")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--eta1", type=float, default=1.0 / 6.0)
+    ap.add_argument("--eta2", type=float, default=0.045)
+    ap.add_argument("--kernel", type=int, default=0)
+    ap.add_argument("--splits", type=int, default=None)
+    ap.add_argument("--layer-order", default="owners_first", choices=["owners_first", "ascending"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2510_11236_b200 import workloads as W
+    w = dict(W.CONFIGS[args.config])
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2510_11236_b200 as xq
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    w["seed"] = w["seed"] + 101 * rank  # every rank holds its own sequences
+
+    L, B, Hq, Hkv, D, S = w["n_layers"], w["batch"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"], w["seq"]
+    K, Wm = args.steps, args.warmup
+    n_total = Wm + 3 * K + 8  # warm-up, then three timed passes (device, per-kernel events, host buffers)
+    cfg = W.make_xq_config(w, max_seq=S + n_total + 1, eta1=args.eta1, eta2=args.eta2, kernel=args.kernel,
+                           n_splits=args.splits)
+    cache = xq.Cache(cfg, dev)
+
+    # ---- prefill to S - warmup tokens, so that the warm-up steps end at S and the first timed step
+    # ---- quantizes the full window of every layer
+    S0 = max(1, S - Wm)
+    for pair in range(L // 2):
+        for c0 in range(0, S0, W.CHUNK):
+            c1 = min(S0, c0 + W.CHUNK)
+            k0, v0, k1, v1 = W.pair_tokens(w, pair, c0, c1, dev)
+            cache.append_kv(2 * pair, k0, v0)
+            cache.append_kv(2 * pair + 1, k1, v1)
+    torch.cuda.synchronize()
+
+    # ---- per-step inputs (distinct every step), on the device and in pinned host memory
+    g = torch.Generator(device=dev).manual_seed(1234 + rank)
+    n_pool = min(n_total, 64)
+    pool = []
+    for i in range(n_pool):
+        kn = torch.randn(L, B, Hkv, 1, D, generator=g, device=dev).to(torch.bfloat16)
+        vn = torch.randn(L, B, Hkv, 1, D, generator=g, device=dev).to(torch.bfloat16)
+        qn = torch.randn(L, B, Hq, D, generator=g, device=dev).to(torch.bfloat16)
+        pool.append((kn, vn, qn))
+    host_pool = [(a.cpu().pin_memory(), b.cpu().pin_memory(), c.cpu().pin_memory()) for a, b, c in pool[:8]]
+    out_dev = torch.empty(L, B, Hq, D, dtype=torch.bfloat16, device=dev)
+    out_host = torch.empty(L, B, Hq, D, dtype=torch.bfloat16).pin_memory()
+    order = None
+    if args.layer_order == "owners_first":
+        order = list(range(0, L, 2)) + list(range(1, L, 2))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    step_no = [0]
+
+    def device_step():
+        kn, vn, qn = pool[step_no[0] % n_pool]
+        step_no[0] += 1
+        cache.decode_step(kn, vn, qn, out_dev, order)
+
+    def step_bytes(first_seq, n_steps):
+        tot = 0
+        for i in range(n_steps):
+            for l in range(L):
+                tot += W.algorithmic_bytes(w, first_seq + i, l)
+        return tot
+
+    for _ in range(Wm):
+        device_step()
+    barrier()
+
+    # ---- pass 1: whole steps, inputs resident in HBM
+    seq_before = cache.seq_len(0)
+    launches_before = xq.xq_launch_count(cache.handle)
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(K):
+        device_step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+    launches = xq.xq_launch_count(cache.handle) - launches_before
+    bytes_pass1 = step_bytes(seq_before + 1, K)
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+    value = world * bytes_pass1 / (ms_max * 1e-3) / 1e9
+    tokens_per_s = world * B * sum(seq_before + 1 + i for i in range(K)) * L / (ms_max * 1e-3) / L
+
+    # ---- pass 2: the same steps with CUDA events around every kernel (roofline of the dominant kernel)
+    xq.xq_timing_enable(cache.handle, 1)
+    seq_before2 = cache.seq_len(0)
+    barrier()
+    for _ in range(K):
+        device_step()
+    barrier()
+    kinds = {}
+    for kind, name in enumerate(("decode_split", "merge", "quantize_pack", "window_append")):
+        rc, n, tot = xq.xq_timing_read(cache.handle, kind)
+        kinds[name] = {"launches": n, "total_ms": tot, "avg_us": (tot / n * 1e3) if n else None}
+    xq.xq_timing_enable(cache.handle, 0)
+    dec = kinds["decode_split"]
+    bytes_pass2 = step_bytes(seq_before2 + 1, K)
+    peak, peak_kind = _peaks()
+    achieved = bytes_pass2 / (dec["total_ms"] * 1e-3) / 1e9 if dec["launches"] else 0.0
+
+    # ---- pass 3: end to end through the C ABI with host buffers
+    seq_before3 = cache.seq_len(0)
+    h2d = sum(x.numel() * 2 for x in host_pool[0])
+    d2h = out_host.numel() * 2
+    stream = torch.cuda.current_stream()
+    barrier()
+    t0 = time.perf_counter()
+    e0.record()
+    for i in range(K):
+        kn, vn, qn = host_pool[i % len(host_pool)]
+        cache.decode_step(kn, vn, qn, out_host, order, mem=xq.XQ_MEM_HOST)
+        stream.synchronize()  # the host reads the step's result
+    e1.record()
+    barrier()
+    ms3 = e0.elapsed_time(e1)
+    t = torch.tensor([ms3], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_val = world * step_bytes(seq_before3 + 1, K) / (float(t.item()) * 1e-3) / 1e9
+
+    if rank == 0:
+        nsq = nsw = None
+        rc, nsq, nsw = xq.xq_split_plan(cache.handle, 0)
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f16 mma operands, f32 accumulate, bf16 io", "data": "synthetic",
+            "config": {"workload": f"{args.config}: BASELINE.json configs[{args.config[1:]}]",
+                       **{k: w[k] for k in ("n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "seq",
+                                            "residual_len", "group_size", "kq", "vq", "km", "vm")},
+                       "eta1": args.eta1, "eta2": args.eta2, "equiv_bits": xq.xq_equiv_bits(cfg),
+                       "step": "per layer: append 1 token (+ quantize-and-pack when the window block fills) and decode attention",
+                       "layer_order": args.layer_order,
+                       "l2": "inputs larger than L2: each step streams ~%.1f GB of cache; owners-first layer order keeps a pair's shared codes from being re-served by L2" % (bytes_pass1 / K / 1e9),
+                       "splits_quantized": nsq, "splits_window": nsw,
+                       "algorithmic_bytes_per_layer_call": W.algorithmic_bytes(w, S, 0)},
+            "frac_of_8TBps": value / world / 8000.0,
+            "frac_of_measured_hbm": value / world / peak,
+            "attended_tokens_per_s": tokens_per_s,
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "e2e": {"value": e2e_val, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": float(t.item()) / K},
+            "roofline": {"bound": "hbm", "kernel": "decode split kernel", "achieved": achieved, "peak": peak,
+                         "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                         "frac_of_8TBps": achieved / 8000.0, "traffic": None,
+                         "avg_launch_us": dec["avg_us"], "launches": dec["launches"]},
+            "kernels": kinds,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            n_streams = min(B * Hkv, 32)
+            smp = OracleSample(w, n_streams, args.eta1, args.eta2)
+            dt = smp.run()
+            line["cpu_baseline"] = {
+                "value": smp.bytes / dt / 1e9, "unit": "GB/s", "cores": smp.cores, "kind": "oracle",
+                "sample": f"decode attention of one layer for {n_streams} of {B * Hkv} (sequence, kv head) streams at S={S} "
+                          f"(dequantize + attention, fp64 numpy), {dt:.1f} s"}
+        print(json.dumps(line), flush=True)
+    cache.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -130,16 +130,19 @@ int xq_decode_attention(xq_cache* c, int layer, const void* q, void* out, void* 
  * head_dim] (the accumulator before the final rounding to bfloat16). */
 int xq_decode_attention_f32(xq_cache* c, int layer, const void* q, float* out, void* stream);
 
-/* One decode step of a whole model: for each layer l in ascending order, append
- * one token and run decode attention.  K_new, V_new: [n_layers, batch,
- * n_kv_heads, 1, head_dim]; q, out: [n_layers, batch, n_q_heads, head_dim];
- * bfloat16.  mem = XQ_MEM_DEVICE: device pointers, used in place.
+/* One decode step of a whole model: for each layer, append one token and run
+ * decode attention.  K_new, V_new: [n_layers, batch, n_kv_heads, 1, head_dim];
+ * q, out: [n_layers, batch, n_q_heads, head_dim]; bfloat16; slice l belongs to
+ * layer l.  layer_order: host array of n_layers distinct layer indices giving
+ * the order in which layers are processed, or NULL for ascending order; a
+ * code-owning layer must come before the layer that borrows its codes.
+ * mem = XQ_MEM_DEVICE: device pointers, used in place.
  * mem = XQ_MEM_HOST: host pointers (pinned memory for the copies to be
  * asynchronous); inputs are copied to the workspace's staging area on `stream`,
  * the result is copied back to `out` on `stream`; the caller synchronizes the
  * stream before reading `out` or reusing the host buffers. */
 int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void* q, void* out,
-                   int mem, void* stream);
+                   const int32_t* layer_order, int mem, void* stream);
 
 /* Equivalent bit-width of Appendix C: stored code bits per cached element,
  * averaged over layers and over keys and values; scale / zero-point excluded,
@@ -159,7 +162,7 @@ int xq_split_plan(const xq_cache* c, int layer, int* n_splits_quantized, int* n_
  * offset from the workspace start and the byte stride between consecutive
  * (sequence, kv head) streams.
  * Layouts (all little-endian, one stream per (sequence, kv head)):
- *   codes: tiles of 128 uint32; see DESIGN notes in xq_layout.cuh for the bit map;
+ *   codes: tiles of 128 uint32 (bit map: csrc/xq_layout.cuh);
  *   key scale/zero: per token group [2][head_dim] fp16 (scale block, zero block),
  *     permuted within the block; value scale/zero: per 16 tokens
  *     [2][16*head_dim/group_size] fp16; windows: [R][head_dim] bfloat16. */

@@ -46,7 +46,8 @@ _SIGNATURES = {
     "xq_decode_attention_f32": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
                                                ctypes.c_void_p]),
     "xq_decode_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
-                                      ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]),
+                                      ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.c_int,
+                                      ctypes.c_void_p]),
     "xq_equiv_bits": (ctypes.c_double, [ctypes.POINTER(xq_config)]),
     "xq_seq_len": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
     "xq_quantized_len": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
@@ -135,8 +136,11 @@ def xq_decode_attention_f32(handle, layer: int, q, out, stream: int = 0) -> int:
     return lib().xq_decode_attention_f32(handle, layer, _ptr(q), _ptr(out), stream)
 
 
-def xq_decode_step(handle, K_new, V_new, q, out, mem: int = XQ_MEM_DEVICE, stream: int = 0) -> int:
-    return lib().xq_decode_step(handle, _ptr(K_new), _ptr(V_new), _ptr(q), _ptr(out), mem, stream)
+def xq_decode_step(handle, K_new, V_new, q, out, layer_order=None, mem: int = XQ_MEM_DEVICE, stream: int = 0) -> int:
+    order = None
+    if layer_order is not None:
+        order = (ctypes.c_int32 * len(layer_order))(*layer_order)
+    return lib().xq_decode_step(handle, _ptr(K_new), _ptr(V_new), _ptr(q), _ptr(out), order, mem, stream)
 
 
 def xq_equiv_bits(cfg: xq_config) -> float:
@@ -248,8 +252,8 @@ class Cache:
             raise XQError(rc, "xq_decode_attention")
         return out
 
-    def decode_step(self, K_new, V_new, q, out, mem=XQ_MEM_DEVICE):
-        rc = xq_decode_step(self.handle, K_new, V_new, q, out, mem, self._stream())
+    def decode_step(self, K_new, V_new, q, out, layer_order=None, mem=XQ_MEM_DEVICE):
+        rc = xq_decode_step(self.handle, K_new, V_new, q, out, layer_order, mem, self._stream())
         if rc:
             raise XQError(rc, "xq_decode_step")
         return out

@@ -364,10 +364,20 @@ int xq_decode_attention_f32(xq_cache* c, int layer, const void* q, float* out, v
   return decode_impl(c, layer, q, out, 1, (cudaStream_t)stream);
 }
 
-int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void* q, void* out, int mem,
-                   void* stream) {
+int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void* q, void* out,
+                   const int32_t* layer_order, int mem, void* stream) {
   if (!c || !K_new || !V_new || !q || !out) return XQ_ERR_ARG;
   if (mem != XQ_MEM_DEVICE && mem != XQ_MEM_HOST) return XQ_ERR_ARG;
+  if (layer_order) {
+    std::vector<char> seen(c->cfg.n_layers, 0);
+    for (int i = 0; i < c->cfg.n_layers; ++i) {
+      int l = layer_order[i];
+      if (l < 0 || l >= c->cfg.n_layers || seen[l]) return XQ_ERR_ARG;
+      bool borrows = !owns_codes(l, c->cfg.km) || !owns_codes(l, c->cfg.vm);
+      if (borrows && !seen[l - 1]) return XQ_ERR_ORDER;
+      seen[l] = 1;
+    }
+  }
   cudaStream_t st = (cudaStream_t)stream;
   const Dims& dm = c->plan.dm;
   const int L = c->cfg.n_layers;
@@ -387,7 +397,8 @@ int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void
     if (e != cudaSuccess) return fail_cuda(c, e);
     dk = sk; dv = sv; dq = sq; dout = so;
   }
-  for (int l = 0; l < L; ++l) {
+  for (int i = 0; i < L; ++i) {
+    const int l = layer_order ? layer_order[i] : i;
     int rc = xq_append_kv(c, l, dk + l * kv_layer, dv + l * kv_layer, 1, stream);
     if (rc != XQ_OK) return rc;
     rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st);
