@@ -1,6 +1,513 @@
-// Tensor-core decode kernel (placeholder until the kernel lands).
+// Tensor-core decode attention over the packed cache (head_dim 128, up to 8
+// query heads per kv head).
+//
+// Why mma.sync from registers and not tcgen05: the packed cache delivers
+// ~1.8e13 quantized elements/s at the HBM roofline.  tcgen05.mma takes its
+// operands from shared memory (or TMEM), so every dequantized element would
+// have to be written to and read back from on-chip memory at 2 bytes each --
+// more than the SMs' shared-memory bandwidth.  Here the codes never leave
+// registers in dequantized form: the packed word layout is the A-fragment
+// layout of mma.sync.m16n8k16, so `word & mask` IS an fp16x2 operand register
+// (the code sits in the mantissa bits of an fp16 subnormal: value c * 2^(pos-24)),
+// and scale / zero-point are folded into the other operand:
+//
+//   q . k_hat_t = sum_d (q_d s_d) c_td + sum_d q_d z_d        (keys, per channel)
+//   sum_t p_t v_hat_td = sum_t (p_t s_tg) c_td + sum_t p_t z_tg  (values, per token)
+//
+// Tokens are the M dimension of both products (S^T = Kc * Q'^T, O^T = Vc^T * P'),
+// so a GQA group of up to 8 query heads fills the N = 8 columns.
+//
+// Work split: grid (split, kv head, sequence).  The first ns_w splits take the
+// 16-bit window (scalar path, 16 tokens per tile); the remaining ns_q splits take
+// ranges of 32-token units of the packed region.  In a packed split the 4 warps
+// interleave units; each warp stages its own units in shared memory with
+// cp.async (NST stages ahead) and keeps a private online softmax; the warps'
+// states are merged at the end and the CTA writes one partial per query head.
+#include <cuda_fp16.h>
+#include <math_constants.h>
+
 #include "xq_internal.h"
+
 namespace xq {
-bool decode_mma_supported(const Dims&, int, int) { return false; }
-cudaError_t launch_decode_mma(const DecodeParams&, cudaStream_t) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int MMA_WARPS = 4;
+constexpr int MMA_THREADS = MMA_WARPS * 32;
+constexpr int NST = 4;  // cp.async stages per warp
+constexpr int HD = 128;
+
+__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(d) : "r"(a));
+  return d;
+}
+
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+  uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+}
+
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ uint32_t hmul2_u(uint32_t a, uint32_t b) {
+  __half2 r = __hmul2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<__half2*>(&b));
+  return *reinterpret_cast<uint32_t*>(&r);
+}
+__device__ __forceinline__ float bf16_to_f(uint16_t u) { return __uint_as_float(((uint32_t)u) << 16); }
+
+// Slot s (0..7) of a word holds, per 16-bit half, a BITS-bit code at bit BITS*s
+// (1-bit words carry a second sub-tile in slots 8..15, reached by a shift of 8).
+// Slots whose bits fall outside the fp16 mantissa are reached by one shift.
+template <int BITS>
+struct Slots;
+template <>
+struct Slots<2> {
+  static constexpr int SHIFT = 10;                                   // slots 5..7 -> bit 0, 2, 4
+  __host__ __device__ static constexpr int e(int s) { return s < 5 ? 2 * s : 2 * (s - 5); }  // log2 weight
+  __device__ static constexpr uint32_t mask(int s) { return 0x00030003u << e(s); }
+  __device__ static constexpr bool shifted(int s) { return s >= 5; }
+};
+template <>
+struct Slots<1> {
+  static constexpr int SHIFT = 8;  // second sub-tile
+  __host__ __device__ static constexpr int e(int s) { return s; }
+  __device__ static constexpr uint32_t mask(int s) { return 0x00010001u << s; }
+  __device__ static constexpr bool shifted(int) { return false; }
+};
+
+template <int BK, int BV, int GS>
+struct Stage {
+  static constexpr int NG = HD / GS;
+  static constexpr int KC = 512 * BK;  // key codes of one 32-token unit
+  static constexpr int KS = 256;       // key scale block of the unit's token group
+  static constexpr int VC = 512 * BV;
+  static constexpr int VM = 128 * NG;  // value scale + zero blocks of the unit's two 16-token tiles
+  static constexpr int OFF_KS = KC;
+  static constexpr int OFF_VC = KC + KS;
+  static constexpr int OFF_VM = KC + KS + VC;
+  static constexpr int BYTES = KC + KS + VC + VM;
+};
+
+constexpr int MS = HD + 4;  // merge-buffer row: acc[HD], m, l, padding (keeps rows 16-byte aligned)
+constexpr int MERGE_BYTES = MMA_WARPS * 8 * MS * 4;
+
+template <int BK, int BV, int GS>
+constexpr int smem_bytes() {
+  int pipe = MMA_WARPS * NST * Stage<BK, BV, GS>::BYTES + 32 * 64;  // stages + q in B-operand layout
+  return pipe > MERGE_BYTES ? pipe : MERGE_BYTES;
+}
+
+// ---------------------------------------------------------------------------
+// window path: plain fp32 over 16-bit tokens, one token per warp iteration
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void window_split(const DecodeParams& p, int sw, int hk, int b, float* smem_f) {
+  const Dims& dm = p.dm;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = b * dm.Hkv + hk;
+  const int G = dm.G;
+  const int tiles = (p.r + 15) / 16;
+  const int t0 = (int)(((long long)sw * tiles) / p.ns_w) * 16;
+  const int t1 = min((int)(((long long)(sw + 1) * tiles) / p.ns_w) * 16, p.r);
+  const uint16_t* wk = p.L.win_k + (size_t)bh * dm.R * HD;
+  const uint16_t* wv = p.L.win_v + (size_t)bh * dm.R * HD;
+  const float scale2 = p.scale * 1.4426950408889634f;
+  float q[8][4], acc[8][4], m[8], l[8];
+#pragma unroll
+  for (int a = 0; a < 8; ++a) {
+    m[a] = -CUDART_INF_F;
+    l[a] = 0.f;
+    const uint16_t* qp = p.q + ((size_t)b * dm.Hq + hk * G + (a < G ? a : 0)) * HD + lane * 4;
+    uint2 raw = *reinterpret_cast<const uint2*>(qp);
+    q[a][0] = bf16_to_f(raw.x & 0xffff); q[a][1] = bf16_to_f(raw.x >> 16);
+    q[a][2] = bf16_to_f(raw.y & 0xffff); q[a][3] = bf16_to_f(raw.y >> 16);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[a][j] = 0.f;
+  }
+  for (int t = t0 + warp; t < t1; t += MMA_WARPS) {
+    uint2 kr = *reinterpret_cast<const uint2*>(wk + (size_t)t * HD + lane * 4);
+    uint2 vr = *reinterpret_cast<const uint2*>(wv + (size_t)t * HD + lane * 4);
+    float kx[4] = {bf16_to_f(kr.x & 0xffff), bf16_to_f(kr.x >> 16), bf16_to_f(kr.y & 0xffff), bf16_to_f(kr.y >> 16)};
+    float vx[4] = {bf16_to_f(vr.x & 0xffff), bf16_to_f(vr.x >> 16), bf16_to_f(vr.y & 0xffff), bf16_to_f(vr.y >> 16)};
+#pragma unroll
+    for (int a = 0; a < 8; ++a) {
+      if (a < G) {
+        float dot = q[a][0] * kx[0];
+        dot = fmaf(q[a][1], kx[1], dot);
+        dot = fmaf(q[a][2], kx[2], dot);
+        dot = fmaf(q[a][3], kx[3], dot);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        float x = dot * scale2;
+        float mn = fmaxf(m[a], x);
+        float corr = exp2f(m[a] - mn);
+        float pe = exp2f(x - mn);
+        l[a] = l[a] * corr + pe;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[a][j] = acc[a][j] * corr + pe * vx[j];
+        m[a] = mn;
+      }
+    }
+  }
+  // merge buffer: [warp][head][MS]
+  float* mb = smem_f + (size_t)warp * 8 * MS;
+#pragma unroll
+  for (int a = 0; a < 8; ++a) {
+    if (a < G) {
+      float* row = mb + a * MS;
+      *reinterpret_cast<float4*>(row + lane * 4) = make_float4(acc[a][0], acc[a][1], acc[a][2], acc[a][3]);
+      if (lane == 0) {
+        row[HD] = m[a];
+        row[HD + 1] = l[a];
+      }
+    }
+  }
+}
+
+// Combines the 4 warps' states in the merge buffer and writes the CTA's partial.
+__device__ __forceinline__ void write_partial(const DecodeParams& p, const float* smem_f, int split, int hk, int b) {
+  const Dims& dm = p.dm;
+  const int ns = p.ns_q + p.ns_w;
+  const int d = threadIdx.x;  // MMA_THREADS == HD
+  for (int a = 0; a < dm.G; ++a) {
+    float M = -CUDART_INF_F;
+#pragma unroll
+    for (int w = 0; w < MMA_WARPS; ++w) M = fmaxf(M, smem_f[(w * 8 + a) * MS + HD]);
+    float Lsum = 0.f, A = 0.f;
+#pragma unroll
+    for (int w = 0; w < MMA_WARPS; ++w) {
+      const float* row = smem_f + (w * 8 + a) * MS;
+      float mw = row[HD];
+      float f = (mw == -CUDART_INF_F) ? 0.f : exp2f(mw - M);
+      Lsum += row[HD + 1] * f;
+      A += row[d] * f;
+    }
+    size_t hq = (size_t)b * dm.Hq + hk * dm.G + a;
+    p.part_acc[(hq * ns + split) * HD + d] = A;
+    if (d == 0) {
+      p.part_ml[(hq * ns + split) * 2 + 0] = M;
+      p.part_ml[(hq * ns + split) * 2 + 1] = Lsum;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// the kernel
+// ---------------------------------------------------------------------------
+template <int BK, int BV, int GS>
+__global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams p) {
+  using St = Stage<BK, BV, GS>;
+  constexpr int NG = St::NG;
+  extern __shared__ __align__(128) uint8_t smem[];
+  float* smem_f = reinterpret_cast<float*>(smem);
+
+  const Dims& dm = p.dm;
+  const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gid = lane >> 2, tig = lane & 3;
+
+  if (split < p.ns_w) {  // window splits come first so that they start early
+    window_split(p, split, hk, b, smem_f);
+    __syncthreads();
+    write_partial(p, smem_f, split, hk, b);
+    return;
+  }
+
+  const int sq = split - p.ns_w;
+  const int units = p.n_q / 32;
+  const int u0 = (int)(((long long)sq * units) / p.ns_q);
+  const int u1 = (int)(((long long)(sq + 1) * units) / p.ns_q);
+  const int n_my = (u1 - u0 - warp + MMA_WARPS - 1) / MMA_WARPS;  // units of this warp: u0 + warp + 4 j
+  const int bh = b * dm.Hkv + hk;
+  const int G = dm.G;
+
+  const uint8_t* kc_g = reinterpret_cast<const uint8_t*>(p.L.k_codes) + (size_t)bh * ((size_t)dm.nq_cap * HD * BK / 8);
+  const uint8_t* vc_g = reinterpret_cast<const uint8_t*>(p.L.v_codes) + (size_t)bh * ((size_t)dm.nq_cap * HD * BV / 8);
+  const uint8_t* km_g = reinterpret_cast<const uint8_t*>(p.L.k_meta) + (size_t)bh * (dm.nq_cap / GS) * 512;
+  const uint8_t* vm_g = reinterpret_cast<const uint8_t*>(p.L.v_meta) + (size_t)bh * (dm.nq_cap / 16) * (64 * NG);
+
+  uint8_t* my_stages = smem + (size_t)warp * NST * St::BYTES;
+  uint32_t* q_sm = reinterpret_cast<uint32_t*>(smem + MMA_WARPS * NST * St::BYTES);  // [lane][16] half2
+
+  auto issue = [&](int j) {  // stage unit j of this warp
+    if (j < n_my) {
+      const int u = u0 + warp + MMA_WARPS * j;
+      uint8_t* st = my_stages + (size_t)(j % NST) * St::BYTES;
+#pragma unroll
+      for (int c = 0; c < St::KC / 512; ++c) cp_async16(st + c * 512 + lane * 16, kc_g + (size_t)u * St::KC + c * 512 + lane * 16);
+      if (lane < 16) cp_async16(st + St::OFF_KS + lane * 16, km_g + (size_t)((u * 32) / GS) * 512 + lane * 16);
+#pragma unroll
+      for (int c = 0; c < St::VC / 512; ++c)
+        cp_async16(st + St::OFF_VC + c * 512 + lane * 16, vc_g + (size_t)u * St::VC + c * 512 + lane * 16);
+      if (lane * 16 < St::VM) cp_async16(st + St::OFF_VM + lane * 16, vm_g + (size_t)u * St::VM + lane * 16);
+    }
+    cp_async_commit();
+  };
+
+  // prologue: start the pipeline, then set up q while the copies fly
+#pragma unroll
+  for (int j = 0; j < NST - 1; ++j) issue(j);
+
+  // q of head gid in B-operand order: qraw[2s + j] = (q[16s + 2tig + 8j], q[16s + 2tig + 8j + 1]) as fp16
+  uint32_t qe[16];  // scaled by 2^-e(s), the weight the code's slot carries
+  {
+    const bool real = gid < G;
+    const uint16_t* qp = p.q + ((size_t)b * dm.Hq + hk * G + (real ? gid : 0)) * HD;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        uint32_t raw = *reinterpret_cast<const uint32_t*>(qp + 16 * s + 2 * tig + 8 * j);
+        float lo = real ? bf16_to_f(raw & 0xffff) : 0.f, hi = real ? bf16_to_f(raw >> 16) : 0.f;
+        uint32_t plain = pack_half2(lo, hi);
+        if (warp == 0) q_sm[lane * 16 + 2 * s + j] = plain;
+        const float sc = 1.0f / (float)(1 << Slots<BK>::e(s));
+        qe[2 * s + j] = pack_half2(lo * sc, hi * sc);
+      }
+    }
+  }
+  __syncthreads();
+
+  const float scale2 = p.scale * 1.4426950408889634f;
+  const float c1 = scale2 * 16777216.0f;  // undoes the 2^-24 of the subnormal code operand
+  float accO[8][4];                        // O^T: rows = channels 16 mt + gid (+8), cols = heads 2 tig (+1)
+  float accZ[4] = {0.f, 0.f, 0.f, 0.f};    // rows 0..NG-1: sum_t p_t z_tg ; row 8: sum_t p_t
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) accO[mt][i] = 0.f;
+  float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;  // running max (log2 units) of heads 2 tig, 2 tig + 1
+  float zb[4] = {0.f, 0.f, 0.f, 0.f};            // key zero-point bias of 16 units: rows = units
+
+  for (int j = 0; j < n_my; ++j) {
+    __syncwarp();  // everyone is done with the stage that is about to be refilled
+    issue(j + NST - 1);
+
+    if ((j & 15) == 0) {
+      // bias tile: zb[unit row][head] = sum_d q_d z_d for this warp's next 16 units (plain loads)
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      const int ja = j + gid, jb = j + gid + 8;
+      const uint8_t* za = km_g + (size_t)(((u0 + warp + MMA_WARPS * ja) * 32) / GS) * 512 + 256 + tig * 64;
+      const uint8_t* zbp = km_g + (size_t)(((u0 + warp + MMA_WARPS * jb) * 32) / GS) * 512 + 256 + tig * 64;
+      uint4 ra[4], rb[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        ra[i] = (ja < n_my) ? *reinterpret_cast<const uint4*>(za + i * 16) : make_uint4(0, 0, 0, 0);
+        rb[i] = (jb < n_my) ? *reinterpret_cast<const uint4*>(zbp + i * 16) : make_uint4(0, 0, 0, 0);
+      }
+      const uint4* qs = reinterpret_cast<const uint4*>(q_sm + lane * 16);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        uint4 qq = qs[i];  // k-steps 2i, 2i+1
+        mma16816(acc, ra[i].x, rb[i].x, ra[i].y, rb[i].y, qq.x, qq.y);
+        mma16816(acc, ra[i].z, rb[i].z, ra[i].w, rb[i].w, qq.z, qq.w);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) zb[i] = acc[i] * scale2;
+    }
+
+    cp_async_wait<NST - 1>();
+    __syncwarp();
+    const uint8_t* st = my_stages + (size_t)(j % NST) * St::BYTES;
+
+    // ---- S^T = Kc (q s)^T for the unit's 32 tokens ----
+    uint32_t bq[16];
+    {
+      const uint4* sp = reinterpret_cast<const uint4*>(st + St::OFF_KS + tig * 64);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        uint4 sv = sp[i];
+        bq[4 * i + 0] = hmul2_u(qe[4 * i + 0], sv.x);
+        bq[4 * i + 1] = hmul2_u(qe[4 * i + 1], sv.y);
+        bq[4 * i + 2] = hmul2_u(qe[4 * i + 2], sv.z);
+        bq[4 * i + 3] = hmul2_u(qe[4 * i + 3], sv.w);
+      }
+    }
+    float accS[2][4];
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) accS[mt][i] = 0.f;
+      uint4 w;
+      if (BK == 2) {
+        w = *reinterpret_cast<const uint4*>(st + mt * 512 + lane * 16);
+      } else {
+        w = *reinterpret_cast<const uint4*>(st + lane * 16);
+        if (mt == 1) { w.x >>= 8; w.y >>= 8; w.z >>= 8; w.w >>= 8; }
+      }
+      uint4 ws = make_uint4(w.x >> Slots<BK>::SHIFT, w.y >> Slots<BK>::SHIFT, w.z >> Slots<BK>::SHIFT,
+                            w.w >> Slots<BK>::SHIFT);
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        const uint32_t mk = Slots<BK>::mask(s);
+        const uint4& src = Slots<BK>::shifted(s) ? ws : w;
+        mma16816(accS[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, bq[2 * s], bq[2 * s + 1]);
+      }
+    }
+
+    // ---- online softmax (log2 domain); the unit's key bias is common to its 32 tokens ----
+    const int jr = j & 15;
+    float bz0 = __shfl_sync(0xffffffffu, jr < 8 ? zb[0] : zb[2], (jr & 7) * 4 + tig);
+    float bz1 = __shfl_sync(0xffffffffu, jr < 8 ? zb[1] : zb[3], (jr & 7) * 4 + tig);
+    float r0 = fmaxf(fmaxf(accS[0][0], accS[0][2]), fmaxf(accS[1][0], accS[1][2]));
+    float r1 = fmaxf(fmaxf(accS[0][1], accS[0][3]), fmaxf(accS[1][1], accS[1][3]));
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+      r0 = fmaxf(r0, __shfl_xor_sync(0xffffffffu, r0, o));
+      r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, o));
+    }
+    const float mn0 = fmaxf(m0, fmaf(r0, c1, bz0)), mn1 = fmaxf(m1, fmaf(r1, c1, bz1));
+    if (__any_sync(0xffffffffu, (mn0 > m0) | (mn1 > m1))) {
+      const float f0 = exp2f(m0 - mn0), f1 = exp2f(m1 - mn1);
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt) {
+        accO[mt][0] *= f0; accO[mt][1] *= f1; accO[mt][2] *= f0; accO[mt][3] *= f1;
+      }
+      accZ[0] *= f0; accZ[1] *= f1; accZ[2] *= f0; accZ[3] *= f1;
+      m0 = mn0; m1 = mn1;
+    }
+    const float t0 = bz0 - m0, t1 = bz1 - m1;
+    uint32_t pb[2][2];  // P as B operand: [16-token tile][b0, b1]
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      float p0 = exp2f(fmaf(accS[mt][0], c1, t0)), p1 = exp2f(fmaf(accS[mt][1], c1, t1));
+      float p2 = exp2f(fmaf(accS[mt][2], c1, t0)), p3 = exp2f(fmaf(accS[mt][3], c1, t1));
+      pb[mt][0] = movmatrix_trans(pack_half2(p0, p1));
+      pb[mt][1] = movmatrix_trans(pack_half2(p2, p3));
+    }
+
+    // ---- O^T += Vc^T (p s), zero-point and normaliser sums ----
+    uint4 wv;
+    if (BV == 1) wv = *reinterpret_cast<const uint4*>(st + St::OFF_VC + lane * 16);
+#pragma unroll
+    for (int tt = 0; tt < 2; ++tt) {
+      const uint8_t* vmeta = st + St::OFF_VM + tt * (64 * NG);
+      uint32_t sv[2 * NG];
+      if (NG == 4) {
+        uint4 x0 = *reinterpret_cast<const uint4*>(vmeta + tig * 32), x1 = *reinterpret_cast<const uint4*>(vmeta + tig * 32 + 16);
+        sv[0] = x0.x; sv[1] = x0.y; sv[2] = x0.z; sv[3] = x0.w;
+        sv[4 % (2 * NG)] = x1.x; sv[5 % (2 * NG)] = x1.y; sv[6 % (2 * NG)] = x1.z; sv[7 % (2 * NG)] = x1.w;
+      } else {
+        uint4 x0 = *reinterpret_cast<const uint4*>(vmeta + tig * 16);
+        sv[0] = x0.x; sv[1] = x0.y; sv[2] = x0.z; sv[3] = x0.w;
+      }
+      uint32_t za0 = 0, za2 = 0;
+      if (gid < NG) {
+        uint2 zz = *reinterpret_cast<const uint2*>(vmeta + 32 * NG + tig * (8 * NG) + gid * 8);
+        za0 = zz.x; za2 = zz.y;
+      }
+      const uint32_t ones = (gid == 0) ? 0x3C003C00u : 0u;
+      mma16816(accZ, za0, ones, za2, ones, pb[tt][0], pb[tt][1]);
+      uint32_t pg[NG][2];
+#pragma unroll
+      for (int gi = 0; gi < NG; ++gi) {
+        pg[gi][0] = hmul2_u(pb[tt][0], sv[2 * gi]);
+        pg[gi][1] = hmul2_u(pb[tt][1], sv[2 * gi + 1]);
+      }
+      uint4 w;
+      if (BV == 2) {
+        w = *reinterpret_cast<const uint4*>(st + St::OFF_VC + tt * 512 + lane * 16);
+      } else {
+        w = wv;
+        if (tt == 1) { w.x >>= 8; w.y >>= 8; w.z >>= 8; w.w >>= 8; }
+      }
+      uint4 ws = make_uint4(w.x >> Slots<BV>::SHIFT, w.y >> Slots<BV>::SHIFT, w.z >> Slots<BV>::SHIFT,
+                            w.w >> Slots<BV>::SHIFT);
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt) {
+        const uint32_t mk = Slots<BV>::mask(mt);
+        const uint4& src = Slots<BV>::shifted(mt) ? ws : w;
+        const int gi = (16 * mt) / GS;
+        mma16816(accO[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, pg[gi][0], pg[gi][1]);
+      }
+    }
+  }
+  cp_async_wait<0>();
+  __syncthreads();  // all warps are done with their stages: the memory becomes the merge buffer
+
+  // ---- epilogue: undo slot weights, add the zero-point sums, hand the state to the merge buffer ----
+  const float l0 = __shfl_sync(0xffffffffu, accZ[2], tig), l1 = __shfl_sync(0xffffffffu, accZ[3], tig);
+  float* mb = smem_f + (size_t)warp * 8 * MS;
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt) {
+    const int gi = (16 * mt) / GS;
+    const float z0 = __shfl_sync(0xffffffffu, accZ[0], 4 * gi + tig), z1 = __shfl_sync(0xffffffffu, accZ[1], 4 * gi + tig);
+    const float wgt = (float)(1u << (24 - Slots<BV>::e(mt)));
+    const int ch = 16 * mt + gid;
+    if (2 * tig < G) {
+      float* row = mb + (2 * tig) * MS;
+      row[ch] = fmaf(accO[mt][0], wgt, z0);
+      row[ch + 8] = fmaf(accO[mt][2], wgt, z0);
+    }
+    if (2 * tig + 1 < G) {
+      float* row = mb + (2 * tig + 1) * MS;
+      row[ch] = fmaf(accO[mt][1], wgt, z1);
+      row[ch + 8] = fmaf(accO[mt][3], wgt, z1);
+    }
+  }
+  if (gid == 0) {
+    if (2 * tig < G) {
+      mb[(2 * tig) * MS + HD] = m0;
+      mb[(2 * tig) * MS + HD + 1] = l0;
+    }
+    if (2 * tig + 1 < G) {
+      mb[(2 * tig + 1) * MS + HD] = m1;
+      mb[(2 * tig + 1) * MS + HD + 1] = l1;
+    }
+  }
+  __syncthreads();
+  write_partial(p, smem_f, split, hk, b);
+}
+
+template <int BK, int BV, int GS>
+cudaError_t launch_t(const DecodeParams& p, cudaStream_t st) {
+  constexpr int smem = smem_bytes<BK, BV, GS>();
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<BK, BV, GS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  dim3 grid(p.ns_q + p.ns_w, p.dm.Hkv, p.dm.B);
+  decode_mma_kernel<BK, BV, GS><<<grid, MMA_THREADS, smem, st>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool decode_mma_supported(const Dims& dm, int bk, int bv) {
+  (void)bk; (void)bv;
+  return dm.D == HD && dm.G <= 8 && (dm.g == 32 || dm.g == 64);
+}
+
+cudaError_t launch_decode_mma(const DecodeParams& p, cudaStream_t st) {
+  const int key = p.L.bk * 100 + p.L.bv * 10 + (p.dm.g == 64);
+  switch (key) {
+    case 220: return launch_t<2, 2, 32>(p, st);
+    case 221: return launch_t<2, 2, 64>(p, st);
+    case 210: return launch_t<2, 1, 32>(p, st);
+    case 211: return launch_t<2, 1, 64>(p, st);
+    case 120: return launch_t<1, 2, 32>(p, st);
+    case 121: return launch_t<1, 2, 64>(p, st);
+    case 110: return launch_t<1, 1, 32>(p, st);
+    case 111: return launch_t<1, 1, 64>(p, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
 }  // namespace xq
