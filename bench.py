@@ -175,10 +175,17 @@ def main():
     ap.add_argument("--splits", type=int, default=None)
     ap.add_argument("--layer-order", default="owners_first", choices=["owners_first", "ascending"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=None, help="fewer layers than the workload names (profiling captures only)")
+    ap.add_argument("--seq", type=int, default=None, help="another context length (profiling captures only)")
     args = ap.parse_args()
 
     from paper_2510_11236_b200 import workloads as W
     w = dict(W.CONFIGS[args.config])
+    if args.layers:
+        w["n_layers"] = args.layers
+        w["kq"], w["vq"] = min(w["kq"], args.layers), min(w["vq"], args.layers)
+    if args.seq:
+        w["seq"] = args.seq
     if args.impl == "reference":
         run_reference(args, w)
         return

@@ -17,12 +17,16 @@
 // Tokens are the M dimension of both products (S^T = Kc * Q'^T, O^T = Vc^T * P'),
 // so a GQA group of up to 8 query heads fills the N = 8 columns.
 //
-// Work split: grid (split, kv head, sequence).  The first ns_w splits take the
-// 16-bit window (scalar path, 16 tokens per tile); the remaining ns_q splits take
-// ranges of 32-token units of the packed region.  In a packed split the 4 warps
-// interleave units; each warp stages its own units in shared memory with
-// cp.async (NST stages ahead) and keeps a private online softmax; the warps'
-// states are merged at the end and the CTA writes one partial per query head.
+// Work split: grid (split, kv head, sequence), sized by the host to one wave of
+// long-lived CTAs.  Every split takes a range of 32-token units of the packed
+// region plus an equal share of the 16-bit window tokens (scalar fp32 path, done
+// first while the first packed stages are in flight).  The 4 warps interleave
+// units; each warp stages its own units in shared memory with cp.async (NST
+// stages ahead) and keeps a private online softmax; the warps' states are merged
+// at the end and the CTA writes one partial (m, l, acc[D]) per query head.  The
+// CTA that finishes last for a (sequence, kv head) -- found with an atomic ticket,
+// never by waiting -- merges the partials and writes the output.
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <math_constants.h>
 
@@ -45,15 +49,30 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// D = A * B (accumulator input zero)
+__device__ __forceinline__ void mma16816_z(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                           uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};\n"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+}
+
+// 2^x, approximate (relative error ~2^-22), flushes denormals; 2^-inf = 0
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
   uint32_t d;
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(d) : "r"(a));
   return d;
 }
 
-__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
-  uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem));
+__device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void* gmem) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_addr), "l"(gmem));
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
 template <int N>
@@ -104,28 +123,29 @@ struct Stage {
   static constexpr int BYTES = KC + KS + VC + VM;
 };
 
-constexpr int MS = HD + 4;  // merge-buffer row: acc[HD], m, l, padding (keeps rows 16-byte aligned)
+constexpr int MS = HD + 4;  // state row: acc[HD], m, l, padding (keeps rows 16-byte aligned)
 constexpr int MERGE_BYTES = MMA_WARPS * 8 * MS * 4;
 
+// dynamic shared memory: [stages of 4 warps | merge buffer (aliases the stages)] [q, B-operand order] [window states]
 template <int BK, int BV, int GS>
-constexpr int smem_bytes() {
-  int pipe = MMA_WARPS * NST * Stage<BK, BV, GS>::BYTES + 32 * 64;  // stages + q in B-operand layout
+constexpr int pipe_bytes() {
+  int pipe = MMA_WARPS * NST * Stage<BK, BV, GS>::BYTES;
   return pipe > MERGE_BYTES ? pipe : MERGE_BYTES;
 }
+constexpr int Q_BYTES = 32 * 64;
+__host__ __device__ inline int wstate_bytes(int G) { return MMA_WARPS * G * MS * 4; }
 
 // ---------------------------------------------------------------------------
-// window path: plain fp32 over 16-bit tokens, one token per warp iteration
+// window path: plain fp32 over 16-bit tokens [t0, t1), one token per warp
+// iteration; each warp leaves its state (acc, m, l per head) in `ws`.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ void window_split(const DecodeParams& p, int sw, int hk, int b, float* smem_f) {
+__device__ __forceinline__ void window_tokens(const DecodeParams& p, int t0, int t1, int hk, int b, float* ws) {
   const Dims& dm = p.dm;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int bh = b * dm.Hkv + hk;
   const int G = dm.G;
-  const int tiles = (p.r + 15) / 16;
-  const int t0 = (int)(((long long)sw * tiles) / p.ns_w) * 16;
-  const int t1 = min((int)(((long long)(sw + 1) * tiles) / p.ns_w) * 16, p.r);
-  const uint16_t* wk = p.L.win_k + (size_t)bh * dm.R * HD;
-  const uint16_t* wv = p.L.win_v + (size_t)bh * dm.R * HD;
+  const uint16_t* wk = p.L.win_k + (size_t)bh * dm.R * HD + lane * 4;
+  const uint16_t* wv = p.L.win_v + (size_t)bh * dm.R * HD + lane * 4;
   const float scale2 = p.scale * 1.4426950408889634f;
   float q[8][4], acc[8][4], m[8], l[8];
 #pragma unroll
@@ -134,29 +154,28 @@ __device__ __forceinline__ void window_split(const DecodeParams& p, int sw, int 
     l[a] = 0.f;
     const uint16_t* qp = p.q + ((size_t)b * dm.Hq + hk * G + (a < G ? a : 0)) * HD + lane * 4;
     uint2 raw = *reinterpret_cast<const uint2*>(qp);
-    q[a][0] = bf16_to_f(raw.x & 0xffff); q[a][1] = bf16_to_f(raw.x >> 16);
-    q[a][2] = bf16_to_f(raw.y & 0xffff); q[a][3] = bf16_to_f(raw.y >> 16);
+    q[a][0] = bf16_to_f(raw.x & 0xffff) * scale2; q[a][1] = bf16_to_f(raw.x >> 16) * scale2;
+    q[a][2] = bf16_to_f(raw.y & 0xffff) * scale2; q[a][3] = bf16_to_f(raw.y >> 16) * scale2;
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[a][j] = 0.f;
   }
   for (int t = t0 + warp; t < t1; t += MMA_WARPS) {
-    uint2 kr = *reinterpret_cast<const uint2*>(wk + (size_t)t * HD + lane * 4);
-    uint2 vr = *reinterpret_cast<const uint2*>(wv + (size_t)t * HD + lane * 4);
+    uint2 kr = *reinterpret_cast<const uint2*>(wk + (size_t)t * HD);
+    uint2 vr = *reinterpret_cast<const uint2*>(wv + (size_t)t * HD);
     float kx[4] = {bf16_to_f(kr.x & 0xffff), bf16_to_f(kr.x >> 16), bf16_to_f(kr.y & 0xffff), bf16_to_f(kr.y >> 16)};
     float vx[4] = {bf16_to_f(vr.x & 0xffff), bf16_to_f(vr.x >> 16), bf16_to_f(vr.y & 0xffff), bf16_to_f(vr.y >> 16)};
 #pragma unroll
     for (int a = 0; a < 8; ++a) {
       if (a < G) {
-        float dot = q[a][0] * kx[0];
-        dot = fmaf(q[a][1], kx[1], dot);
-        dot = fmaf(q[a][2], kx[2], dot);
-        dot = fmaf(q[a][3], kx[3], dot);
+        float x = q[a][0] * kx[0];
+        x = fmaf(q[a][1], kx[1], x);
+        x = fmaf(q[a][2], kx[2], x);
+        x = fmaf(q[a][3], kx[3], x);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        float x = dot * scale2;
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
         float mn = fmaxf(m[a], x);
-        float corr = exp2f(m[a] - mn);
-        float pe = exp2f(x - mn);
+        float corr = ex2(m[a] - mn);
+        float pe = ex2(x - mn);
         l[a] = l[a] * corr + pe;
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[a][j] = acc[a][j] * corr + pe * vx[j];
@@ -164,12 +183,11 @@ __device__ __forceinline__ void window_split(const DecodeParams& p, int sw, int 
       }
     }
   }
-  // merge buffer: [warp][head][MS]
-  float* mb = smem_f + (size_t)warp * 8 * MS;
+  float* mine = ws + (size_t)warp * G * MS;
 #pragma unroll
   for (int a = 0; a < 8; ++a) {
     if (a < G) {
-      float* row = mb + a * MS;
+      float* row = mine + a * MS;
       *reinterpret_cast<float4*>(row + lane * 4) = make_float4(acc[a][0], acc[a][1], acc[a][2], acc[a][3]);
       if (lane == 0) {
         row[HD] = m[a];
@@ -179,31 +197,99 @@ __device__ __forceinline__ void window_split(const DecodeParams& p, int sw, int 
   }
 }
 
-// Combines the 4 warps' states in the merge buffer and writes the CTA's partial.
-__device__ __forceinline__ void write_partial(const DecodeParams& p, const float* smem_f, int split, int hk, int b) {
+// Combines warp states (rows of MS floats: mb has 8 rows per warp, ws has G rows
+// per warp; either may be absent) and writes the CTA's partial for each head.
+__device__ __forceinline__ void write_partial(const DecodeParams& p, const float* mb, const float* ws, int split,
+                                              int ns, int hk, int b) {
   const Dims& dm = p.dm;
-  const int ns = p.ns_q + p.ns_w;
   const int d = threadIdx.x;  // MMA_THREADS == HD
-  for (int a = 0; a < dm.G; ++a) {
+  const int G = dm.G;
+  for (int a = 0; a < G; ++a) {
     float M = -CUDART_INF_F;
 #pragma unroll
-    for (int w = 0; w < MMA_WARPS; ++w) M = fmaxf(M, smem_f[(w * 8 + a) * MS + HD]);
+    for (int w = 0; w < MMA_WARPS; ++w) {
+      if (mb) M = fmaxf(M, mb[(w * 8 + a) * MS + HD]);
+      if (ws) M = fmaxf(M, ws[(w * G + a) * MS + HD]);
+    }
     float Lsum = 0.f, A = 0.f;
 #pragma unroll
     for (int w = 0; w < MMA_WARPS; ++w) {
-      const float* row = smem_f + (w * 8 + a) * MS;
-      float mw = row[HD];
-      float f = (mw == -CUDART_INF_F) ? 0.f : exp2f(mw - M);
-      Lsum += row[HD + 1] * f;
-      A += row[d] * f;
+      if (mb) {
+        const float* row = mb + (w * 8 + a) * MS;
+        float f = ex2(row[HD] - M);  // 2^-inf = 0 for an empty state; M is finite whenever any state is not empty
+        Lsum = fmaf(row[HD + 1], f, Lsum);
+        A = fmaf(row[d], f, A);
+      }
+      if (ws) {
+        const float* row = ws + (w * G + a) * MS;
+        float f = ex2(row[HD] - M);
+        Lsum = fmaf(row[HD + 1], f, Lsum);
+        A = fmaf(row[d], f, A);
+      }
     }
-    size_t hq = (size_t)b * dm.Hq + hk * dm.G + a;
+    size_t hq = (size_t)b * dm.Hq + hk * G + a;
     p.part_acc[(hq * ns + split) * HD + d] = A;
-    if (d == 0) {
-      p.part_ml[(hq * ns + split) * 2 + 0] = M;
-      p.part_ml[(hq * ns + split) * 2 + 1] = Lsum;
+    if (d == 0) *reinterpret_cast<float2*>(p.part_ml + (hq * ns + split) * 2) = make_float2(M, Lsum);
+  }
+}
+
+__device__ __forceinline__ float ld_cg(const float* p) {
+  float v;
+  asm volatile("ld.global.cg.f32 %0, [%1];\n" : "=f"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ float4 ld_cg4(const float* p) {
+  float4 v;
+  asm volatile("ld.global.cg.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
+}
+
+// Split-K merge by the last CTA of a (sequence, kv head): takes a ticket after
+// its partials are visible device-wide; the CTA that draws the last ticket reads
+// all partials from L2 and writes out = sum_s acc_s 2^(m_s-M) / sum_s l_s 2^(m_s-M).
+// No CTA ever waits for another.
+__device__ __forceinline__ void ticket_merge(const DecodeParams& p, int ns, int hk, int b, int* s_flag) {
+  const Dims& dm = p.dm;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = b * dm.Hkv + hk;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned t = atomicAdd(p.tickets + bh, 1u);
+    *s_flag = (t == (unsigned)(ns - 1));
+  }
+  __syncthreads();
+  if (!*s_flag) return;
+  __threadfence();
+  for (int a = warp; a < dm.G; a += MMA_WARPS) {
+    const size_t hq = (size_t)b * dm.Hq + hk * dm.G + a;
+    const float* ml = p.part_ml + hq * ns * 2;
+    const float* pa = p.part_acc + hq * ns * HD + lane * 4;
+    float M = -CUDART_INF_F;
+    for (int s = lane; s < ns; s += 32) M = fmaxf(M, ld_cg(ml + 2 * s));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float Ls = 0.f;
+#pragma unroll 4
+    for (int s = 0; s < ns; ++s) {
+      float f = ex2(ld_cg(ml + 2 * s) - M);
+      Ls = fmaf(ld_cg(ml + 2 * s + 1), f, Ls);
+      float4 v = ld_cg4(pa + (size_t)s * HD);
+      acc.x = fmaf(v.x, f, acc.x); acc.y = fmaf(v.y, f, acc.y);
+      acc.z = fmaf(v.z, f, acc.z); acc.w = fmaf(v.w, f, acc.w);
+    }
+    const float inv = 1.0f / Ls;
+    acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    if (p.out_f32) {
+      *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + hq * HD + lane * 4) = acc;
+    } else {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+      uint2 pk = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+      *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + hq * HD + lane * 4) = pk;
     }
   }
+  if (threadIdx.x == 0) p.tickets[bh] = 0u;  // ready for the next launch on this stream
 }
 
 // ---------------------------------------------------------------------------
@@ -213,69 +299,92 @@ template <int BK, int BV, int GS>
 __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams p) {
   using St = Stage<BK, BV, GS>;
   constexpr int NG = St::NG;
+  constexpr int PIPE = pipe_bytes<BK, BV, GS>();
   extern __shared__ __align__(128) uint8_t smem[];
-  float* smem_f = reinterpret_cast<float*>(smem);
+  __shared__ int s_flag;
+  float* mb = reinterpret_cast<float*>(smem);                           // merge buffer (after the loop)
+  uint32_t* q_sm = reinterpret_cast<uint32_t*>(smem + PIPE);             // [lane][16] half2
+  float* ws = reinterpret_cast<float*>(smem + PIPE + Q_BYTES);          // window states
 
   const Dims& dm = p.dm;
   const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gid = lane >> 2, tig = lane & 3;
+  const int G = dm.G;
 
-  if (split < p.ns_w) {  // window splits come first so that they start early
-    window_split(p, split, hk, b, smem_f);
+  if (p.ns_q == 0) {  // nothing is quantized yet: window-only splits
+    const int ns = p.ns_w;
+    const int tiles = (p.r + 15) / 16;
+    const int t0 = (int)(((long long)split * tiles) / ns) * 16;
+    const int t1 = min((int)(((long long)(split + 1) * tiles) / ns) * 16, p.r);
+    window_tokens(p, t0, t1, hk, b, ws);
     __syncthreads();
-    write_partial(p, smem_f, split, hk, b);
+    write_partial(p, nullptr, ws, split, ns, hk, b);
+    ticket_merge(p, ns, hk, b, &s_flag);
     return;
   }
 
-  const int sq = split - p.ns_w;
+  const int ns = p.ns_q;
   const int units = p.n_q / 32;
-  const int u0 = (int)(((long long)sq * units) / p.ns_q);
-  const int u1 = (int)(((long long)(sq + 1) * units) / p.ns_q);
+  const int u0 = (int)(((long long)split * units) / ns);
+  const int u1 = (int)(((long long)(split + 1) * units) / ns);
   const int n_my = (u1 - u0 - warp + MMA_WARPS - 1) / MMA_WARPS;  // units of this warp: u0 + warp + 4 j
   const int bh = b * dm.Hkv + hk;
-  const int G = dm.G;
 
-  const uint8_t* kc_g = reinterpret_cast<const uint8_t*>(p.L.k_codes) + (size_t)bh * ((size_t)dm.nq_cap * HD * BK / 8);
-  const uint8_t* vc_g = reinterpret_cast<const uint8_t*>(p.L.v_codes) + (size_t)bh * ((size_t)dm.nq_cap * HD * BV / 8);
+  // per-warp cursors into the four streams (this lane's 16-byte column)
+  const int uw = u0 + warp;
+  const uint8_t* gk = reinterpret_cast<const uint8_t*>(p.L.k_codes) + (size_t)bh * ((size_t)dm.nq_cap * (HD * BK / 8)) +
+                      (size_t)uw * St::KC + lane * 16;
+  const uint8_t* gv = reinterpret_cast<const uint8_t*>(p.L.v_codes) + (size_t)bh * ((size_t)dm.nq_cap * (HD * BV / 8)) +
+                      (size_t)uw * St::VC + lane * 16;
   const uint8_t* km_g = reinterpret_cast<const uint8_t*>(p.L.k_meta) + (size_t)bh * (dm.nq_cap / GS) * 512;
-  const uint8_t* vm_g = reinterpret_cast<const uint8_t*>(p.L.v_meta) + (size_t)bh * (dm.nq_cap / 16) * (64 * NG);
+  const uint8_t* gs = km_g + (size_t)((uw * 32) / GS) * 512 + lane * 16;
+  const uint8_t* gm = reinterpret_cast<const uint8_t*>(p.L.v_meta) + (size_t)bh * (dm.nq_cap / 16) * (64 * NG) +
+                      (size_t)uw * St::VM + lane * 16;
+  constexpr int GS_STEP = (MMA_WARPS * 32 / GS) * 512;  // key-scale bytes between a warp's consecutive units
 
-  uint8_t* my_stages = smem + (size_t)warp * NST * St::BYTES;
-  uint32_t* q_sm = reinterpret_cast<uint32_t*>(smem + MMA_WARPS * NST * St::BYTES);  // [lane][16] half2
-
-  auto issue = [&](int j) {  // stage unit j of this warp
-    if (j < n_my) {
-      const int u = u0 + warp + MMA_WARPS * j;
-      uint8_t* st = my_stages + (size_t)(j % NST) * St::BYTES;
-#pragma unroll
-      for (int c = 0; c < St::KC / 512; ++c) cp_async16(st + c * 512 + lane * 16, kc_g + (size_t)u * St::KC + c * 512 + lane * 16);
-      if (lane < 16) cp_async16(st + St::OFF_KS + lane * 16, km_g + (size_t)((u * 32) / GS) * 512 + lane * 16);
-#pragma unroll
-      for (int c = 0; c < St::VC / 512; ++c)
-        cp_async16(st + St::OFF_VC + c * 512 + lane * 16, vc_g + (size_t)u * St::VC + c * 512 + lane * 16);
-      if (lane * 16 < St::VM) cp_async16(st + St::OFF_VM + lane * 16, vm_g + (size_t)u * St::VM + lane * 16);
+  const uint32_t stage0 = (uint32_t)__cvta_generic_to_shared(smem) + warp * (NST * St::BYTES);
+  uint32_t st_issue = stage0;
+  int n_issued = 0;
+  auto issue = [&]() {  // stage this warp's next unit
+    if (n_issued < n_my) {
+      const uint32_t s = st_issue + lane * 16;
+      cp_async16(s, gk);
+      if (St::KC == 1024) cp_async16(s + 512, gk + 512);
+      if (lane < 16) cp_async16(s + St::OFF_KS, gs);
+      cp_async16(s + St::OFF_VC, gv);
+      if (St::VC == 1024) cp_async16(s + St::OFF_VC + 512, gv + 512);
+      if (lane * 16 < St::VM) cp_async16(s + St::OFF_VM, gm);
+      gk += MMA_WARPS * St::KC;
+      gv += MMA_WARPS * St::VC;
+      gm += MMA_WARPS * St::VM;
+      gs += GS_STEP;
     }
     cp_async_commit();
+    ++n_issued;
+    st_issue = (st_issue == stage0 + (NST - 1) * St::BYTES) ? stage0 : st_issue + St::BYTES;
   };
 
-  // prologue: start the pipeline, then set up q while the copies fly
+  // prologue: start the pipeline, then do this split's share of the window while the copies fly
 #pragma unroll
-  for (int j = 0; j < NST - 1; ++j) issue(j);
+  for (int j = 0; j < NST - 1; ++j) issue();
+  {
+    const int t0 = (int)(((long long)split * p.r) / ns), t1 = (int)(((long long)(split + 1) * p.r) / ns);
+    window_tokens(p, t0, t1, hk, b, ws);
+  }
 
-  // q of head gid in B-operand order: qraw[2s + j] = (q[16s + 2tig + 8j], q[16s + 2tig + 8j + 1]) as fp16
-  uint32_t qe[16];  // scaled by 2^-e(s), the weight the code's slot carries
+  // q of head gid in B-operand order: (q[16s + 2tig + 8j], q[16s + 2tig + 8j + 1]) as fp16, j = 0, 1
+  uint32_t qe[16];  // pre-scaled by 2^-e(s), the weight the code's slot carries
   {
     const bool real = gid < G;
-    const uint16_t* qp = p.q + ((size_t)b * dm.Hq + hk * G + (real ? gid : 0)) * HD;
+    const uint16_t* qp = p.q + ((size_t)b * dm.Hq + hk * G + (real ? gid : 0)) * HD + 2 * tig;
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
-        uint32_t raw = *reinterpret_cast<const uint32_t*>(qp + 16 * s + 2 * tig + 8 * j);
-        float lo = real ? bf16_to_f(raw & 0xffff) : 0.f, hi = real ? bf16_to_f(raw >> 16) : 0.f;
-        uint32_t plain = pack_half2(lo, hi);
-        if (warp == 0) q_sm[lane * 16 + 2 * s + j] = plain;
+        uint32_t raw = real ? *reinterpret_cast<const uint32_t*>(qp + 16 * s + 8 * j) : 0u;
+        float lo = bf16_to_f(raw & 0xffff), hi = bf16_to_f(raw >> 16);
+        if (warp == 0) q_sm[lane * 16 + 2 * s + j] = pack_half2(lo, hi);
         const float sc = 1.0f / (float)(1 << Slots<BK>::e(s));
         qe[2 * s + j] = pack_half2(lo * sc, hi * sc);
       }
@@ -293,24 +402,25 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     for (int i = 0; i < 4; ++i) accO[mt][i] = 0.f;
   float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;  // running max (log2 units) of heads 2 tig, 2 tig + 1
   float zb[4] = {0.f, 0.f, 0.f, 0.f};            // key zero-point bias of 16 units: rows = units
+  uint32_t st_read = stage0;
 
   for (int j = 0; j < n_my; ++j) {
     __syncwarp();  // everyone is done with the stage that is about to be refilled
-    issue(j + NST - 1);
+    issue();
 
     if ((j & 15) == 0) {
-      // bias tile: zb[unit row][head] = sum_d q_d z_d for this warp's next 16 units (plain loads)
-      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      // bias tile: zb[unit row][head] = scale * sum_d q_d z_d for this warp's next 16 units (plain loads)
       const int ja = j + gid, jb = j + gid + 8;
-      const uint8_t* za = km_g + (size_t)(((u0 + warp + MMA_WARPS * ja) * 32) / GS) * 512 + 256 + tig * 64;
-      const uint8_t* zbp = km_g + (size_t)(((u0 + warp + MMA_WARPS * jb) * 32) / GS) * 512 + 256 + tig * 64;
+      const uint8_t* za = km_g + (size_t)(((uw + MMA_WARPS * ja) * 32) / GS) * 512 + 256 + tig * 64;
+      const uint8_t* zc = km_g + (size_t)(((uw + MMA_WARPS * jb) * 32) / GS) * 512 + 256 + tig * 64;
       uint4 ra[4], rb[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         ra[i] = (ja < n_my) ? *reinterpret_cast<const uint4*>(za + i * 16) : make_uint4(0, 0, 0, 0);
-        rb[i] = (jb < n_my) ? *reinterpret_cast<const uint4*>(zbp + i * 16) : make_uint4(0, 0, 0, 0);
+        rb[i] = (jb < n_my) ? *reinterpret_cast<const uint4*>(zc + i * 16) : make_uint4(0, 0, 0, 0);
       }
       const uint4* qs = reinterpret_cast<const uint4*>(q_sm + lane * 16);
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         uint4 qq = qs[i];  // k-steps 2i, 2i+1
@@ -323,47 +433,56 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
 
     cp_async_wait<NST - 1>();
     __syncwarp();
-    const uint8_t* st = my_stages + (size_t)(j % NST) * St::BYTES;
+    const uint32_t st = st_read;
+    st_read = (st_read == stage0 + (NST - 1) * St::BYTES) ? stage0 : st_read + St::BYTES;
+    auto lds128 = [](uint32_t a) {
+      uint4 v;
+      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+      return v;
+    };
+    auto lds64 = [](uint32_t a) {
+      uint2 v;
+      asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "r"(a));
+      return v;
+    };
 
     // ---- S^T = Kc (q s)^T for the unit's 32 tokens ----
     uint32_t bq[16];
-    {
-      const uint4* sp = reinterpret_cast<const uint4*>(st + St::OFF_KS + tig * 64);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        uint4 sv = sp[i];
-        bq[4 * i + 0] = hmul2_u(qe[4 * i + 0], sv.x);
-        bq[4 * i + 1] = hmul2_u(qe[4 * i + 1], sv.y);
-        bq[4 * i + 2] = hmul2_u(qe[4 * i + 2], sv.z);
-        bq[4 * i + 3] = hmul2_u(qe[4 * i + 3], sv.w);
-      }
+    for (int i = 0; i < 4; ++i) {
+      uint4 sv = lds128(st + St::OFF_KS + tig * 64 + i * 16);
+      bq[4 * i + 0] = hmul2_u(qe[4 * i + 0], sv.x);
+      bq[4 * i + 1] = hmul2_u(qe[4 * i + 1], sv.y);
+      bq[4 * i + 2] = hmul2_u(qe[4 * i + 2], sv.z);
+      bq[4 * i + 3] = hmul2_u(qe[4 * i + 3], sv.w);
     }
     float accS[2][4];
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) accS[mt][i] = 0.f;
       uint4 w;
       if (BK == 2) {
-        w = *reinterpret_cast<const uint4*>(st + mt * 512 + lane * 16);
+        w = lds128(st + mt * 512 + lane * 16);
       } else {
-        w = *reinterpret_cast<const uint4*>(st + lane * 16);
+        w = lds128(st + lane * 16);
         if (mt == 1) { w.x >>= 8; w.y >>= 8; w.z >>= 8; w.w >>= 8; }
       }
-      uint4 ws = make_uint4(w.x >> Slots<BK>::SHIFT, w.y >> Slots<BK>::SHIFT, w.z >> Slots<BK>::SHIFT,
-                            w.w >> Slots<BK>::SHIFT);
+      uint4 wsft = make_uint4(w.x >> Slots<BK>::SHIFT, w.y >> Slots<BK>::SHIFT, w.z >> Slots<BK>::SHIFT,
+                              w.w >> Slots<BK>::SHIFT);
 #pragma unroll
       for (int s = 0; s < 8; ++s) {
         const uint32_t mk = Slots<BK>::mask(s);
-        const uint4& src = Slots<BK>::shifted(s) ? ws : w;
-        mma16816(accS[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, bq[2 * s], bq[2 * s + 1]);
+        const uint4& src = Slots<BK>::shifted(s) ? wsft : w;
+        if (s == 0)
+          mma16816_z(accS[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, bq[0], bq[1]);
+        else
+          mma16816(accS[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, bq[2 * s], bq[2 * s + 1]);
       }
     }
 
     // ---- online softmax (log2 domain); the unit's key bias is common to its 32 tokens ----
     const int jr = j & 15;
-    float bz0 = __shfl_sync(0xffffffffu, jr < 8 ? zb[0] : zb[2], (jr & 7) * 4 + tig);
-    float bz1 = __shfl_sync(0xffffffffu, jr < 8 ? zb[1] : zb[3], (jr & 7) * 4 + tig);
+    const float bz0 = __shfl_sync(0xffffffffu, jr < 8 ? zb[0] : zb[2], (jr & 7) * 4 + tig);
+    const float bz1 = __shfl_sync(0xffffffffu, jr < 8 ? zb[1] : zb[3], (jr & 7) * 4 + tig);
     float r0 = fmaxf(fmaxf(accS[0][0], accS[0][2]), fmaxf(accS[1][0], accS[1][2]));
     float r1 = fmaxf(fmaxf(accS[0][1], accS[0][3]), fmaxf(accS[1][1], accS[1][3]));
 #pragma unroll
@@ -373,7 +492,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     }
     const float mn0 = fmaxf(m0, fmaf(r0, c1, bz0)), mn1 = fmaxf(m1, fmaf(r1, c1, bz1));
     if (__any_sync(0xffffffffu, (mn0 > m0) | (mn1 > m1))) {
-      const float f0 = exp2f(m0 - mn0), f1 = exp2f(m1 - mn1);
+      const float f0 = ex2(m0 - mn0), f1 = ex2(m1 - mn1);
 #pragma unroll
       for (int mt = 0; mt < 8; ++mt) {
         accO[mt][0] *= f0; accO[mt][1] *= f1; accO[mt][2] *= f0; accO[mt][3] *= f1;
@@ -385,30 +504,30 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     uint32_t pb[2][2];  // P as B operand: [16-token tile][b0, b1]
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
-      float p0 = exp2f(fmaf(accS[mt][0], c1, t0)), p1 = exp2f(fmaf(accS[mt][1], c1, t1));
-      float p2 = exp2f(fmaf(accS[mt][2], c1, t0)), p3 = exp2f(fmaf(accS[mt][3], c1, t1));
+      float p0 = ex2(fmaf(accS[mt][0], c1, t0)), p1 = ex2(fmaf(accS[mt][1], c1, t1));
+      float p2 = ex2(fmaf(accS[mt][2], c1, t0)), p3 = ex2(fmaf(accS[mt][3], c1, t1));
       pb[mt][0] = movmatrix_trans(pack_half2(p0, p1));
       pb[mt][1] = movmatrix_trans(pack_half2(p2, p3));
     }
 
     // ---- O^T += Vc^T (p s), zero-point and normaliser sums ----
-    uint4 wv;
-    if (BV == 1) wv = *reinterpret_cast<const uint4*>(st + St::OFF_VC + lane * 16);
+    uint4 wv1 = make_uint4(0, 0, 0, 0);
+    if (BV == 1) wv1 = lds128(st + St::OFF_VC + lane * 16);
 #pragma unroll
     for (int tt = 0; tt < 2; ++tt) {
-      const uint8_t* vmeta = st + St::OFF_VM + tt * (64 * NG);
+      const uint32_t vmeta = st + St::OFF_VM + tt * (64 * NG);
       uint32_t sv[2 * NG];
       if (NG == 4) {
-        uint4 x0 = *reinterpret_cast<const uint4*>(vmeta + tig * 32), x1 = *reinterpret_cast<const uint4*>(vmeta + tig * 32 + 16);
+        uint4 x0 = lds128(vmeta + tig * 32), x1 = lds128(vmeta + tig * 32 + 16);
         sv[0] = x0.x; sv[1] = x0.y; sv[2] = x0.z; sv[3] = x0.w;
         sv[4 % (2 * NG)] = x1.x; sv[5 % (2 * NG)] = x1.y; sv[6 % (2 * NG)] = x1.z; sv[7 % (2 * NG)] = x1.w;
       } else {
-        uint4 x0 = *reinterpret_cast<const uint4*>(vmeta + tig * 16);
+        uint4 x0 = lds128(vmeta + tig * 16);
         sv[0] = x0.x; sv[1] = x0.y; sv[2] = x0.z; sv[3] = x0.w;
       }
       uint32_t za0 = 0, za2 = 0;
       if (gid < NG) {
-        uint2 zz = *reinterpret_cast<const uint2*>(vmeta + 32 * NG + tig * (8 * NG) + gid * 8);
+        uint2 zz = lds64(vmeta + 32 * NG + tig * (8 * NG) + gid * 8);
         za0 = zz.x; za2 = zz.y;
       }
       const uint32_t ones = (gid == 0) ? 0x3C003C00u : 0u;
@@ -421,17 +540,17 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
       }
       uint4 w;
       if (BV == 2) {
-        w = *reinterpret_cast<const uint4*>(st + St::OFF_VC + tt * 512 + lane * 16);
+        w = lds128(st + St::OFF_VC + tt * 512 + lane * 16);
       } else {
-        w = wv;
+        w = wv1;
         if (tt == 1) { w.x >>= 8; w.y >>= 8; w.z >>= 8; w.w >>= 8; }
       }
-      uint4 ws = make_uint4(w.x >> Slots<BV>::SHIFT, w.y >> Slots<BV>::SHIFT, w.z >> Slots<BV>::SHIFT,
-                            w.w >> Slots<BV>::SHIFT);
+      uint4 wsft = make_uint4(w.x >> Slots<BV>::SHIFT, w.y >> Slots<BV>::SHIFT, w.z >> Slots<BV>::SHIFT,
+                              w.w >> Slots<BV>::SHIFT);
 #pragma unroll
       for (int mt = 0; mt < 8; ++mt) {
         const uint32_t mk = Slots<BV>::mask(mt);
-        const uint4& src = Slots<BV>::shifted(mt) ? ws : w;
+        const uint4& src = Slots<BV>::shifted(mt) ? wsft : w;
         const int gi = (16 * mt) / GS;
         mma16816(accO[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, pg[gi][0], pg[gi][1]);
       }
@@ -442,7 +561,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
 
   // ---- epilogue: undo slot weights, add the zero-point sums, hand the state to the merge buffer ----
   const float l0 = __shfl_sync(0xffffffffu, accZ[2], tig), l1 = __shfl_sync(0xffffffffu, accZ[3], tig);
-  float* mb = smem_f + (size_t)warp * 8 * MS;
+  float* mine = mb + (size_t)warp * 8 * MS;
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
     const int gi = (16 * mt) / GS;
@@ -450,40 +569,42 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     const float wgt = (float)(1u << (24 - Slots<BV>::e(mt)));
     const int ch = 16 * mt + gid;
     if (2 * tig < G) {
-      float* row = mb + (2 * tig) * MS;
+      float* row = mine + (2 * tig) * MS;
       row[ch] = fmaf(accO[mt][0], wgt, z0);
       row[ch + 8] = fmaf(accO[mt][2], wgt, z0);
     }
     if (2 * tig + 1 < G) {
-      float* row = mb + (2 * tig + 1) * MS;
+      float* row = mine + (2 * tig + 1) * MS;
       row[ch] = fmaf(accO[mt][1], wgt, z1);
       row[ch + 8] = fmaf(accO[mt][3], wgt, z1);
     }
   }
   if (gid == 0) {
     if (2 * tig < G) {
-      mb[(2 * tig) * MS + HD] = m0;
-      mb[(2 * tig) * MS + HD + 1] = l0;
+      mine[(2 * tig) * MS + HD] = m0;
+      mine[(2 * tig) * MS + HD + 1] = l0;
     }
     if (2 * tig + 1 < G) {
-      mb[(2 * tig + 1) * MS + HD] = m1;
-      mb[(2 * tig + 1) * MS + HD + 1] = l1;
+      mine[(2 * tig + 1) * MS + HD] = m1;
+      mine[(2 * tig + 1) * MS + HD + 1] = l1;
     }
   }
   __syncthreads();
-  write_partial(p, smem_f, split, hk, b);
+  write_partial(p, mb, ws, split, ns, hk, b);
+  ticket_merge(p, ns, hk, b, &s_flag);
 }
 
 template <int BK, int BV, int GS>
 cudaError_t launch_t(const DecodeParams& p, cudaStream_t st) {
-  constexpr int smem = smem_bytes<BK, BV, GS>();
-  static bool configured = false;
-  if (!configured) {
+  const int smem = pipe_bytes<BK, BV, GS>() + Q_BYTES + wstate_bytes(p.dm.G);
+  static int configured = 0;
+  if (configured < smem) {
     cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<BK, BV, GS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured = smem;
   }
-  dim3 grid(p.ns_q + p.ns_w, p.dm.Hkv, p.dm.B);
+  const int ns = p.ns_q > 0 ? p.ns_q : p.ns_w;
+  dim3 grid(ns, p.dm.Hkv, p.dm.B);
   decode_mma_kernel<BK, BV, GS><<<grid, MMA_THREADS, smem, st>>>(p);
   return cudaGetLastError();
 }
@@ -494,6 +615,8 @@ bool decode_mma_supported(const Dims& dm, int bk, int bv) {
   (void)bk; (void)bv;
   return dm.D == HD && dm.G <= 8 && (dm.g == 32 || dm.g == 64);
 }
+
+int decode_mma_ctas_per_sm() { return 3; }
 
 cudaError_t launch_decode_mma(const DecodeParams& p, cudaStream_t st) {
   const int key = p.L.bk * 100 + p.L.bv * 10 + (p.dm.g == 64);

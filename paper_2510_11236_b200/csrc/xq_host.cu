@@ -28,7 +28,7 @@ struct LayerRegions {
 struct Plan {
   Dims dm;
   std::vector<LayerRegions> layers;
-  size_t part_acc, part_ml, staging, total;
+  size_t part_acc, part_ml, tickets, staging, total;
   size_t staging_kv_bytes, staging_q_bytes;
 };
 
@@ -85,6 +85,7 @@ void make_plan(const xq_config* c, Plan& pl) {
   }
   pl.part_acc = take((size_t)dm.B * dm.Hq * XQ_MAX_SPLITS * dm.D * 4);
   pl.part_ml = take((size_t)dm.B * dm.Hq * XQ_MAX_SPLITS * 2 * 4);
+  pl.tickets = take(BH * 4);
   pl.staging_kv_bytes = (size_t)c->n_layers * BH * dm.D * 2;
   pl.staging_q_bytes = (size_t)c->n_layers * dm.B * dm.Hq * dm.D * 2;
   pl.staging = take(2 * align_up(pl.staging_kv_bytes, 256) + 2 * align_up(pl.staging_q_bytes, 256));
@@ -107,6 +108,7 @@ struct xq_cache {
   int last_cuda;
   float scale;
   int sm_count;
+  bool tickets_clean;  // the ticket counters have been zeroed on a stream
   // timing
   bool timing;
   std::vector<EventPair> pool;
@@ -139,11 +141,48 @@ void token_bytes(const xq_cache* c, int l, double& q_bytes, double& w_bytes) {
   w_bytes = 4.0 * dm.D;
 }
 
+bool layer_uses_mma(const xq_cache* c, int l) {
+  if (c->cfg.kernel == XQ_KERNEL_GENERIC) return false;
+  return decode_mma_supported(c->plan.dm, layer_bits(l, c->cfg.kq), layer_bits(l, c->cfg.vq));
+}
+
+// Splits per (sequence, kv head) stream.  Tensor-core kernel: every split takes
+// packed units and a share of the window (ns_w = 0 unless nothing is packed yet),
+// sized towards whole waves of resident CTAs.  Generic kernel: separate splits for
+// the packed region and for the window, in proportion to their bytes.
 void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w) {
   const Dims& dm = c->plan.dm;
   int S = c->seq[l];
   int r = residual_count(S, dm.R), nq = S - r;
   int units = nq / 32, tiles = (r + 15) / 16;
+  const int streams = dm.B * dm.Hkv;
+  if (layer_uses_mma(c, l)) {
+    if (units == 0) {
+      ns_q = 0;
+      ns_w = c->cfg.n_splits > 0 ? c->cfg.n_splits : 4;
+      if (ns_w > tiles) ns_w = tiles;
+      if (ns_w < 1) ns_w = 1;
+      return;
+    }
+    ns_w = 0;
+    if (c->cfg.n_splits > 0) {
+      ns_q = c->cfg.n_splits < units ? c->cfg.n_splits : units;
+      return;
+    }
+    const double slots = (double)c->sm_count * decode_mma_ctas_per_sm();
+    int best = 1;
+    double best_score = -1.0;
+    for (int ns = 1; ns <= 64 && ns <= units; ++ns) {
+      double ctas = (double)ns * streams;
+      double waves = ceil(ctas / slots);
+      double fill = ctas / (waves * slots);
+      double upc = (double)units / ns;          // units per CTA
+      double score = fill * upc / (upc + 12.0);  // ~12 units' worth of fixed cost per CTA
+      if (score > best_score) { best_score = score; best = ns; }
+    }
+    ns_q = best;
+    return;
+  }
   double qb, wb;
   token_bytes(c, l, qb, wb);
   double bytes_q = qb * nq, bytes_w = wb * r;
@@ -151,9 +190,7 @@ void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w) {
   if (c->cfg.n_splits > 0) {
     total = c->cfg.n_splits;
   } else {
-    // aim for ~48 KB of cache per CTA, then round the grid to whole waves of 2 CTAs per SM
     double per_stream = bytes_q + bytes_w;
-    int streams = dm.B * dm.Hkv;
     int want = (int)ceil(per_stream / 49152.0);
     if (want < 1) want = 1;
     long long ctas = (long long)want * streams;
@@ -171,11 +208,6 @@ void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w) {
     ns_q = 0;
     ns_w = total < tiles ? total : tiles;
     if (ns_w < 1) ns_w = 1;
-    return;
-  }
-  if (tiles == 0) {  // not reachable with S > 0, kept for safety
-    ns_w = 0;
-    ns_q = total < units ? total : units;
     return;
   }
   int w = (int)floor(total * bytes_w / (bytes_q + bytes_w) + 0.5);
@@ -227,12 +259,29 @@ int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, c
   p.scale = c->scale;
   p.part_acc = (float*)(c->ws + c->plan.part_acc);
   p.part_ml = (float*)(c->ws + c->plan.part_ml);
-  bool use_mma = c->cfg.kernel != XQ_KERNEL_GENERIC && decode_mma_supported(dm, p.L.bk, p.L.bv);
+  bool use_mma = layer_uses_mma(c, layer);
   if (c->cfg.kernel == XQ_KERNEL_MMA && !use_mma) return XQ_ERR_CONFIG;
+  p.out = out;
+  p.out_f32 = out_f32;
+  p.tickets = (unsigned int*)(c->ws + c->plan.tickets);
   cudaError_t e;
+  if (use_mma) {
+    if (!c->tickets_clean) {
+      e = cudaMemsetAsync(p.tickets, 0, (size_t)dm.B * dm.Hkv * 4, st);
+      if (e != cudaSuccess) return fail_cuda(c, e);
+      c->tickets_clean = true;
+    }
+    {
+      Timer t(c, st, 0);
+      e = launch_decode_mma(p, st);  // merges the partials itself
+    }
+    c->launches++;
+    if (e != cudaSuccess) { c->tickets_clean = false; return fail_cuda(c, e); }
+    return XQ_OK;
+  }
   {
     Timer t(c, st, 0);
-    e = use_mma ? launch_decode_mma(p, st) : launch_decode_generic(p, st);
+    e = launch_decode_generic(p, st);
   }
   c->launches++;
   if (e != cudaSuccess) return fail_cuda(c, e);
@@ -283,6 +332,7 @@ int xq_create(const xq_config* cfg, void* dev_workspace, size_t bytes, xq_cache*
   c->timing = false;
   c->used = 0;
   c->sm_count = 148;
+  c->tickets_clean = false;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) == cudaSuccess &&
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)

@@ -57,6 +57,10 @@ struct DecodeParams {
   float scale;
   float* part_acc;    // [B,Hq,ns,D]
   float* part_ml;     // [B,Hq,ns,2]  (running max in log2 units, sum)
+  // used by kernels that merge the partials themselves (last CTA of a stream):
+  void* out;              // [B,Hq,D] bf16 or f32
+  int out_f32;
+  unsigned int* tickets;  // [B*Hkv], zero between launches
 };
 
 struct MergeParams {
@@ -73,6 +77,7 @@ cudaError_t launch_window_append(const WindowParams& p, cudaStream_t st);
 cudaError_t launch_decode_generic(const DecodeParams& p, cudaStream_t st);
 cudaError_t launch_decode_mma(const DecodeParams& p, cudaStream_t st);
 bool decode_mma_supported(const Dims& dm, int bk, int bv);
+int decode_mma_ctas_per_sm();
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t st);
 
 }  // namespace xq
