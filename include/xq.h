@@ -130,6 +130,33 @@ int xq_decode_attention(xq_cache* c, int layer, const void* q, void* out, void* 
  * head_dim] (the accumulator before the final rounding to bfloat16). */
 int xq_decode_attention_f32(xq_cache* c, int layer, const void* q, float* out, void* stream);
 
+/* xq_decode_attention for callers that cannot provide scratch memory of their
+ * own.  (The paper has no counterpart: this is a deployment variant, not part of
+ * the method.)  Some hosts hand every byte of device memory to their own pools at
+ * start-up and forbid cudaMalloc afterwards -- an inference server that runs this
+ * library as a plug-in, a real-time loop that must not enter the allocator, a
+ * process whose memory budget was fixed before this library was loaded.  Such a
+ * caller still passes q and out (device, [batch, n_q_heads, head_dim] bfloat16,
+ * 16-byte aligned) but the split-K partials and merge tickets, which
+ * xq_decode_attention keeps in the caller's workspace, live here in a
+ * XQ_STATIC_SCRATCH_BYTES array that is part of the library image: every GPU
+ * that loads the library holds that much device memory until the process exits.
+ * The call allocates and frees nothing, on the host side of CUDA or through any
+ * library.  Result: identical to xq_decode_attention.
+ * Limits: the partials of the call (batch * n_q_heads * splits * (head_dim + 2)
+ * floats, plus one ticket per (sequence, kv head)) must fit the array, else
+ * XQ_ERR_CAPACITY and nothing is launched; a smaller n_splits in xq_config
+ * shrinks them.  The array is shared by every handle and every call on a device
+ * and keeps the previous call's contents; the call clears the part that must
+ * start at zero (the tickets) on `stream` before its kernel.  Two such calls
+ * whose kernels may overlap on the GPU (different streams without an ordering
+ * between them) race on the array: keep them on one stream or order them.
+ * The first call on each device looks up the array's device address (a short
+ * synchronous CUDA runtime query, no allocation); make that first call outside
+ * any stream capture.  Other errors as xq_decode_attention. */
+#define XQ_STATIC_SCRATCH_BYTES (8u << 20)
+int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out, void* stream);
+
 /* One decode step of a whole model: for each layer, append one token and run
  * decode attention.  K_new, V_new: [n_layers, batch, n_kv_heads, 1, head_dim];
  * q, out: [n_layers, batch, n_q_heads, head_dim]; bfloat16; slice l belongs to

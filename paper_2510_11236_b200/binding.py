@@ -19,6 +19,7 @@ XQ_BF16 = 0
 XQ_KERNEL_AUTO, XQ_KERNEL_GENERIC, XQ_KERNEL_MMA = 0, 1, 2
 XQ_MEM_DEVICE, XQ_MEM_HOST = 0, 1
 XQ_MAX_SPLITS = 256
+XQ_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class xq_config(ctypes.Structure):
@@ -45,6 +46,8 @@ _SIGNATURES = {
                                            ctypes.c_void_p]),
     "xq_decode_attention_f32": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
                                                ctypes.c_void_p]),
+    "xq_decode_attention_static": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                                  ctypes.c_void_p]),
     "xq_decode_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                       ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.c_int,
                                       ctypes.c_void_p]),
@@ -134,6 +137,10 @@ def xq_decode_attention(handle, layer: int, q, out, stream: int = 0) -> int:
 
 def xq_decode_attention_f32(handle, layer: int, q, out, stream: int = 0) -> int:
     return lib().xq_decode_attention_f32(handle, layer, _ptr(q), _ptr(out), stream)
+
+
+def xq_decode_attention_static(handle, layer: int, q, out, stream: int = 0) -> int:
+    return lib().xq_decode_attention_static(handle, layer, _ptr(q), _ptr(out), stream)
 
 
 def xq_decode_step(handle, K_new, V_new, q, out, layer_order=None, mem: int = XQ_MEM_DEVICE, stream: int = 0) -> int:

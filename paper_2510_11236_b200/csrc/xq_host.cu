@@ -5,6 +5,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -96,6 +97,38 @@ constexpr int N_KINDS = 4;
 constexpr int TIMING_POOL = 1 << 15;
 
 struct EventPair { cudaEvent_t a, b; int kind; };
+
+}  // namespace
+
+// Scratch of xq_decode_attention_static: part of the library image, one copy per
+// GPU that loads it.  In host code this name is only a handle for the runtime's
+// symbol table, never a device address: kernels get the address that
+// cudaGetSymbolAddress returns for the current device.
+static __device__ __align__(256) unsigned char g_static_scratch[XQ_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int STATIC_MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+uint8_t* g_static_address[STATIC_MAX_DEVICES] = {};
+
+// Device address of g_static_scratch on the current device; looked up once per device.
+cudaError_t static_scratch_address(uint8_t** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= STATIC_MAX_DEVICES) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_address[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    if (!p || ((uintptr_t)p & 255)) return cudaErrorInvalidSymbol;
+    g_static_address[dev] = (uint8_t*)p;
+  }
+  *out = g_static_address[dev];
+  return cudaSuccess;
+}
 
 }  // namespace
 
@@ -412,6 +445,77 @@ int xq_decode_attention(xq_cache* c, int layer, const void* q, void* out, void* 
 
 int xq_decode_attention_f32(xq_cache* c, int layer, const void* q, float* out, void* stream) {
   return decode_impl(c, layer, q, out, 1, (cudaStream_t)stream);
+}
+
+int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out, void* stream) {
+  if (!c || !q || !out) return XQ_ERR_ARG;
+  if (layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
+  if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return XQ_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const Dims& dm = c->plan.dm;
+  const int S = c->seq[layer];
+  if (S < 1) return XQ_ERR_ARG;
+  const int r = residual_count(S, dm.R), nq = S - r;
+  if (!owns_codes(layer, c->cfg.km) || !owns_codes(layer, c->cfg.vm)) {
+    const int So = c->seq[layer - 1];
+    if (So - residual_count(So, dm.R) < nq) return XQ_ERR_ORDER;
+  }
+  const bool use_mma = layer_uses_mma(c, layer);
+  if (c->cfg.kernel == XQ_KERNEL_MMA && !use_mma) return XQ_ERR_CONFIG;
+  DecodeParams p;
+  p.dm = dm;
+  p.L = layer_ptrs(c, layer);
+  p.q = (const uint16_t*)q;
+  p.n_q = nq;
+  p.r = r;
+  plan_splits(c, layer, p.ns_q, p.ns_w);
+  p.scale = c->scale;
+  p.out = out;
+  p.out_f32 = 0;
+  // carve the static array: [partial accumulators | partial (max, sum) | tickets]
+  const size_t ns = (size_t)p.ns_q + (size_t)p.ns_w;
+  const size_t acc_bytes = align_up((size_t)dm.B * dm.Hq * ns * dm.D * 4, 256);
+  const size_t ml_bytes = align_up((size_t)dm.B * dm.Hq * ns * 2 * 4, 256);
+  const size_t ticket_bytes = (size_t)dm.B * dm.Hkv * 4;
+  if (acc_bytes + ml_bytes + ticket_bytes > (size_t)XQ_STATIC_SCRATCH_BYTES) return XQ_ERR_CAPACITY;
+  uint8_t* base = nullptr;
+  cudaError_t e = static_scratch_address(&base);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  p.part_acc = (float*)base;
+  p.part_ml = (float*)(base + acc_bytes);
+  p.tickets = (unsigned int*)(base + acc_bytes + ml_bytes);
+  if (use_mma) {
+    // the array keeps whatever the previous call (of any handle) left: tickets must start at zero
+    e = cudaMemsetAsync(p.tickets, 0, ticket_bytes, st);
+    if (e != cudaSuccess) return fail_cuda(c, e);
+    {
+      Timer t(c, st, 0);
+      e = launch_decode_mma(p, st);
+    }
+    c->launches++;
+    if (e != cudaSuccess) return fail_cuda(c, e);
+    return XQ_OK;
+  }
+  {
+    Timer t(c, st, 0);
+    e = launch_decode_generic(p, st);
+  }
+  c->launches++;
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  MergeParams m;
+  m.dm = dm;
+  m.ns = (int)ns;
+  m.part_acc = p.part_acc;
+  m.part_ml = p.part_ml;
+  m.out = out;
+  m.out_f32 = 0;
+  {
+    Timer t(c, st, 1);
+    e = launch_merge(m, st);
+  }
+  c->launches++;
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  return XQ_OK;
 }
 
 int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void* q, void* out,
