@@ -190,8 +190,9 @@ int xq_split_plan(const xq_cache* c, int layer, int* n_splits_quantized, int* n_
  * (sequence, kv head) streams.
  * Layouts (all little-endian, one stream per (sequence, kv head)):
  *   codes: tiles of 128 uint32 (bit map: csrc/xq_layout.cuh);
- *   key scale/zero: per token group [2][head_dim] fp16 (scale block, zero block),
- *     permuted within the block; value scale/zero: per 16 tokens
+ *   key scale/zero: [2][group capacity][head_dim] fp16 (all scale blocks, then all
+ *     zero-point blocks; group capacity = stream_stride / (4 * head_dim)), permuted
+ *     within a block; value scale/zero: per 16 tokens
  *     [2][16*head_dim/group_size] fp16; windows: [R][head_dim] bfloat16. */
 int xq_region(const xq_cache* c, int layer, int which, size_t* offset, size_t* stream_stride);
 

@@ -315,22 +315,24 @@ def unpack_v_codes(words, T, D, bits):
 
 def k_meta_position(d: int, D: int) -> int:
     """Index of channel d inside the D-entry scale (or zero-point) block of one
-    key token-group."""
+    key token-group: 8-entry chunks, chunk 4*(d//32) + ((d%16)%8)//2, and inside
+    the chunk the entry ((d//16)%2)*4 + ((d%16)//8)*2 + d%2."""
     cb, kk = divmod(d, 16)
-    return ((kk % 8) // 2) * (D // 4) + cb * 4 + (kk // 8) * 2 + (kk % 2)
+    chunk = (cb // 2) * 4 + (kk % 8) // 2
+    return chunk * 8 + (cb % 2) * 4 + (kk // 8) * 2 + (kk % 2)
 
 
 def pack_k_meta(s_hat: np.ndarray, z_hat: np.ndarray) -> np.ndarray:
-    """[n_groups, D] fp16 scale and zero -> uint16 [n_groups, 2, D]: per token
-    group the permuted scale block followed by the permuted zero-point block."""
+    """[n_groups, D] fp16 scale and zero -> uint16 [2, n_groups, D]: the plane of
+    permuted scale blocks, then the plane of permuted zero-point blocks."""
     n, D = s_hat.shape
-    out = np.zeros((n, 2, D), dtype=np.uint16)
+    out = np.zeros((2, n, D), dtype=np.uint16)
     su = s_hat.astype(np.float16).view(np.uint16)
     zu = z_hat.astype(np.float16).view(np.uint16)
     for d in range(D):
         p = k_meta_position(d, D)
-        out[:, 0, p] = su[:, d]
-        out[:, 1, p] = zu[:, d]
+        out[0, :, p] = su[:, d]
+        out[1, :, p] = zu[:, d]
     return out
 
 

@@ -79,9 +79,9 @@ __global__ void __launch_bounds__(GEN_WARPS * 32) decode_generic_kernel(DecodePa
         if (quant) {
           CodePos pk = k_code_position(t, d, bk, D);
           float c = (float)((kc[pk.word] >> pk.bit) & ((1u << bk) - 1));
-          const uint16_t* mk = km + (size_t)(t / g) * 2 * D;
+          const uint16_t* mk = km + (size_t)(t / g) * D;  // scale plane; the zero-point plane follows it
           int pos = k_meta_position(d, D);
-          kx[j] = fmaf(c, f16_bits_f(mk[pos]), f16_bits_f(mk[D + pos]));
+          kx[j] = fmaf(c, f16_bits_f(mk[pos]), f16_bits_f(mk[(size_t)(dm.nq_cap / g) * D + pos]));
           CodePos pv = v_code_position(t, d, bv, D);
           float cv = (float)((vc[pv.word] >> pv.bit) & ((1u << bv) - 1));
           const uint16_t* mv = vm + (size_t)(t / 16) * 2 * 16 * NG;

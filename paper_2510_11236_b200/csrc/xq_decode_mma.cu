@@ -4,9 +4,9 @@
 // Why mma.sync from registers and not tcgen05: the packed cache delivers
 // ~1.8e13 quantized elements/s at the HBM roofline.  tcgen05.mma takes its
 // operands from shared memory (or TMEM), so every dequantized element would
-// have to be written to and read back from on-chip memory at 2 bytes each --
-// more than the SMs' shared-memory bandwidth.  Here the codes never leave
-// registers in dequantized form: the packed word layout is the A-fragment
+// have to be written to and read back from on-chip memory at one byte or more
+// each -- more than the SMs' shared-memory bandwidth.  Here the codes never
+// leave registers in expanded form: the packed word layout is the A-fragment
 // layout of mma.sync.m16n8k16, so `word & mask` IS an fp16x2 operand register
 // (the code sits in the mantissa bits of an fp16 subnormal: value c * 2^(pos-24)),
 // and scale / zero-point are folded into the other operand:
@@ -18,17 +18,27 @@
 // so a GQA group of up to 8 query heads fills the N = 8 columns.
 //
 // Work split: grid (split, kv head, sequence), sized by the host to one wave of
-// long-lived CTAs.  Every split takes a range of 32-token units of the packed
-// region plus an equal share of the 16-bit window tokens (scalar fp32 path, done
-// first while the first packed stages are in flight).  The 4 warps interleave
-// units; each warp stages its own units in shared memory with cp.async (NST
-// stages ahead) and keeps a private online softmax; the warps' states are merged
-// at the end and the CTA writes one partial (m, l, acc[D]) per query head.  The
-// CTA that finishes last for a (sequence, kv head) -- found with an atomic ticket,
-// never by waiting -- merges the partials and writes the output.
+// long-lived CTAs.  Every split takes a contiguous range of 32-token units of the
+// packed region, cut into four contiguous warp ranges, plus an equal share of the
+// 16-bit window tokens (scalar fp32 path, its loads issued together, done while
+// the first packed stages are in flight).  Each warp stages its own units in
+// shared memory with cp.async (a ring of NST stages: key codes, key scales, value
+// codes, value scale / zero-point of one unit) and, once per 16 units, the key
+// zero-point rows of the next 16 units, from which the q . z biases of those
+// units are computed with one set of MMAs.  The loop is software-pipelined:
+// iteration j computes the logits of unit j + 1 and, from the logits of unit j,
+// the softmax numerators and the value product, so that the two MMA chains
+// overlap.  The softmax reference is only raised when a logit exceeds it by more
+// than TAU (checked with one vote, no shuffles), which keeps every numerator
+// below 2^TAU.  The warps' states are merged at the end and the CTA writes one
+// partial (m, l, acc[D]) per query head.  The CTA that finishes last for a
+// (sequence, kv head) -- found with an atomic ticket, never by waiting -- merges
+// the partials and writes the output.  No thread ever spins on memory.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <math_constants.h>
+
+#include <type_traits>
 
 #include "xq_internal.h"
 
@@ -38,8 +48,10 @@ namespace {
 
 constexpr int MMA_WARPS = 4;
 constexpr int MMA_THREADS = MMA_WARPS * 32;
-constexpr int NST = 4;  // cp.async stages per warp
+constexpr int NST = 4;       // stages per warp: two being consumed, two in flight
 constexpr int HD = 128;
+constexpr int ZROWS = 16;    // units per zero-point bias batch
+constexpr float TAU = 4.0f;  // log2 units a logit may exceed the softmax reference before it is raised
 
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
@@ -72,12 +84,12 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
 }
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void* gmem) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_addr), "l"(gmem));
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_addr), "l"(gmem) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
 
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
@@ -89,6 +101,25 @@ __device__ __forceinline__ uint32_t hmul2_u(uint32_t a, uint32_t b) {
   return *reinterpret_cast<uint32_t*>(&r);
 }
 __device__ __forceinline__ float bf16_to_f(uint16_t u) { return __uint_as_float(((uint32_t)u) << 16); }
+
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ float2 lds64f(uint32_t a) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];\n" : "=f"(v.x), "=f"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts64f(uint32_t a, float x, float y) {
+  asm volatile("st.shared.v2.f32 [%0], {%1,%2};\n" ::"r"(a), "f"(x), "f"(y) : "memory");
+}
 
 // Slot s (0..7) of a word holds, per 16-bit half, a BITS-bit code at bit BITS*s
 // (1-bit words carry a second sub-tile in slots 8..15, reached by a shift of 8).
@@ -123,21 +154,30 @@ struct Stage {
   static constexpr int BYTES = KC + KS + VC + VM;
 };
 
-constexpr int MS = HD + 4;  // state row: acc[HD], m, l, padding (keeps rows 16-byte aligned)
+constexpr int ZBUF_BYTES = ZROWS * 256;    // key zero-point rows of one batch
+constexpr int ZTAB_BYTES = ZROWS * 8 * 4;  // q . z biases [unit][head], fp32, log2 units
+constexpr int MS = HD + 4;                 // state row: acc[HD], m, l, padding (keeps rows 16-byte aligned)
 constexpr int MERGE_BYTES = MMA_WARPS * 8 * MS * 4;
-
-// dynamic shared memory: [stages of 4 warps | merge buffer (aliases the stages)] [q, B-operand order] [window states]
-template <int BK, int BV, int GS>
-constexpr int pipe_bytes() {
-  int pipe = MMA_WARPS * NST * Stage<BK, BV, GS>::BYTES;
-  return pipe > MERGE_BYTES ? pipe : MERGE_BYTES;
-}
 constexpr int Q_BYTES = 32 * 64;
 __host__ __device__ inline int wstate_bytes(int G) { return MMA_WARPS * G * MS * 4; }
 
+// dynamic shared memory:
+//   [per warp: NST stages | zero-point rows | bias table]   (the merge buffer aliases the start after the loop)
+//   [q in B-operand order] [window states]
+template <int BK, int BV, int GS>
+constexpr int warp_bytes() {
+  return NST * Stage<BK, BV, GS>::BYTES + ZBUF_BYTES + ZTAB_BYTES;
+}
+template <int BK, int BV, int GS>
+constexpr int pipe_bytes() {
+  static_assert(MMA_WARPS * warp_bytes<BK, BV, GS>() >= MERGE_BYTES, "the merge buffer aliases the stages");
+  return MMA_WARPS * warp_bytes<BK, BV, GS>();
+}
+
 // ---------------------------------------------------------------------------
-// window path: plain fp32 over 16-bit tokens [t0, t1), one token per warp
-// iteration; each warp leaves its state (acc, m, l per head) in `ws`.
+// window path: plain fp32 over 16-bit tokens [t0, t1); warp w takes tokens
+// t0 + w, t0 + w + 4, ... four at a time (their loads are issued together);
+// each warp leaves its state (acc, m, l per head) in `ws`.
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ void window_tokens(const DecodeParams& p, int t0, int t1, int hk, int b, float* ws) {
   const Dims& dm = p.dm;
@@ -159,27 +199,42 @@ __device__ __forceinline__ void window_tokens(const DecodeParams& p, int t0, int
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[a][j] = 0.f;
   }
-  for (int t = t0 + warp; t < t1; t += MMA_WARPS) {
-    uint2 kr = *reinterpret_cast<const uint2*>(wk + (size_t)t * HD);
-    uint2 vr = *reinterpret_cast<const uint2*>(wv + (size_t)t * HD);
-    float kx[4] = {bf16_to_f(kr.x & 0xffff), bf16_to_f(kr.x >> 16), bf16_to_f(kr.y & 0xffff), bf16_to_f(kr.y >> 16)};
-    float vx[4] = {bf16_to_f(vr.x & 0xffff), bf16_to_f(vr.x >> 16), bf16_to_f(vr.y & 0xffff), bf16_to_f(vr.y >> 16)};
+  for (int tb = t0 + warp; tb < t1; tb += 4 * MMA_WARPS) {
+    uint2 kr[4], vr[4];
 #pragma unroll
-    for (int a = 0; a < 8; ++a) {
-      if (a < G) {
-        float x = q[a][0] * kx[0];
-        x = fmaf(q[a][1], kx[1], x);
-        x = fmaf(q[a][2], kx[2], x);
-        x = fmaf(q[a][3], kx[3], x);
+    for (int i = 0; i < 4; ++i) {
+      const int t = tb + i * MMA_WARPS;
+      kr[i] = vr[i] = make_uint2(0u, 0u);
+      if (t < t1) {
+        kr[i] = *reinterpret_cast<const uint2*>(wk + (size_t)t * HD);
+        vr[i] = *reinterpret_cast<const uint2*>(wv + (size_t)t * HD);
+      }
+    }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-        float mn = fmaxf(m[a], x);
-        float corr = ex2(m[a] - mn);
-        float pe = ex2(x - mn);
-        l[a] = l[a] * corr + pe;
+    for (int i = 0; i < 4; ++i) {
+      if (tb + i * MMA_WARPS < t1) {
+        const float kx[4] = {bf16_to_f(kr[i].x & 0xffff), bf16_to_f(kr[i].x >> 16), bf16_to_f(kr[i].y & 0xffff),
+                             bf16_to_f(kr[i].y >> 16)};
+        const float vx[4] = {bf16_to_f(vr[i].x & 0xffff), bf16_to_f(vr[i].x >> 16), bf16_to_f(vr[i].y & 0xffff),
+                             bf16_to_f(vr[i].y >> 16)};
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[a][j] = acc[a][j] * corr + pe * vx[j];
-        m[a] = mn;
+        for (int a = 0; a < 8; ++a) {
+          if (a < G) {
+            float x = q[a][0] * kx[0];
+            x = fmaf(q[a][1], kx[1], x);
+            x = fmaf(q[a][2], kx[2], x);
+            x = fmaf(q[a][3], kx[3], x);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+            float mn = fmaxf(m[a], x);
+            float corr = ex2(m[a] - mn);
+            float pe = ex2(x - mn);
+            l[a] = l[a] * corr + pe;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[a][j] = acc[a][j] * corr + pe * vx[j];
+            m[a] = mn;
+          }
+        }
       }
     }
   }
@@ -292,6 +347,99 @@ __device__ __forceinline__ void ticket_merge(const DecodeParams& p, int ns, int 
   if (threadIdx.x == 0) p.tickets[bh] = 0u;  // ready for the next launch on this stream
 }
 
+// S^T = Kc (q s)^T for the 32 tokens of the unit staged at `st`:
+// accS[mt] rows = tokens 16 mt + gid (+8), cols = heads 2 tig (+1); values carry a factor 2^-24.
+template <int BK, int BV, int GS>
+__device__ __forceinline__ void unit_logits(uint32_t st, const uint32_t (&qe)[16], float (&accS)[2][4], int lane,
+                                            int tig) {
+  using St = Stage<BK, BV, GS>;
+  uint4 w[2];
+  if (BK == 2) {
+    w[0] = lds128(st + lane * 16);
+    w[1] = lds128(st + 512 + lane * 16);
+  } else {
+    w[0] = lds128(st + lane * 16);
+    w[1] = make_uint4(w[0].x >> 8, w[0].y >> 8, w[0].z >> 8, w[0].w >> 8);
+  }
+  uint4 wsft[2];
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+    wsft[mt] = make_uint4(w[mt].x >> Slots<BK>::SHIFT, w[mt].y >> Slots<BK>::SHIFT, w[mt].z >> Slots<BK>::SHIFT,
+                          w[mt].w >> Slots<BK>::SHIFT);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint4 sv = lds128(st + St::OFF_KS + i * 64 + tig * 16);  // scales of k-steps 2i, 2i+1
+    const uint32_t bq[4] = {hmul2_u(qe[4 * i + 0], sv.x), hmul2_u(qe[4 * i + 1], sv.y),
+                            hmul2_u(qe[4 * i + 2], sv.z), hmul2_u(qe[4 * i + 3], sv.w)};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int s = 2 * i + h;
+      const uint32_t mk = Slots<BK>::mask(s);
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        const uint4& src = Slots<BK>::shifted(s) ? wsft[mt] : w[mt];
+        if (s == 0)
+          mma16816_z(accS[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, bq[2 * h], bq[2 * h + 1]);
+        else
+          mma16816(accS[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, bq[2 * h], bq[2 * h + 1]);
+      }
+    }
+  }
+}
+
+// O^T += Vc^T (p s) for the unit staged at `st`, plus the zero-point and normaliser sums.
+// pb: P as B operand, [16-token tile][b0, b1].
+template <int BK, int BV, int GS>
+__device__ __forceinline__ void unit_values(uint32_t st, const uint32_t (&pb)[2][2], float (&accO)[8][4],
+                                            float (&accZ)[4], int lane, int gid, int tig) {
+  using St = Stage<BK, BV, GS>;
+  constexpr int NG = St::NG;
+  uint4 wv1 = make_uint4(0, 0, 0, 0);
+  if (BV == 1) wv1 = lds128(st + St::OFF_VC + lane * 16);
+#pragma unroll
+  for (int tt = 0; tt < 2; ++tt) {
+    const uint32_t vmeta = st + St::OFF_VM + tt * (64 * NG);
+    uint32_t sv[2 * NG];
+    if (NG == 4) {
+      uint4 x0 = lds128(vmeta + tig * 32), x1 = lds128(vmeta + tig * 32 + 16);
+      sv[0] = x0.x; sv[1] = x0.y; sv[2] = x0.z; sv[3] = x0.w;
+      sv[4 % (2 * NG)] = x1.x; sv[5 % (2 * NG)] = x1.y; sv[6 % (2 * NG)] = x1.z; sv[7 % (2 * NG)] = x1.w;
+    } else {
+      uint4 x0 = lds128(vmeta + tig * 16);
+      sv[0] = x0.x; sv[1] = x0.y; sv[2] = x0.z; sv[3] = x0.w;
+    }
+    uint32_t za0 = 0, za2 = 0;
+    if (gid < NG) {
+      uint2 zz = lds64(vmeta + 32 * NG + tig * (8 * NG) + gid * 8);
+      za0 = zz.x; za2 = zz.y;
+    }
+    const uint32_t ones = (gid == 0) ? 0x3C003C00u : 0u;
+    mma16816(accZ, za0, ones, za2, ones, pb[tt][0], pb[tt][1]);
+    uint32_t pg[NG][2];
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) {
+      pg[gi][0] = hmul2_u(pb[tt][0], sv[2 * gi]);
+      pg[gi][1] = hmul2_u(pb[tt][1], sv[2 * gi + 1]);
+    }
+    uint4 w;
+    if (BV == 2) {
+      w = lds128(st + St::OFF_VC + tt * 512 + lane * 16);
+    } else {
+      w = wv1;
+      if (tt == 1) { w.x >>= 8; w.y >>= 8; w.z >>= 8; w.w >>= 8; }
+    }
+    uint4 wsft = make_uint4(w.x >> Slots<BV>::SHIFT, w.y >> Slots<BV>::SHIFT, w.z >> Slots<BV>::SHIFT,
+                            w.w >> Slots<BV>::SHIFT);
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt) {
+      const uint32_t mk = Slots<BV>::mask(mt);
+      const uint4& src = Slots<BV>::shifted(mt) ? wsft : w;
+      const int gi = (16 * mt) / GS;
+      mma16816(accO[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, pg[gi][0], pg[gi][1]);
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
@@ -299,12 +447,13 @@ template <int BK, int BV, int GS>
 __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams p) {
   using St = Stage<BK, BV, GS>;
   constexpr int NG = St::NG;
+  constexpr int WARP_BYTES = warp_bytes<BK, BV, GS>();
   constexpr int PIPE = pipe_bytes<BK, BV, GS>();
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ int s_flag;
-  float* mb = reinterpret_cast<float*>(smem);                           // merge buffer (after the loop)
-  uint32_t* q_sm = reinterpret_cast<uint32_t*>(smem + PIPE);             // [lane][16] half2
-  float* ws = reinterpret_cast<float*>(smem + PIPE + Q_BYTES);          // window states
+  float* mb = reinterpret_cast<float*>(smem);                   // merge buffer (after the loop)
+  uint32_t* q_sm = reinterpret_cast<uint32_t*>(smem + PIPE);     // [4 chunks][lane][4] half2
+  float* ws = reinterpret_cast<float*>(smem + PIPE + Q_BYTES);  // window states
 
   const Dims& dm = p.dm;
   const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
@@ -328,49 +477,56 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   const int units = p.n_q / 32;
   const int u0 = (int)(((long long)split * units) / ns);
   const int u1 = (int)(((long long)(split + 1) * units) / ns);
-  const int n_my = (u1 - u0 - warp + MMA_WARPS - 1) / MMA_WARPS;  // units of this warp: u0 + warp + 4 j
+  const int n_cta = u1 - u0;
+  const int uw = u0 + (warp * n_cta) / MMA_WARPS;  // this warp's units: [uw, uw + n_my)
+  const int n_my = u0 + ((warp + 1) * n_cta) / MMA_WARPS - uw;
   const int bh = b * dm.Hkv + hk;
 
-  // per-warp cursors into the four streams (this lane's 16-byte column)
-  const int uw = u0 + warp;
+  // this lane's 16-byte column of this warp's first unit in the four streams
   const uint8_t* gk = reinterpret_cast<const uint8_t*>(p.L.k_codes) + (size_t)bh * ((size_t)dm.nq_cap * (HD * BK / 8)) +
                       (size_t)uw * St::KC + lane * 16;
   const uint8_t* gv = reinterpret_cast<const uint8_t*>(p.L.v_codes) + (size_t)bh * ((size_t)dm.nq_cap * (HD * BV / 8)) +
                       (size_t)uw * St::VC + lane * 16;
-  const uint8_t* km_g = reinterpret_cast<const uint8_t*>(p.L.k_meta) + (size_t)bh * (dm.nq_cap / GS) * 512;
-  const uint8_t* gs = km_g + (size_t)((uw * 32) / GS) * 512 + lane * 16;
-  const uint8_t* gm = reinterpret_cast<const uint8_t*>(p.L.v_meta) + (size_t)bh * (dm.nq_cap / 16) * (64 * NG) +
-                      (size_t)uw * St::VM + lane * 16;
-  constexpr int GS_STEP = (MMA_WARPS * 32 / GS) * 512;  // key-scale bytes between a warp's consecutive units
+  const uint8_t* gvm = reinterpret_cast<const uint8_t*>(p.L.v_meta) + (size_t)bh * (dm.nq_cap / 16) * (64 * NG) +
+                       (size_t)uw * St::VM + lane * 16;
+  const size_t plane = (size_t)(dm.nq_cap / GS) * 256;  // bytes of the key scale plane (= of the zero-point plane)
+  const uint8_t* gks = reinterpret_cast<const uint8_t*>(p.L.k_meta) + (size_t)bh * 2 * plane + lane * 16;
+  const uint8_t* gkz = gks + plane;
 
-  const uint32_t stage0 = (uint32_t)__cvta_generic_to_shared(smem) + warp * (NST * St::BYTES);
-  uint32_t st_issue = stage0;
-  int n_issued = 0;
-  auto issue = [&]() {  // stage this warp's next unit
-    if (n_issued < n_my) {
-      const uint32_t s = st_issue + lane * 16;
-      cp_async16(s, gk);
-      if (St::KC == 1024) cp_async16(s + 512, gk + 512);
-      if (lane < 16) cp_async16(s + St::OFF_KS, gs);
-      cp_async16(s + St::OFF_VC, gv);
-      if (St::VC == 1024) cp_async16(s + St::OFF_VC + 512, gv + 512);
-      if (lane * 16 < St::VM) cp_async16(s + St::OFF_VM, gm);
-      gk += MMA_WARPS * St::KC;
-      gv += MMA_WARPS * St::VC;
-      gm += MMA_WARPS * St::VM;
-      gs += GS_STEP;
-    }
-    cp_async_commit();
-    ++n_issued;
-    st_issue = (st_issue == stage0 + (NST - 1) * St::BYTES) ? stage0 : st_issue + St::BYTES;
+  const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(smem);
+  const uint32_t my = sm_base + warp * WARP_BYTES;  // this warp's stages
+  const uint32_t zbuf = my + NST * St::BYTES;
+  const uint32_t ztab = zbuf + ZBUF_BYTES;
+
+  // stage unit jj of this warp (no commit)
+  auto issue_unit = [&](int jj) {
+    const uint32_t s = my + (jj & (NST - 1)) * St::BYTES + lane * 16;
+    const uint8_t* k = gk + (size_t)(uint32_t)jj * St::KC;
+    cp_async16(s, k);
+    if (St::KC == 1024) cp_async16(s + 512, k + 512);
+    if (lane < 16) cp_async16(s + St::OFF_KS, gks + (size_t)(uint32_t)(((uw + jj) * 32) / GS) * 256);
+    const uint8_t* v = gv + (size_t)(uint32_t)jj * St::VC;
+    cp_async16(s + St::OFF_VC, v);
+    if (St::VC == 1024) cp_async16(s + St::OFF_VC + 512, v + 512);
+    if (lane * 16 < St::VM) cp_async16(s + St::OFF_VM, gvm + (size_t)(uint32_t)jj * St::VM);
+  };
+  // stage the key zero-point rows of the groups of units [jb, jb + ZROWS) (no commit)
+  auto issue_zero_rows = [&](int jb) {
+    const int rows = min(ZROWS, n_my - jb);
+    const int g_first = ((uw + jb) * 32) / GS, g_last = ((uw + jb + rows - 1) * 32) / GS;
+    const int bytes = (g_last - g_first + 1) * 256;
+    const uint8_t* src = gkz + (size_t)g_first * 256;
+#pragma unroll
+    for (int i = 0; i < ZBUF_BYTES / 512; ++i)
+      if (i * 512 + lane * 16 < bytes) cp_async16(zbuf + i * 512 + lane * 16, src + i * 512);
   };
 
-  // prologue: start the pipeline, then do this split's share of the window while the copies fly
+  // prologue: start the pipeline (group jj holds unit jj; group 0 also the first zero-point rows)
+  if (n_my > 0) issue_zero_rows(0);
 #pragma unroll
-  for (int j = 0; j < NST - 1; ++j) issue();
-  {
-    const int t0 = (int)(((long long)split * p.r) / ns), t1 = (int)(((long long)(split + 1) * p.r) / ns);
-    window_tokens(p, t0, t1, hk, b, ws);
+  for (int jj = 0; jj < NST - 1; ++jj) {
+    if (jj < n_my) issue_unit(jj);
+    cp_async_commit();
   }
 
   // q of head gid in B-operand order: (q[16s + 2tig + 8j], q[16s + 2tig + 8j + 1]) as fp16, j = 0, 1
@@ -378,17 +534,24 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   {
     const bool real = gid < G;
     const uint16_t* qp = p.q + ((size_t)b * dm.Hq + hk * G + (real ? gid : 0)) * HD + 2 * tig;
+    uint32_t raw[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) raw[i] = real ? *reinterpret_cast<const uint32_t*>(qp + 16 * (i >> 1) + 8 * (i & 1)) : 0u;
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
-        uint32_t raw = real ? *reinterpret_cast<const uint32_t*>(qp + 16 * s + 8 * j) : 0u;
-        float lo = bf16_to_f(raw & 0xffff), hi = bf16_to_f(raw >> 16);
-        if (warp == 0) q_sm[lane * 16 + 2 * s + j] = pack_half2(lo, hi);
+        float lo = bf16_to_f(raw[2 * s + j] & 0xffff), hi = bf16_to_f(raw[2 * s + j] >> 16);
+        if (warp == 0) q_sm[((s >> 1) * 32 + lane) * 4 + (s & 1) * 2 + j] = pack_half2(lo, hi);
         const float sc = 1.0f / (float)(1 << Slots<BK>::e(s));
         qe[2 * s + j] = pack_half2(lo * sc, hi * sc);
       }
     }
+  }
+  // this split's share of the window, while the copies fly
+  {
+    const int t0 = (int)(((long long)split * p.r) / ns), t1 = (int)(((long long)(split + 1) * p.r) / ns);
+    window_tokens(p, t0, t1, hk, b, ws);
   }
   __syncthreads();
 
@@ -400,108 +563,77 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   for (int mt = 0; mt < 8; ++mt)
 #pragma unroll
     for (int i = 0; i < 4; ++i) accO[mt][i] = 0.f;
-  float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;  // running max (log2 units) of heads 2 tig, 2 tig + 1
-  float zb[4] = {0.f, 0.f, 0.f, 0.f};            // key zero-point bias of 16 units: rows = units
-  uint32_t st_read = stage0;
+  float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;  // softmax reference (log2 units) of heads 2 tig, 2 tig + 1
+  float accS[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 
-  for (int j = 0; j < n_my; ++j) {
-    __syncwarp();  // everyone is done with the stage that is about to be refilled
-    issue();
+  if (n_my > 0) {
+    cp_async_wait<NST - 2>();  // unit 0 and the first zero-point rows have landed
+    __syncwarp();
+    unit_logits<BK, BV, GS>(my, qe, accS, lane, tig);
+  }
 
-    if ((j & 15) == 0) {
-      // bias tile: zb[unit row][head] = scale * sum_d q_d z_d for this warp's next 16 units (plain loads)
-      const int ja = j + gid, jb = j + gid + 8;
-      const uint8_t* za = km_g + (size_t)(((uw + MMA_WARPS * ja) * 32) / GS) * 512 + 256 + tig * 64;
-      const uint8_t* zc = km_g + (size_t)(((uw + MMA_WARPS * jb) * 32) / GS) * 512 + 256 + tig * 64;
-      uint4 ra[4], rb[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        ra[i] = (ja < n_my) ? *reinterpret_cast<const uint4*>(za + i * 16) : make_uint4(0, 0, 0, 0);
-        rb[i] = (jb < n_my) ? *reinterpret_cast<const uint4*>(zc + i * 16) : make_uint4(0, 0, 0, 0);
-      }
-      const uint4* qs = reinterpret_cast<const uint4*>(q_sm + lane * 16);
+  // One iteration: bias table every ZROWS units, refill of the stage unit j - 1 used, softmax reference,
+  // numerators of unit j, then (MORE) logits of unit j + 1 next to the value product of unit j.
+  auto step = [&](int j, auto more_tag) {
+    constexpr bool MORE = decltype(more_tag)::value;
+    const int jr = j & (ZROWS - 1);
+    if (jr == 0) {
+      // bias table of units [j, j + 16): ztab[row][head] = scale * sum_d q_d z_d (log2 units)
+      const int rows = min(ZROWS, n_my - j);
+      const int g_first = ((uw + j) * 32) / GS;
+      const int ra_row = ((uw + j + min(gid, rows - 1)) * 32) / GS - g_first;
+      const int rb_row = ((uw + j + min(gid + 8, rows - 1)) * 32) / GS - g_first;
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        uint4 qq = qs[i];  // k-steps 2i, 2i+1
-        mma16816(acc, ra[i].x, rb[i].x, ra[i].y, rb[i].y, qq.x, qq.y);
-        mma16816(acc, ra[i].z, rb[i].z, ra[i].w, rb[i].w, qq.z, qq.w);
+        const uint4 ra = lds128(zbuf + ra_row * 256 + i * 64 + tig * 16);
+        const uint4 rb = lds128(zbuf + rb_row * 256 + i * 64 + tig * 16);
+        const uint4 qq = *reinterpret_cast<const uint4*>(q_sm + (i * 32 + lane) * 4);  // k-steps 2i, 2i+1
+        mma16816(acc, ra.x, rb.x, ra.y, rb.y, qq.x, qq.y);
+        mma16816(acc, ra.z, rb.z, ra.w, rb.w, qq.z, qq.w);
       }
-#pragma unroll
-      for (int i = 0; i < 4; ++i) zb[i] = acc[i] * scale2;
+      sts64f(ztab + gid * 32 + tig * 8, acc[0] * scale2, acc[1] * scale2);
+      sts64f(ztab + (gid + 8) * 32 + tig * 8, acc[2] * scale2, acc[3] * scale2);
+      __syncwarp();  // table visible; every lane is done with the rows
+      if (j + ZROWS < n_my) issue_zero_rows(j + ZROWS);  // lands with this iteration's group, 16 units early
     }
 
-    cp_async_wait<NST - 1>();
-    __syncwarp();
-    const uint32_t st = st_read;
-    st_read = (st_read == stage0 + (NST - 1) * St::BYTES) ? stage0 : st_read + St::BYTES;
-    auto lds128 = [](uint32_t a) {
-      uint4 v;
-      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
-      return v;
-    };
-    auto lds64 = [](uint32_t a) {
-      uint2 v;
-      asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "r"(a));
-      return v;
-    };
+    __syncwarp();  // every lane is done with the stage of unit j - 1
+    if (j + NST - 1 < n_my) issue_unit(j + NST - 1);
+    cp_async_commit();
 
-    // ---- S^T = Kc (q s)^T for the unit's 32 tokens ----
-    uint32_t bq[16];
+    // ---- softmax reference: raise it only when a logit of unit j exceeds it by more than TAU ----
+    const float2 bz = lds64f(ztab + jr * 32 + tig * 8);
+    {
+      const float lm0 = fmaxf(fmaxf(accS[0][0], accS[0][2]), fmaxf(accS[1][0], accS[1][2]));
+      const float lm1 = fmaxf(fmaxf(accS[0][1], accS[0][3]), fmaxf(accS[1][1], accS[1][3]));
+      float x0 = fmaf(lm0, c1, bz.x), x1 = fmaf(lm1, c1, bz.y);
+      if (__any_sync(0xffffffffu, (x0 > m0 + TAU) | (x1 > m1 + TAU))) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      uint4 sv = lds128(st + St::OFF_KS + tig * 64 + i * 16);
-      bq[4 * i + 0] = hmul2_u(qe[4 * i + 0], sv.x);
-      bq[4 * i + 1] = hmul2_u(qe[4 * i + 1], sv.y);
-      bq[4 * i + 2] = hmul2_u(qe[4 * i + 2], sv.z);
-      bq[4 * i + 3] = hmul2_u(qe[4 * i + 3], sv.w);
-    }
-    float accS[2][4];
+        for (int o = 4; o < 32; o <<= 1) {
+          x0 = fmaxf(x0, __shfl_xor_sync(0xffffffffu, x0, o));
+          x1 = fmaxf(x1, __shfl_xor_sync(0xffffffffu, x1, o));
+        }
+        const float mn0 = fmaxf(m0, x0), mn1 = fmaxf(m1, x1);
+        const float f0 = ex2(m0 - mn0), f1 = ex2(m1 - mn1);
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt) {
-      uint4 w;
-      if (BK == 2) {
-        w = lds128(st + mt * 512 + lane * 16);
-      } else {
-        w = lds128(st + lane * 16);
-        if (mt == 1) { w.x >>= 8; w.y >>= 8; w.z >>= 8; w.w >>= 8; }
-      }
-      uint4 wsft = make_uint4(w.x >> Slots<BK>::SHIFT, w.y >> Slots<BK>::SHIFT, w.z >> Slots<BK>::SHIFT,
-                              w.w >> Slots<BK>::SHIFT);
-#pragma unroll
-      for (int s = 0; s < 8; ++s) {
-        const uint32_t mk = Slots<BK>::mask(s);
-        const uint4& src = Slots<BK>::shifted(s) ? wsft : w;
-        if (s == 0)
-          mma16816_z(accS[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, bq[0], bq[1]);
-        else
-          mma16816(accS[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, bq[2 * s], bq[2 * s + 1]);
+        for (int mt = 0; mt < 8; ++mt) {
+          accO[mt][0] *= f0; accO[mt][1] *= f1; accO[mt][2] *= f0; accO[mt][3] *= f1;
+        }
+        accZ[0] *= f0; accZ[1] *= f1; accZ[2] *= f0; accZ[3] *= f1;
+        m0 = mn0; m1 = mn1;
       }
     }
 
-    // ---- online softmax (log2 domain); the unit's key bias is common to its 32 tokens ----
-    const int jr = j & 15;
-    const float bz0 = __shfl_sync(0xffffffffu, jr < 8 ? zb[0] : zb[2], (jr & 7) * 4 + tig);
-    const float bz1 = __shfl_sync(0xffffffffu, jr < 8 ? zb[1] : zb[3], (jr & 7) * 4 + tig);
-    float r0 = fmaxf(fmaxf(accS[0][0], accS[0][2]), fmaxf(accS[1][0], accS[1][2]));
-    float r1 = fmaxf(fmaxf(accS[0][1], accS[0][3]), fmaxf(accS[1][1], accS[1][3]));
-#pragma unroll
-    for (int o = 4; o < 32; o <<= 1) {
-      r0 = fmaxf(r0, __shfl_xor_sync(0xffffffffu, r0, o));
-      r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, o));
+    if (MORE) {
+      cp_async_wait<NST - 2>();  // unit j + 1 has landed
+      __syncwarp();
     }
-    const float mn0 = fmaxf(m0, fmaf(r0, c1, bz0)), mn1 = fmaxf(m1, fmaf(r1, c1, bz1));
-    if (__any_sync(0xffffffffu, (mn0 > m0) | (mn1 > m1))) {
-      const float f0 = ex2(m0 - mn0), f1 = ex2(m1 - mn1);
-#pragma unroll
-      for (int mt = 0; mt < 8; ++mt) {
-        accO[mt][0] *= f0; accO[mt][1] *= f1; accO[mt][2] *= f0; accO[mt][3] *= f1;
-      }
-      accZ[0] *= f0; accZ[1] *= f1; accZ[2] *= f0; accZ[3] *= f1;
-      m0 = mn0; m1 = mn1;
-    }
-    const float t0 = bz0 - m0, t1 = bz1 - m1;
-    uint32_t pb[2][2];  // P as B operand: [16-token tile][b0, b1]
+    const uint32_t st = my + (j & (NST - 1)) * St::BYTES;
+
+    // ---- softmax numerators of unit j (log2 domain; the unit's key bias is common to its 32 tokens) ----
+    const float t0 = bz.x - m0, t1 = bz.y - m1;
+    uint32_t pb[2][2];
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
       float p0 = ex2(fmaf(accS[mt][0], c1, t0)), p1 = ex2(fmaf(accS[mt][1], c1, t1));
@@ -509,53 +641,12 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
       pb[mt][0] = movmatrix_trans(pack_half2(p0, p1));
       pb[mt][1] = movmatrix_trans(pack_half2(p2, p3));
     }
+    if (MORE) unit_logits<BK, BV, GS>(my + ((j + 1) & (NST - 1)) * St::BYTES, qe, accS, lane, tig);
+    unit_values<BK, BV, GS>(st, pb, accO, accZ, lane, gid, tig);
+  };
 
-    // ---- O^T += Vc^T (p s), zero-point and normaliser sums ----
-    uint4 wv1 = make_uint4(0, 0, 0, 0);
-    if (BV == 1) wv1 = lds128(st + St::OFF_VC + lane * 16);
-#pragma unroll
-    for (int tt = 0; tt < 2; ++tt) {
-      const uint32_t vmeta = st + St::OFF_VM + tt * (64 * NG);
-      uint32_t sv[2 * NG];
-      if (NG == 4) {
-        uint4 x0 = lds128(vmeta + tig * 32), x1 = lds128(vmeta + tig * 32 + 16);
-        sv[0] = x0.x; sv[1] = x0.y; sv[2] = x0.z; sv[3] = x0.w;
-        sv[4 % (2 * NG)] = x1.x; sv[5 % (2 * NG)] = x1.y; sv[6 % (2 * NG)] = x1.z; sv[7 % (2 * NG)] = x1.w;
-      } else {
-        uint4 x0 = lds128(vmeta + tig * 16);
-        sv[0] = x0.x; sv[1] = x0.y; sv[2] = x0.z; sv[3] = x0.w;
-      }
-      uint32_t za0 = 0, za2 = 0;
-      if (gid < NG) {
-        uint2 zz = lds64(vmeta + 32 * NG + tig * (8 * NG) + gid * 8);
-        za0 = zz.x; za2 = zz.y;
-      }
-      const uint32_t ones = (gid == 0) ? 0x3C003C00u : 0u;
-      mma16816(accZ, za0, ones, za2, ones, pb[tt][0], pb[tt][1]);
-      uint32_t pg[NG][2];
-#pragma unroll
-      for (int gi = 0; gi < NG; ++gi) {
-        pg[gi][0] = hmul2_u(pb[tt][0], sv[2 * gi]);
-        pg[gi][1] = hmul2_u(pb[tt][1], sv[2 * gi + 1]);
-      }
-      uint4 w;
-      if (BV == 2) {
-        w = lds128(st + St::OFF_VC + tt * 512 + lane * 16);
-      } else {
-        w = wv1;
-        if (tt == 1) { w.x >>= 8; w.y >>= 8; w.z >>= 8; w.w >>= 8; }
-      }
-      uint4 wsft = make_uint4(w.x >> Slots<BV>::SHIFT, w.y >> Slots<BV>::SHIFT, w.z >> Slots<BV>::SHIFT,
-                              w.w >> Slots<BV>::SHIFT);
-#pragma unroll
-      for (int mt = 0; mt < 8; ++mt) {
-        const uint32_t mk = Slots<BV>::mask(mt);
-        const uint4& src = Slots<BV>::shifted(mt) ? wsft : w;
-        const int gi = (16 * mt) / GS;
-        mma16816(accO[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, pg[gi][0], pg[gi][1]);
-      }
-    }
-  }
+  for (int j = 0; j + 1 < n_my; ++j) step(j, std::true_type{});
+  if (n_my > 0) step(n_my - 1, std::false_type{});
   cp_async_wait<0>();
   __syncthreads();  // all warps are done with their stages: the memory becomes the merge buffer
 
@@ -595,8 +686,13 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
 }
 
 template <int BK, int BV, int GS>
+int smem_bytes(int G) {
+  return pipe_bytes<BK, BV, GS>() + Q_BYTES + wstate_bytes(G);
+}
+
+template <int BK, int BV, int GS>
 cudaError_t launch_t(const DecodeParams& p, cudaStream_t st) {
-  const int smem = pipe_bytes<BK, BV, GS>() + Q_BYTES + wstate_bytes(p.dm.G);
+  const int smem = smem_bytes<BK, BV, GS>(p.dm.G);
   static int configured = 0;
   if (configured < smem) {
     cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<BK, BV, GS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -609,6 +705,22 @@ cudaError_t launch_t(const DecodeParams& p, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+template <int BK, int BV, int GS>
+int ctas_per_sm_t(int G) {
+  const int smem = smem_bytes<BK, BV, GS>(G);
+  if (cudaFuncSetAttribute(decode_mma_kernel<BK, BV, GS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  int n = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_mma_kernel<BK, BV, GS>, MMA_THREADS, smem) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return n;
+}
+
 }  // namespace
 
 bool decode_mma_supported(const Dims& dm, int bk, int bv) {
@@ -616,20 +728,28 @@ bool decode_mma_supported(const Dims& dm, int bk, int bv) {
   return dm.D == HD && dm.G <= 8 && (dm.g == 32 || dm.g == 64);
 }
 
-int decode_mma_ctas_per_sm() { return 3; }
+#define XQ_DISPATCH(FN, ...)                    \
+  switch (bk * 100 + bv * 10 + (g == 64)) {     \
+    case 220: return FN<2, 2, 32>(__VA_ARGS__); \
+    case 221: return FN<2, 2, 64>(__VA_ARGS__); \
+    case 210: return FN<2, 1, 32>(__VA_ARGS__); \
+    case 211: return FN<2, 1, 64>(__VA_ARGS__); \
+    case 120: return FN<1, 2, 32>(__VA_ARGS__); \
+    case 121: return FN<1, 2, 64>(__VA_ARGS__); \
+    case 110: return FN<1, 1, 32>(__VA_ARGS__); \
+    case 111: return FN<1, 1, 64>(__VA_ARGS__); \
+  }
+
+// Resident CTAs per SM of the kernel variant for these bit-widths (0 if unknown: no device).
+int decode_mma_ctas_per_sm(const Dims& dm, int bk, int bv) {
+  const int g = dm.g;
+  XQ_DISPATCH(ctas_per_sm_t, dm.G)
+  return 0;
+}
 
 cudaError_t launch_decode_mma(const DecodeParams& p, cudaStream_t st) {
-  const int key = p.L.bk * 100 + p.L.bv * 10 + (p.dm.g == 64);
-  switch (key) {
-    case 220: return launch_t<2, 2, 32>(p, st);
-    case 221: return launch_t<2, 2, 64>(p, st);
-    case 210: return launch_t<2, 1, 32>(p, st);
-    case 211: return launch_t<2, 1, 64>(p, st);
-    case 120: return launch_t<1, 2, 32>(p, st);
-    case 121: return launch_t<1, 2, 64>(p, st);
-    case 110: return launch_t<1, 1, 32>(p, st);
-    case 111: return launch_t<1, 1, 64>(p, st);
-  }
+  const int bk = p.L.bk, bv = p.L.bv, g = p.dm.g;
+  XQ_DISPATCH(launch_t, p, st)
   return cudaErrorInvalidValue;
 }
 

@@ -142,6 +142,7 @@ struct xq_cache {
   float scale;
   int sm_count;
   bool tickets_clean;  // the ticket counters have been zeroed on a stream
+  int mma_ctas[2][2];  // resident CTAs per SM of the tensor-core kernel by (key bits - 1, value bits - 1); 0 = not asked yet
   // timing
   bool timing;
   std::vector<EventPair> pool;
@@ -179,6 +180,16 @@ bool layer_uses_mma(const xq_cache* c, int l) {
   return decode_mma_supported(c->plan.dm, layer_bits(l, c->cfg.kq), layer_bits(l, c->cfg.vq));
 }
 
+int mma_ctas_per_sm(const xq_cache* c, int l) {
+  int bk = layer_bits(l, c->cfg.kq), bv = layer_bits(l, c->cfg.vq);
+  int& slot = const_cast<xq_cache*>(c)->mma_ctas[bk - 1][bv - 1];
+  if (slot == 0) {
+    slot = decode_mma_ctas_per_sm(c->plan.dm, bk, bv);
+    if (slot <= 0) slot = 3;  // no device to ask
+  }
+  return slot;
+}
+
 // Splits per (sequence, kv head) stream.  Tensor-core kernel: every split takes
 // packed units and a share of the window (ns_w = 0 unless nothing is packed yet),
 // sized towards whole waves of resident CTAs.  Generic kernel: separate splits for
@@ -202,7 +213,7 @@ void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w) {
       ns_q = c->cfg.n_splits < units ? c->cfg.n_splits : units;
       return;
     }
-    const double slots = (double)c->sm_count * decode_mma_ctas_per_sm();
+    const double slots = (double)c->sm_count * mma_ctas_per_sm(c, l);
     int best = 1;
     double best_score = -1.0;
     for (int ns = 1; ns <= 64 && ns <= units; ++ns) {
@@ -366,6 +377,7 @@ int xq_create(const xq_config* cfg, void* dev_workspace, size_t bytes, xq_cache*
   c->used = 0;
   c->sm_count = 148;
   c->tickets_clean = false;
+  memset(c->mma_ctas, 0, sizeof(c->mma_ctas));
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) == cudaSuccess &&
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)

@@ -14,7 +14,7 @@ struct Dims {
 struct LayerPtrs {
   uint16_t* win_k;   // [B,Hkv,R,D] bf16
   uint16_t* win_v;
-  uint16_t* k_meta;  // [B,Hkv,nq_cap/g,2,D] fp16
+  uint16_t* k_meta;  // [B,Hkv,2,nq_cap/g,D] fp16 (scale plane, zero-point plane)
   uint16_t* v_meta;  // [B,Hkv,nq_cap/16,2,16*NG] fp16
   uint32_t* k_codes; // [B,Hkv,nq_cap*D*bk/32]
   uint32_t* v_codes;
@@ -77,7 +77,7 @@ cudaError_t launch_window_append(const WindowParams& p, cudaStream_t st);
 cudaError_t launch_decode_generic(const DecodeParams& p, cudaStream_t st);
 cudaError_t launch_decode_mma(const DecodeParams& p, cudaStream_t st);
 bool decode_mma_supported(const Dims& dm, int bk, int bv);
-int decode_mma_ctas_per_sm();
+int decode_mma_ctas_per_sm(const Dims& dm, int bk, int bv);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t st);
 
 }  // namespace xq

@@ -14,9 +14,14 @@
 // is, for every slot, a ready fp16x2 fragment register whose two halves hold the
 // integer code times 2^(bits*slot) as fp16 subnormals (value * 2^-24).
 //
-// Key scale/zero: per group of g tokens two blocks of D fp16 (scale, then zero),
-// channel d at index ((d%16 % 8)/2) * (D/4) + (d/16) * 4 + ((d%16)/8) * 2 + d%2,
-// so that the 32 values a B-operand thread needs are contiguous.
+// Key scale/zero: per stream two planes of [groups][D] fp16, all scale blocks
+// first, then all zero-point blocks (plane stride = group capacity * D), so that
+// the zero-point blocks of consecutive token groups are contiguous.  Inside a
+// block the D values are cut into 16-byte chunks, chunk (d/32)*4 + ((d%16)%8)/2
+// holding, for the two 16-channel blocks 2*(d/32) and 2*(d/32)+1, the four
+// values (d%16 in {2t, 2t+1, 2t+8, 2t+9}) that B-operand thread t of an
+// mma.sync.m16n8k16 needs: index ((d/16)%2)*4 + ((d%16)/8)*2 + d%2 in the chunk.
+// The four threads of a quad then read 64 contiguous bytes per load.
 // Value scale/zero: per 16 tokens two blocks of 16*NG fp16 (NG = D/g), entry
 // (token tk, group gi) at ((tk%8)/2) * (4*NG) + gi*4 + (tk/8)*2 + tk%2.
 #pragma once
@@ -55,8 +60,10 @@ __host__ __device__ inline CodePos v_code_position(int t, int d, int bits, int D
 }
 
 __host__ __device__ inline int k_meta_position(int d, int D) {
+  (void)D;
   int cb = d / 16, kk = d % 16;
-  return ((kk & 7) >> 1) * (D / 4) + cb * 4 + (kk >> 3) * 2 + (kk & 1);
+  int chunk = (cb >> 1) * 4 + ((kk & 7) >> 1);
+  return chunk * 8 + (cb & 1) * 4 + (kk >> 3) * 2 + (kk & 1);
 }
 
 __host__ __device__ inline int v_meta_position(int tk, int gi, int n_g) {

@@ -87,10 +87,11 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
       group_params(mn, mx, bits, eta, z, s, zh, sh);
       z_arr[item] = z;
       s_arr[item] = s;
-      size_t grp = (size_t)bh * (dm.nq_cap / g) + (tq0 / g + gl);
+      const size_t cap_g = (size_t)(dm.nq_cap / g);
+      size_t grp = (size_t)bh * 2 * cap_g + (tq0 / g + gl);  // scale plane, then zero-point plane
       int pos = k_meta_position(d, D);
-      meta[(grp * 2 + 0) * D + pos] = sh;
-      meta[(grp * 2 + 1) * D + pos] = zh;
+      meta[grp * D + pos] = sh;
+      meta[(grp + cap_g) * D + pos] = zh;
     }
   } else {
     // values: one group per (token, run of g channels)

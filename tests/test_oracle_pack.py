@@ -66,10 +66,10 @@ def test_meta_pack_places_values():
     rng = np.random.default_rng(0)
     s = rng.random((3, 128)).astype(np.float16); z = rng.random((3, 128)).astype(np.float16)
     m = O.pack_k_meta(s, z)
-    assert m.shape == (3, 2, 128)
+    assert m.shape == (2, 3, 128)
     for d in (0, 1, 17, 127):
         p = O.k_meta_position(d, 128)
-        assert m[2, 0, p] == s[2, d].view(np.uint16) and m[2, 1, p] == z[2, d].view(np.uint16)
+        assert m[0, 2, p] == s[2, d].view(np.uint16) and m[1, 2, p] == z[2, d].view(np.uint16)
     s = rng.random((32, 4)).astype(np.float16); z = rng.random((32, 4)).astype(np.float16)
     m = O.pack_v_meta(s, z)
     assert m.shape == (2, 2, 64)
