@@ -38,8 +38,6 @@
 #include <cuda_fp16.h>
 #include <math_constants.h>
 
-#include <type_traits>
-
 #include "xq_internal.h"
 
 namespace xq {
@@ -85,6 +83,17 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void* gmem) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_addr), "l"(gmem) : "memory");
+}
+// the same, issued only where `on` is true (a predicated instruction, no branch)
+__device__ __forceinline__ void cp_async16_if(uint32_t smem_addr, const void* gmem, bool on) {
+  asm volatile(
+      "{\n"
+      ".reg .pred q;\n"
+      "setp.ne.b32 q, %2, 0;\n"
+      "@q cp.async.cg.shared.global [%0], [%1], 16;\n"
+      "}\n" ::"r"(smem_addr),
+      "l"(gmem), "r"((int)on)
+      : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
@@ -176,47 +185,68 @@ constexpr int pipe_bytes() {
 
 // ---------------------------------------------------------------------------
 // window path: plain fp32 over 16-bit tokens [t0, t1); warp w takes tokens
-// t0 + w, t0 + w + 4, ... four at a time (their loads are issued together);
-// each warp leaves its state (acc, m, l per head) in `ws`.
+// t0 + w, t0 + w + 4, ... four at a time.  The loads of q and of the first four
+// tokens are issued by window_preload (before the packed stream's copies are
+// queued), later rounds load one round ahead.  Each warp leaves its state
+// (acc, m, l per head) in `ws`.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ void window_tokens(const DecodeParams& p, int t0, int t1, int hk, int b, float* ws) {
+struct WindowRegs {
+  uint2 q[8];   // this lane's 4 channels of each query head of the group
+  uint2 k[4];   // this lane's 4 channels of up to four window tokens
+  uint2 v[4];
+};
+
+__device__ __forceinline__ void window_load_round(const DecodeParams& p, int tb, int t1, int hk, int b, uint2 (&k)[4],
+                                                  uint2 (&v)[4]) {
+  const Dims& dm = p.dm;
+  const int lane = threadIdx.x & 31;
+  const size_t row0 = (size_t)(b * dm.Hkv + hk) * dm.R;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int t = tb + i * MMA_WARPS;
+    k[i] = v[i] = make_uint2(0u, 0u);
+    if (t < t1) {
+      k[i] = *reinterpret_cast<const uint2*>(p.L.win_k + (row0 + t) * HD + lane * 4);
+      v[i] = *reinterpret_cast<const uint2*>(p.L.win_v + (row0 + t) * HD + lane * 4);
+    }
+  }
+}
+
+__device__ __forceinline__ void window_preload(const DecodeParams& p, int t0, int t1, int hk, int b, WindowRegs& w) {
   const Dims& dm = p.dm;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int bh = b * dm.Hkv + hk;
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+    w.q[a] = *reinterpret_cast<const uint2*>(p.q + ((size_t)b * dm.Hq + hk * dm.G + (a < dm.G ? a : 0)) * HD + lane * 4);
+  window_load_round(p, t0 + warp, t1, hk, b, w.k, w.v);
+}
+
+__device__ __forceinline__ void window_tokens(const DecodeParams& p, int t0, int t1, int hk, int b, float* ws,
+                                              WindowRegs& w) {
+  const Dims& dm = p.dm;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = dm.G;
-  const uint16_t* wk = p.L.win_k + (size_t)bh * dm.R * HD + lane * 4;
-  const uint16_t* wv = p.L.win_v + (size_t)bh * dm.R * HD + lane * 4;
   const float scale2 = p.scale * 1.4426950408889634f;
   float q[8][4], acc[8][4], m[8], l[8];
 #pragma unroll
   for (int a = 0; a < 8; ++a) {
     m[a] = -CUDART_INF_F;
     l[a] = 0.f;
-    const uint16_t* qp = p.q + ((size_t)b * dm.Hq + hk * G + (a < G ? a : 0)) * HD + lane * 4;
-    uint2 raw = *reinterpret_cast<const uint2*>(qp);
-    q[a][0] = bf16_to_f(raw.x & 0xffff) * scale2; q[a][1] = bf16_to_f(raw.x >> 16) * scale2;
-    q[a][2] = bf16_to_f(raw.y & 0xffff) * scale2; q[a][3] = bf16_to_f(raw.y >> 16) * scale2;
+    q[a][0] = bf16_to_f(w.q[a].x & 0xffff) * scale2; q[a][1] = bf16_to_f(w.q[a].x >> 16) * scale2;
+    q[a][2] = bf16_to_f(w.q[a].y & 0xffff) * scale2; q[a][3] = bf16_to_f(w.q[a].y >> 16) * scale2;
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[a][j] = 0.f;
   }
   for (int tb = t0 + warp; tb < t1; tb += 4 * MMA_WARPS) {
-    uint2 kr[4], vr[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int t = tb + i * MMA_WARPS;
-      kr[i] = vr[i] = make_uint2(0u, 0u);
-      if (t < t1) {
-        kr[i] = *reinterpret_cast<const uint2*>(wk + (size_t)t * HD);
-        vr[i] = *reinterpret_cast<const uint2*>(wv + (size_t)t * HD);
-      }
-    }
+    uint2 kn[4], vn[4];
+    window_load_round(p, tb + 4 * MMA_WARPS, t1, hk, b, kn, vn);  // next round, in flight during this one
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       if (tb + i * MMA_WARPS < t1) {
-        const float kx[4] = {bf16_to_f(kr[i].x & 0xffff), bf16_to_f(kr[i].x >> 16), bf16_to_f(kr[i].y & 0xffff),
-                             bf16_to_f(kr[i].y >> 16)};
-        const float vx[4] = {bf16_to_f(vr[i].x & 0xffff), bf16_to_f(vr[i].x >> 16), bf16_to_f(vr[i].y & 0xffff),
-                             bf16_to_f(vr[i].y >> 16)};
+        const float kx[4] = {bf16_to_f(w.k[i].x & 0xffff), bf16_to_f(w.k[i].x >> 16), bf16_to_f(w.k[i].y & 0xffff),
+                             bf16_to_f(w.k[i].y >> 16)};
+        const float vx[4] = {bf16_to_f(w.v[i].x & 0xffff), bf16_to_f(w.v[i].x >> 16), bf16_to_f(w.v[i].y & 0xffff),
+                             bf16_to_f(w.v[i].y >> 16)};
 #pragma unroll
         for (int a = 0; a < 8; ++a) {
           if (a < G) {
@@ -236,6 +266,11 @@ __device__ __forceinline__ void window_tokens(const DecodeParams& p, int t0, int
           }
         }
       }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      w.k[i] = kn[i];
+      w.v[i] = vn[i];
     }
   }
   float* mine = ws + (size_t)warp * G * MS;
@@ -466,7 +501,9 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     const int tiles = (p.r + 15) / 16;
     const int t0 = (int)(((long long)split * tiles) / ns) * 16;
     const int t1 = min((int)(((long long)(split + 1) * tiles) / ns) * 16, p.r);
-    window_tokens(p, t0, t1, hk, b, ws);
+    WindowRegs wr;
+    window_preload(p, t0, t1, hk, b, wr);
+    window_tokens(p, t0, t1, hk, b, ws, wr);
     __syncthreads();
     write_partial(p, nullptr, ws, split, ns, hk, b);
     ticket_merge(p, ns, hk, b, &s_flag);
@@ -498,17 +535,18 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   const uint32_t zbuf = my + NST * St::BYTES;
   const uint32_t ztab = zbuf + ZBUF_BYTES;
 
-  // stage unit jj of this warp (no commit)
-  auto issue_unit = [&](int jj) {
-    const uint32_t s = my + (jj & (NST - 1)) * St::BYTES + lane * 16;
+  // stage unit jj of this warp at byte offset `soff` of its ring, if it exists (no commit, no branch)
+  auto issue_unit = [&](int jj, uint32_t soff) {
+    const bool on = jj < n_my;
+    const uint32_t s = my + soff + lane * 16;
     const uint8_t* k = gk + (size_t)(uint32_t)jj * St::KC;
-    cp_async16(s, k);
-    if (St::KC == 1024) cp_async16(s + 512, k + 512);
-    if (lane < 16) cp_async16(s + St::OFF_KS, gks + (size_t)(uint32_t)(((uw + jj) * 32) / GS) * 256);
+    cp_async16_if(s, k, on);
+    if (St::KC == 1024) cp_async16_if(s + 512, k + 512, on);
+    cp_async16_if(s + St::OFF_KS, gks + (size_t)(uint32_t)(((uw + jj) * 32) / GS) * 256, on && lane < 16);
     const uint8_t* v = gv + (size_t)(uint32_t)jj * St::VC;
-    cp_async16(s + St::OFF_VC, v);
-    if (St::VC == 1024) cp_async16(s + St::OFF_VC + 512, v + 512);
-    if (lane * 16 < St::VM) cp_async16(s + St::OFF_VM, gvm + (size_t)(uint32_t)jj * St::VM);
+    cp_async16_if(s + St::OFF_VC, v, on);
+    if (St::VC == 1024) cp_async16_if(s + St::OFF_VC + 512, v + 512, on);
+    cp_async16_if(s + St::OFF_VM, gvm + (size_t)(uint32_t)jj * St::VM, on && lane * 16 < St::VM);
   };
   // stage the key zero-point rows of the groups of units [jb, jb + ZROWS) (no commit)
   auto issue_zero_rows = [&](int jb) {
@@ -521,38 +559,39 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
       if (i * 512 + lane * 16 < bytes) cp_async16(zbuf + i * 512 + lane * 16, src + i * 512);
   };
 
-  // prologue: start the pipeline (group jj holds unit jj; group 0 also the first zero-point rows)
-  if (n_my > 0) issue_zero_rows(0);
-#pragma unroll
-  for (int jj = 0; jj < NST - 1; ++jj) {
-    if (jj < n_my) issue_unit(jj);
-    cp_async_commit();
-  }
-
-  // q of head gid in B-operand order: (q[16s + 2tig + 8j], q[16s + 2tig + 8j + 1]) as fp16, j = 0, 1
-  uint32_t qe[16];  // pre-scaled by 2^-e(s), the weight the code's slot carries
+  // Loads the prologue waits for go out first: q in B-operand order, q and the first rows of this split's
+  // share of the window.  Then the packed stream's copies are queued behind them.
+  const int wt0 = (int)(((long long)split * p.r) / ns), wt1 = (int)(((long long)(split + 1) * p.r) / ns);
+  uint32_t raw[16];  // q of head gid: (q[16s + 2tig + 8j], q[16s + 2tig + 8j + 1]), j = 0, 1
   {
     const bool real = gid < G;
     const uint16_t* qp = p.q + ((size_t)b * dm.Hq + hk * G + (real ? gid : 0)) * HD + 2 * tig;
-    uint32_t raw[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) raw[i] = real ? *reinterpret_cast<const uint32_t*>(qp + 16 * (i >> 1) + 8 * (i & 1)) : 0u;
+  }
+  WindowRegs wr;
+  window_preload(p, wt0, wt1, hk, b, wr);
+
+  // start the pipeline (group jj holds unit jj; group 0 also the first zero-point rows)
 #pragma unroll
-    for (int s = 0; s < 8; ++s) {
+  for (int jj = 0; jj < NST - 1; ++jj) {
+    issue_unit(jj, jj * St::BYTES);
+    if (jj == 0 && n_my > 0) issue_zero_rows(0);
+    cp_async_commit();
+  }
+
+  uint32_t qe[16];  // q as fp16 B operand, pre-scaled by 2^-e(s), the weight the code's slot carries
 #pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        float lo = bf16_to_f(raw[2 * s + j] & 0xffff), hi = bf16_to_f(raw[2 * s + j] >> 16);
-        if (warp == 0) q_sm[((s >> 1) * 32 + lane) * 4 + (s & 1) * 2 + j] = pack_half2(lo, hi);
-        const float sc = 1.0f / (float)(1 << Slots<BK>::e(s));
-        qe[2 * s + j] = pack_half2(lo * sc, hi * sc);
-      }
+  for (int s = 0; s < 8; ++s) {
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      float lo = bf16_to_f(raw[2 * s + j] & 0xffff), hi = bf16_to_f(raw[2 * s + j] >> 16);
+      if (warp == 0) q_sm[((s >> 1) * 32 + lane) * 4 + (s & 1) * 2 + j] = pack_half2(lo, hi);
+      const float sc = 1.0f / (float)(1 << Slots<BK>::e(s));
+      qe[2 * s + j] = pack_half2(lo * sc, hi * sc);
     }
   }
-  // this split's share of the window, while the copies fly
-  {
-    const int t0 = (int)(((long long)split * p.r) / ns), t1 = (int)(((long long)(split + 1) * p.r) / ns);
-    window_tokens(p, t0, t1, hk, b, ws);
-  }
+  window_tokens(p, wt0, wt1, hk, b, ws, wr);  // while the copies fly
   __syncthreads();
 
   const float scale2 = p.scale * 1.4426950408889634f;
@@ -574,8 +613,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
 
   // One iteration: bias table every ZROWS units, refill of the stage unit j - 1 used, softmax reference,
   // numerators of unit j, then (MORE) logits of unit j + 1 next to the value product of unit j.
-  auto step = [&](int j, auto more_tag) {
-    constexpr bool MORE = decltype(more_tag)::value;
+  // off_prev / off_cur / off_next: ring offsets of the stages of units j - 1 (free, refilled), j and j + 1.
+  auto step = [&](int j, bool more, uint32_t off_prev, uint32_t off_cur, uint32_t off_next) {
     const int jr = j & (ZROWS - 1);
     if (jr == 0) {
       // bias table of units [j, j + 16): ztab[row][head] = scale * sum_d q_d z_d (log2 units)
@@ -599,7 +638,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     }
 
     __syncwarp();  // every lane is done with the stage of unit j - 1
-    if (j + NST - 1 < n_my) issue_unit(j + NST - 1);
+    issue_unit(j + NST - 1, off_prev);
     cp_async_commit();
 
     // ---- softmax reference: raise it only when a logit of unit j exceeds it by more than TAU ----
@@ -625,11 +664,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
       }
     }
 
-    if (MORE) {
-      cp_async_wait<NST - 2>();  // unit j + 1 has landed
-      __syncwarp();
-    }
-    const uint32_t st = my + (j & (NST - 1)) * St::BYTES;
+    cp_async_wait<NST - 2>();  // unit j + 1 has landed
+    __syncwarp();
 
     // ---- softmax numerators of unit j (log2 domain; the unit's key bias is common to its 32 tokens) ----
     const float t0 = bz.x - m0, t1 = bz.y - m1;
@@ -641,12 +677,21 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
       pb[mt][0] = movmatrix_trans(pack_half2(p0, p1));
       pb[mt][1] = movmatrix_trans(pack_half2(p2, p3));
     }
-    if (MORE) unit_logits<BK, BV, GS>(my + ((j + 1) & (NST - 1)) * St::BYTES, qe, accS, lane, tig);
-    unit_values<BK, BV, GS>(st, pb, accO, accZ, lane, gid, tig);
+    if (more) unit_logits<BK, BV, GS>(my + off_next, qe, accS, lane, tig);
+    unit_values<BK, BV, GS>(my + off_cur, pb, accO, accZ, lane, gid, tig);
   };
 
-  for (int j = 0; j + 1 < n_my; ++j) step(j, std::true_type{});
-  if (n_my > 0) step(n_my - 1, std::false_type{});
+  // main loop, unrolled over the ring so that every stage address is a constant offset
+  static_assert(NST == 4, "the loop below is unrolled for a ring of four stages");
+  int j = 0;
+  for (; j + NST < n_my; j += NST) {
+    step(j + 0, true, 3 * St::BYTES, 0 * St::BYTES, 1 * St::BYTES);
+    step(j + 1, true, 0 * St::BYTES, 1 * St::BYTES, 2 * St::BYTES);
+    step(j + 2, true, 1 * St::BYTES, 2 * St::BYTES, 3 * St::BYTES);
+    step(j + 3, true, 2 * St::BYTES, 3 * St::BYTES, 0 * St::BYTES);
+  }
+  for (; j < n_my; ++j)  // the last one to four units; the very last has no successor
+    step(j, j + 1 < n_my, ((j + 3) & 3) * St::BYTES, (j & 3) * St::BYTES, ((j + 1) & 3) * St::BYTES);
   cp_async_wait<0>();
   __syncthreads();  // all warps are done with their stages: the memory becomes the merge buffer
 
