@@ -46,15 +46,13 @@ namespace xq {
 namespace {
 
 constexpr int UT = 128;  // threads = tensor-memory lanes = tokens per batch = channels
-constexpr int UW = 4;        // compute warps
-constexpr int UT_ALL = 160;  // plus the warp that issues the MMAs
+constexpr int UW = 4;
 constexpr int HD = 128;
 constexpr int BT = 128;    // tokens per batch
-constexpr int NSTB = 4;    // staged batches
+constexpr int NSTB = 6;    // staged batches
 constexpr float TAU = 4.0f;
 constexpr int WAIT_LIMIT = 1 << 22;
-// tensor memory columns: one A buffer (keys and values take turns), S, O
-constexpr uint32_t TM_COLS = 128, COL_AK = 0, COL_AV = 0, COL_S = 64, COL_O = 96;
+constexpr uint32_t TM_COLS = 256, COL_AK = 0, COL_AV = 64, COL_S = 128, COL_O = 160;
 
 // ---------------------------------------------------------------------------
 // small PTX wrappers
@@ -119,33 +117,11 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
-
-// Bounded wait that also gives up when another thread of the CTA has (dead flag in shared memory).
-__device__ __forceinline__ bool mbar_wait_or_dead(uint32_t bar, uint32_t parity, volatile int* dead) {
-  for (int i = 0; i < WAIT_LIMIT; ++i) {
+// Bounded wait; false if the phase did not complete within WAIT_LIMIT polls.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (int i = 0; i < WAIT_LIMIT; ++i)
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 63) == 63 && *dead) return false;
-  }
   return false;
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
-}
-// barriers of the 128 compute threads (hardware barrier 1; barrier 0 is __syncthreads of all 160)
-__device__ __forceinline__ void bar_sync_compute() { asm volatile("bar.sync 1, 128;\n" ::: "memory"); }
-__device__ __forceinline__ bool bar_or_compute(bool v) {
-  uint32_t r;
-  asm volatile(
-      "{\n"
-      ".reg .pred p, q;\n"
-      "setp.ne.b32 p, %1, 0;\n"
-      "bar.red.or.pred q, 1, 128, p;\n"
-      "selp.u32 %0, 1, 0, q;\n"
-      "}\n"
-      : "=r"(r)
-      : "r"((int)v)
-      : "memory");
-  return r != 0;
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
@@ -478,7 +454,7 @@ __device__ __forceinline__ void ticket_merge(const DecodeParams& p, int ns, int 
   __syncthreads();
   if (!*s_flag) return;
   __threadfence();
-  for (int a = warp; a < dm.G && warp < UW; a += UW) {
+  for (int a = warp; a < dm.G; a += UW) {
     const size_t hq = (size_t)b * dm.Hq + hk * dm.G + a;
     const float* ml = p.part_ml + hq * ns * 2;
     const float* pa = p.part_acc + hq * ns * HD + lane * 4;
@@ -513,8 +489,7 @@ __device__ __forceinline__ void ticket_merge(const DecodeParams& p, int ns, int 
 // shared memory plan (dynamic):
 //   [NSTB stages]  (the merge buffer aliases the start after the loop)
 //   [B_K: N_S x 128 fp16, K-major] [B_P: 128 x N_O fp16, N-major; B_Q of the bias MMAs aliases it]
-//   [bias: 128 groups x 8 fp32] [reduction scratch: 4 warps x 32 fp32]
-// The CTA that handles the 16-bit window stages nothing and keeps its warps' states where the stages would be.
+//   [bias: 128 groups x 8 fp32] [reduction scratch: 4 warps x 32 fp32] [window states]
 // ---------------------------------------------------------------------------
 template <int BK, int BV, int GS, int GP>
 struct Plan {
@@ -529,463 +504,455 @@ struct Plan {
   static constexpr int BIAS_BYTES = 128 * 8 * 4;
   static constexpr int OFF_RED = OFF_BIAS + BIAS_BYTES;
   static constexpr int RED_BYTES = UW * 32 * 4;
-  static constexpr int TOTAL = OFF_RED + RED_BYTES;
+  static constexpr int OFF_WS = OFF_RED + RED_BYTES;
   static constexpr int MERGE_BYTES = 8 * MS * 4;
   static_assert(OFF_BK >= MERGE_BYTES, "the merge buffer aliases the stages");
-  static_assert(OFF_BK >= UW * 8 * MS * 4, "the window states of the window CTA alias the stages");
 };
+__host__ __device__ inline int wstate_bytes(int G) { return UW * G * MS * 4; }
 
 // ---------------------------------------------------------------------------
-// the kernel: warps 0..3 compute (thread = tensor-memory lane), warp 4 issues the MMAs
+// the kernel
 // ---------------------------------------------------------------------------
 template <int BK, int BV, int GS, int GP>
-__global__ void __launch_bounds__(UT_ALL, 3) decode_umma_kernel(DecodeParams p) {
+__global__ void __launch_bounds__(UT, 2) decode_umma_kernel(DecodeParams p) {
   using St = Stage<BK, BV, GS>;
   using Pl = Plan<BK, BV, GS, GP>;
   constexpr int NG = St::NG, NGRP = St::NGRP, N_S = Pl::N_S, N_O = Pl::N_O;
   constexpr int WPG = GS / 32;                  // warps whose tokens share a key group
   constexpr int NITEM = (GP * 16) / (32 * WPG); // (head, 8-channel chunk) rows of B_K per lane
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ __align__(8) unsigned long long bar_mem[4];
+  __shared__ __align__(8) unsigned long long bar_mem[2];
   __shared__ uint32_t tmem_base_sm;
   __shared__ int s_flag;
-  __shared__ volatile int dead_sm;
   float* mb = reinterpret_cast<float*>(smem);
   float* bias_sm = reinterpret_cast<float*>(smem + Pl::OFF_BIAS);
   float* red = reinterpret_cast<float*>(smem + Pl::OFF_RED);
-  float* ws = reinterpret_cast<float*>(smem);  // window CTA only
+  float* ws = reinterpret_cast<float*>(smem + Pl::OFF_WS);
 
   const Dims& dm = p.dm;
   const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = dm.G;
 
-  // Window CTAs: every split of a layer with nothing quantized yet, or the one extra CTA (split == ns_q) that takes
-  // the whole 16-bit window of a quantized layer.  Their partial joins the others' in the ticket merge.
-  if (p.ns_q == 0 || split == p.ns_q) {
-    const int ns = p.ns_q + p.ns_w;
-    int t0 = 0, t1 = p.r;
-    if (p.ns_q == 0) {
-      const int tiles = (p.r + 15) / 16;
-      t0 = (int)(((long long)split * tiles) / ns) * 16;
-      t1 = min((int)(((long long)(split + 1) * tiles) / ns) * 16, p.r);
-    }
-    if (warp < UW) {
-      WindowRegs wr;
-      window_preload(p, t0, t1, hk, b, wr);
-      window_tokens(p, t0, t1, hk, b, ws, wr);
-    }
+  if (p.ns_q == 0) {  // nothing is quantized yet: window-only splits
+    const int ns = p.ns_w;
+    const int tiles = (p.r + 15) / 16;
+    const int t0 = (int)(((long long)split * tiles) / ns) * 16;
+    const int t1 = min((int)(((long long)(split + 1) * tiles) / ns) * 16, p.r);
+    WindowRegs wr;
+    window_preload(p, t0, t1, hk, b, wr);
+    window_tokens(p, t0, t1, hk, b, ws, wr);
     __syncthreads();
-    if (warp < UW) write_partial(p, nullptr, ws, split, ns, hk, b);
+    write_partial(p, nullptr, ws, split, ns, hk, b);
     ticket_merge(p, ns, hk, b, &s_flag);
     return;
   }
 
-  const int ns = p.ns_q;           // splits of the packed region; the partials number ns + 1 (window CTA)
+  const int ns = p.ns_q;
   const int nb_total = (p.n_q + BT - 1) / BT;
   const int b0 = (int)(((long long)split * nb_total) / ns);
   const int nb = (int)(((long long)(split + 1) * nb_total) / ns) - b0;  // this CTA's batches: [b0, b0 + nb), 1 <= nb <= GS
   const int bh = b * dm.Hkv + hk;
 
-  const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(smem);
-  const uint32_t barKR = (uint32_t)__cvta_generic_to_shared(&bar_mem[0]);  // A (keys) and B_K written: 128 arrivals
-  const uint32_t barVR = (uint32_t)__cvta_generic_to_shared(&bar_mem[1]);  // A (values) and B_P written: 128 arrivals
-  const uint32_t barS = (uint32_t)__cvta_generic_to_shared(&bar_mem[2]);   // key MMAs complete
-  const uint32_t barO = (uint32_t)__cvta_generic_to_shared(&bar_mem[3]);   // value MMAs complete
-  constexpr uint32_t idescS = idesc_f16(N_S, 0), idescO = idesc_f16(N_O, 1), idescB = idesc_f16(16, 0);
-  constexpr uint32_t LBO_K = (N_S / 8) * 128, LBO_P = (N_O / 8) * 128;
+  // the four streams at this CTA's first batch
+  const uint8_t* gk = reinterpret_cast<const uint8_t*>(p.L.k_codes) + (size_t)bh * ((size_t)dm.nq_cap * (HD * BK / 8)) +
+                      (size_t)b0 * St::KC;
+  const uint8_t* gv = reinterpret_cast<const uint8_t*>(p.L.v_codes) + (size_t)bh * ((size_t)dm.nq_cap * (HD * BV / 8)) +
+                      (size_t)b0 * St::VC;
+  const uint8_t* gvm = reinterpret_cast<const uint8_t*>(p.L.v_meta) + (size_t)bh * ((size_t)dm.nq_cap * 4 * NG) +
+                       (size_t)b0 * St::VM;
+  const size_t plane = (size_t)(dm.nq_cap / GS) * 256;  // bytes of the key scale plane (= of the zero-point plane)
+  const uint8_t* gks = reinterpret_cast<const uint8_t*>(p.L.k_meta) + (size_t)bh * 2 * plane + (size_t)b0 * St::KS;
+  const uint8_t* gkz = gks + plane;
 
-  // ---- set-up: barriers, tensor memory (allocated and freed by the MMA warp), zeroed B operands ----
+  const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(smem);
+  const uint32_t barS = (uint32_t)__cvta_generic_to_shared(&bar_mem[0]);
+  const uint32_t barO = (uint32_t)__cvta_generic_to_shared(&bar_mem[1]);
+
+  // ---- loads the prologue waits for go out first ----
+  const int wt0 = (int)(((long long)split * p.r) / ns), wt1 = (int)(((long long)(split + 1) * p.r) / ns);
+  WindowRegs wr;
+  window_preload(p, wt0, wt1, hk, b, wr);
+
+  // stage batch jj of this CTA into ring slot `slot`, if it exists (no commit, no branch)
+  auto issue_batch = [&](int jj, int slot) {
+    const bool on = jj < nb;
+    const uint32_t s = sm_base + slot * St::BYTES + tid * 16;
+    const uint8_t* k = gk + (size_t)(uint32_t)jj * St::KC + tid * 16;
+#pragma unroll
+    for (int i = 0; i < St::KC / 2048; ++i) cp_async16_if(s + i * 2048, k + i * 2048, on);
+    cp_async16_if(s + St::OFF_KS, gks + (size_t)(uint32_t)jj * St::KS + tid * 16, on && tid * 16 < St::KS);
+    const uint8_t* v = gv + (size_t)(uint32_t)jj * St::VC + tid * 16;
+#pragma unroll
+    for (int i = 0; i < St::VC / 2048; ++i) cp_async16_if(s + St::OFF_VC + i * 2048, v + i * 2048, on);
+    cp_async16_if(s + St::OFF_VM, gvm + (size_t)(uint32_t)jj * St::VM + tid * 16, on && tid * 16 < St::VM);
+  };
+#pragma unroll
+  for (int jj = 0; jj < NSTB - 1; ++jj) {
+    issue_batch(jj, jj);
+    cp_async_commit();
+  }
+
+  // ---- set-up: barriers, tensor memory, zeroed B operands ----
   if (tid == 0) {
-    mbar_init(barKR, UT);
-    mbar_init(barVR, UT);
     mbar_init(barS, 1);
     mbar_init(barO, 1);
-    dead_sm = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
-  if (warp == UW) {
+  if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(
                      (uint32_t)__cvta_generic_to_shared(&tmem_base_sm)),
                  "r"(TM_COLS)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
-  for (int i = tid; i < (Pl::BK_BYTES + Pl::BP_BYTES) / 16; i += UT_ALL) sts128(sm_base + Pl::OFF_BK + i * 16, 0u, 0u, 0u, 0u);
+  for (int i = tid; i < (Pl::BK_BYTES + Pl::BP_BYTES) / 16; i += UT) sts128(sm_base + Pl::OFF_BK + i * 16, 0u, 0u, 0u, 0u);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tbase = tmem_base_sm;
+  const uint32_t lane_base = tbase + ((uint32_t)(warp * 32) << 16);
+  uint32_t phS = 0, phO = 0;  // parities of the next completions of barS / barO
+  bool dead = false;          // a bounded wait gave up
 
-  if (warp == UW) {
-    // ================= MMA warp: one thread issues, in the order the operands become ready =================
-    if (lane == 0) {
-      bool ok = mbar_wait_or_dead(barKR, 0, &dead_sm);  // zero-point rows and q: the bias MMAs
-      if (ok) {
-        tc_fence_after();
-        const uint64_t dq = smem_desc(sm_base + Pl::OFF_BP, 256, 128);
+  // ---- q: B operand of the bias MMAs (unscaled, rows = heads) and this lane's pre-weighted chunks for B_K ----
+  // B_Q[n][k] K-major, N = 16: byte offset (k/8)*256 + (n/8)*128 + (n%8)*16 + (k%8)*2
+  {
+    const int h = tid >> 4, ck = tid & 15;  // 8 heads x 16 chunks of 8 channels
+    if (h < G) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(p.q + ((size_t)b * dm.Hq + hk * G + h) * HD + ck * 8);
+      const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+      uint32_t o[4];
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) umma_ts(tbase + COL_S, tbase + COL_AK + 8 * ks, dq + (uint64_t)(ks * 512 / 16), idescB, ks > 0);
-        umma_commit(barS);
-      }
-      const uint64_t dk = smem_desc(sm_base + Pl::OFF_BK, LBO_K, 128), dp = smem_desc(sm_base + Pl::OFF_BP, LBO_P, 128);
-      uint32_t phK = 1, phV = 0;
-      for (int i = 0; i < nb && ok; ++i) {
-        ok = mbar_wait_or_dead(barKR, phK, &dead_sm);  // keys of batch i
-        phK ^= 1;
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma_ts(tbase + COL_S, tbase + COL_AK + 8 * ks, dk + (uint64_t)(ks * 2 * LBO_K / 16), idescS, ks > 0);
-        umma_commit(barS);
-        ok = mbar_wait_or_dead(barVR, phV, &dead_sm);  // values of batch i
-        phV ^= 1;
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma_ts(tbase + COL_O, tbase + COL_AV + 8 * ks, dp + (uint64_t)(ks * 2 * LBO_P / 16), idescO, (i > 0 || ks > 0) ? 1u : 0u);
-        umma_commit(barO);
-      }
-      if (!ok) dead_sm = 1;
+      for (int i = 0; i < 4; ++i) o[i] = pack_half2(bf16_to_f(rw[i] & 0xffff), bf16_to_f(rw[i] >> 16));
+      sts128(sm_base + Pl::OFF_BP + ck * 256 + (h >> 3) * 128 + (h & 7) * 16, o[0], o[1], o[2], o[3]);
     }
-    __syncwarp();
-  } else {
-    // ================= compute warps =================
-    // the four streams at this CTA's first batch
-    const uint8_t* gk = reinterpret_cast<const uint8_t*>(p.L.k_codes) + (size_t)bh * ((size_t)dm.nq_cap * (HD * BK / 8)) +
-                        (size_t)b0 * St::KC;
-    const uint8_t* gv = reinterpret_cast<const uint8_t*>(p.L.v_codes) + (size_t)bh * ((size_t)dm.nq_cap * (HD * BV / 8)) +
-                        (size_t)b0 * St::VC;
-    const uint8_t* gvm = reinterpret_cast<const uint8_t*>(p.L.v_meta) + (size_t)bh * ((size_t)dm.nq_cap * 4 * NG) +
-                         (size_t)b0 * St::VM;
-    const size_t plane = (size_t)(dm.nq_cap / GS) * 256;  // bytes of the key scale plane (= of the zero-point plane)
-    const uint8_t* gks = reinterpret_cast<const uint8_t*>(p.L.k_meta) + (size_t)bh * 2 * plane + (size_t)b0 * St::KS;
-    const uint8_t* gkz = gks + plane;
-
-    // stage batch jj of this CTA into ring slot `slot`, if it exists (no commit, no branch)
-    auto issue_batch = [&](int jj, int slot) {
-      const bool on = jj < nb;
-      const uint32_t s = sm_base + slot * St::BYTES + tid * 16;
-      const uint8_t* k = gk + (size_t)(uint32_t)jj * St::KC + tid * 16;
+  }
+  const int my_gl = (warp * 32) / GS;  // token group (within the batch) of this warp's tokens
+  uint32_t qk[NITEM][4];               // q chunks of this lane's B_K rows, times 2^-weight of each channel's slot
+  int item_h[NITEM], item_ck[NITEM];
 #pragma unroll
-      for (int i = 0; i < St::KC / 2048; ++i) cp_async16_if(s + i * 2048, k + i * 2048, on);
-      cp_async16_if(s + St::OFF_KS, gks + (size_t)(uint32_t)jj * St::KS + tid * 16, on && tid * 16 < St::KS);
-      const uint8_t* v = gv + (size_t)(uint32_t)jj * St::VC + tid * 16;
+  for (int it = 0; it < NITEM; ++it) {
+    const int item = (warp % WPG) * 32 + lane + it * 32 * WPG;
+    const int h = item >> 4, ck = item & 15;
+    item_h[it] = h;
+    item_ck[it] = ck;
+    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+    if (h < G) raw = *reinterpret_cast<const uint4*>(p.q + ((size_t)b * dm.Hq + hk * G + h) * HD + ck * 8);
+    const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-      for (int i = 0; i < St::VC / 2048; ++i) cp_async16_if(s + St::OFF_VC + i * 2048, v + i * 2048, on);
-      cp_async16_if(s + St::OFF_VM, gvm + (size_t)(uint32_t)jj * St::VM + tid * 16, on && tid * 16 < St::VM);
-    };
-#pragma unroll
-    for (int jj = 0; jj < NSTB - 1; ++jj) {
-      issue_batch(jj, jj);
-      cp_async_commit();
+    for (int i = 0; i < 4; ++i) {
+      const int e = (BK == 2) ? ((((ck & 1) * 4 + i) < 5) ? 2 * ((ck & 1) * 4 + i) : 2 * ((ck & 1) * 4 + i - 5))
+                              : ((((ck & 3) * 4 + i)) % 8);
+      // channels 8 ck + 2 i, 8 ck + 2 i + 1 share a slot
+      const float sc = __int_as_float((127 - e) << 23);
+      qk[it][i] = pack_half2(bf16_to_f(rw[i] & 0xffff) * sc, bf16_to_f(rw[i] >> 16) * sc);
     }
+  }
 
-    const uint32_t lane_base = tbase + ((uint32_t)(warp * 32) << 16);
-    uint32_t phS = 0, phO = 0;  // parities of the next completions of barS / barO
-    bool dead = false;          // a bounded wait gave up
-
-    // ---- q: B operand of the bias MMAs (unscaled, rows = heads) and this lane's pre-weighted chunks for B_K ----
-    // B_Q[n][k] K-major, N = 16: byte offset (k/8)*256 + (n/8)*128 + (n%8)*16 + (k%8)*2
-    {
-      const int h = tid >> 4, ck = tid & 15;  // 8 heads x 16 chunks of 8 channels
-      if (h < G) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(p.q + ((size_t)b * dm.Hq + hk * G + h) * HD + ck * 8);
-        const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
-        uint32_t o[4];
+  // ---- bias of every key token group of this CTA's range: bias_sm[group][head] = scale2 * sum_d q_d z_d ----
+  const float scale2 = p.scale * 1.4426950408889634f;
+  const int n_grp = nb * NGRP;  // <= 128
+  {
+    // thread = group row: its 128 zero-points are already fp16 pairs in channel order = one A row
+    const int gr = min(tid, n_grp - 1);
+    const uint4* zrow = reinterpret_cast<const uint4*>(gkz + (size_t)gr * 256);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) o[i] = pack_half2(bf16_to_f(rw[i] & 0xffff), bf16_to_f(rw[i] >> 16));
-        sts128(sm_base + Pl::OFF_BP + ck * 256 + (h >> 3) * 128 + (h & 7) * 16, o[0], o[1], o[2], o[3]);
-      }
+    for (int q = 0; q < 4; ++q) {
+      uint4 z[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) z[i] = zrow[4 * q + i];
+      const uint32_t r[16] = {z[0].x, z[0].y, z[0].z, z[0].w, z[1].x, z[1].y, z[1].z, z[1].w,
+                              z[2].x, z[2].y, z[2].z, z[2].w, z[3].x, z[3].y, z[3].z, z[3].w};
+      tmem_st16(lane_base + COL_AK + 16 * q, r);
     }
-    const int my_gl = (warp * 32) / GS;  // token group (within the batch) of this warp's tokens
-    uint32_t qk[NITEM][4];               // q chunks of this lane's B_K rows, times 2^-weight of each channel's slot
+    tc_wait_st();
+    proxy_fence();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+      constexpr uint32_t idesc = idesc_f16(16, 0);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        umma_ts(tbase + COL_S, tbase + COL_AK + 8 * ks, smem_desc(sm_base + Pl::OFF_BP + ks * 512, 256, 128), idesc, ks > 0);
+      umma_commit(barS);
+    }
+  }
+  // the window share, while the bias MMAs and the first copies fly
+  window_tokens(p, wt0, wt1, hk, b, ws, wr);
+  dead = __syncthreads_or(!mbar_wait(barS, phS));
+  phS ^= 1;
+  if (!dead) {
+    tc_fence_after();
+    float bz[8];
+    tmem_ld4(lane_base + COL_S, bz);
+    tmem_ld4(lane_base + COL_S + 4, bz + 4);
+    tc_wait_ld();
+#pragma unroll
+    for (int h = 0; h < 8; ++h) bias_sm[tid * 8 + h] = bz[h] * scale2;
+    // B_Q is dead: clear its place for B_P (padding columns must read as zero)
+    for (int i = tid; i < Pl::BP_BYTES / 16; i += UT) sts128(sm_base + Pl::OFF_BP + i * 16, 0u, 0u, 0u, 0u);
+  }
+
+  const float c1 = scale2 * 16777216.0f;  // undoes the 2^-24 of the subnormal code operand
+  float m[GP], L[GP], zacc[NG][GP];
+#pragma unroll
+  for (int h = 0; h < GP; ++h) {
+    m[h] = -CUDART_INF_F;
+    L[h] = 0.f;
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) zacc[gi][h] = 0.f;
+  }
+  const float vw = __int_as_float((127 - v_weight_log2<BV>(lane)) << 23);  // 2^-weight of this lane's token slot (values)
+  constexpr uint32_t idescS = idesc_f16(N_S, 0), idescO = idesc_f16(N_O, 1);
+  constexpr uint32_t LBO_K = (N_S / 8) * 128, LBO_P = (N_O / 8) * 128;
+
+  // B_K rows of this warp's group for the batch staged at `st`
+  auto build_bk = [&](uint32_t st) {
 #pragma unroll
     for (int it = 0; it < NITEM; ++it) {
-      const int item = (warp % WPG) * 32 + lane + it * 32 * WPG;
-      const int h = item >> 4, ck = item & 15;
-      uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-      if (h < G) raw = *reinterpret_cast<const uint4*>(p.q + ((size_t)b * dm.Hq + hk * G + h) * HD + ck * 8);
-      const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        // channels 8 ck + 2 i and 8 ck + 2 i + 1 share a slot
-        const int e = (BK == 2) ? ((((ck & 1) * 4 + i) < 5) ? 2 * ((ck & 1) * 4 + i) : 2 * ((ck & 1) * 4 + i - 5))
-                                : ((((ck & 3) * 4 + i)) % 8);
-        const float sc = __int_as_float((127 - e) << 23);
-        qk[it][i] = pack_half2(bf16_to_f(rw[i] & 0xffff) * sc, bf16_to_f(rw[i] >> 16) * sc);
+      const int h = item_h[it], ck = item_ck[it];
+      if (h < G) {
+        const uint4 sv = lds128(st + St::OFF_KS + my_gl * 256 + ck * 16);
+        const int n = my_gl * GP + h;
+        sts128(sm_base + Pl::OFF_BK + ck * LBO_K + (n >> 3) * 128 + (n & 7) * 16, hmul2_u(qk[it][0], sv.x),
+               hmul2_u(qk[it][1], sv.y), hmul2_u(qk[it][2], sv.z), hmul2_u(qk[it][3], sv.w));
       }
     }
-
-    // ---- bias of every key token group of this CTA's range: bias_sm[group][head] = scale2 * sum_d q_d z_d ----
-    const float scale2 = p.scale * 1.4426950408889634f;
-    const int n_grp = nb * NGRP;  // <= 128
-    {
-      // thread = group row: its 128 zero-points are already fp16 pairs in channel order = one A row
-      const int gr = min(tid, n_grp - 1);
-      const uint4* zrow = reinterpret_cast<const uint4*>(gkz + (size_t)gr * 256);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint4 z[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) z[i] = zrow[4 * q + i];
-        const uint32_t r[16] = {z[0].x, z[0].y, z[0].z, z[0].w, z[1].x, z[1].y, z[1].z, z[1].w,
-                                z[2].x, z[2].y, z[2].z, z[2].w, z[3].x, z[3].y, z[3].z, z[3].w};
-        tmem_st16(lane_base + COL_AK + 16 * q, r);
-      }
-      tc_wait_st();
-      proxy_fence();
-      tc_fence_before();
-      mbar_arrive(barKR);
-    }
-    if (!mbar_wait_or_dead(barS, phS, &dead_sm)) dead_sm = 1;  // found by the first vote of the loop
-    phS ^= 1;
+  };
+  auto issue_key_mmas = [&]() {  // one thread
     tc_fence_after();
-    {
-      float bz[8];
-      tmem_ld4(lane_base + COL_S, bz);
-      tmem_ld4(lane_base + COL_S + 4, bz + 4);
-      tc_wait_ld();
 #pragma unroll
-      for (int h = 0; h < 8; ++h) bias_sm[tid * 8 + h] = bz[h] * scale2;
-      // B_Q is dead: clear its place for B_P (padding columns must read as zero)
-      for (int i = tid; i < Pl::BP_BYTES / 16; i += UT) sts128(sm_base + Pl::OFF_BP + i * 16, 0u, 0u, 0u, 0u);
-    }
+    for (int ks = 0; ks < 8; ++ks)
+      umma_ts(tbase + COL_S, tbase + COL_AK + 8 * ks, smem_desc(sm_base + Pl::OFF_BK + ks * 2 * LBO_K, LBO_K, 128), idescS,
+              ks > 0);
+    umma_commit(barS);
+  };
 
-    const float c1 = scale2 * 16777216.0f;  // undoes the 2^-24 of the subnormal code operand
-    float m[GP], L[GP], zacc[NG][GP];
-#pragma unroll
-    for (int h = 0; h < GP; ++h) {
-      m[h] = -CUDART_INF_F;
-      L[h] = 0.f;
-#pragma unroll
-      for (int gi = 0; gi < NG; ++gi) zacc[gi][h] = 0.f;
-    }
-    const float vw = __int_as_float((127 - v_weight_log2<BV>(lane)) << 23);  // 2^-weight of this lane's token slot (values)
-
-    // B_K rows of this warp's group for the batch staged at `st`
-    auto build_bk = [&](uint32_t st) {
-#pragma unroll
-      for (int it = 0; it < NITEM; ++it) {
-        const int item = (warp % WPG) * 32 + lane + it * 32 * WPG;
-        const int h = item >> 4, ck = item & 15;
-        if (h < G) {
-          const uint4 sv = lds128(st + St::OFF_KS + my_gl * 256 + ck * 16);
-          const int n = my_gl * GP + h;
-          sts128(sm_base + Pl::OFF_BK + ck * LBO_K + (n >> 3) * 128 + (n & 7) * 16, hmul2_u(qk[it][0], sv.x),
-                 hmul2_u(qk[it][1], sv.y), hmul2_u(qk[it][2], sv.z), hmul2_u(qk[it][3], sv.w));
-        }
-      }
-    };
-
-    // ---- first batch: keys expanded, their MMAs requested ----
-    cp_async_wait<NSTB - 2>();  // batch 0 has landed (for this thread)
-    bar_sync_compute();          // ... for every thread; bias table and cleared B_P visible
+  // ---- first batch: keys expanded and their MMAs issued ----
+  cp_async_wait<NSTB - 3>();  // batches 0 and 1 have landed (for this thread)
+  __syncthreads();
+  if (!dead) {
     expand_keys<BK>(sm_base + warp * St::KU, lane, lane_base + COL_AK);
     build_bk(sm_base);
     tc_wait_st();
     proxy_fence();
     tc_fence_before();
-    mbar_arrive(barKR);
+  }
+  __syncthreads();
+  if (tid == 0 && !dead) issue_key_mmas();
 
-    int slot = 0;  // ring slot of batch i
-    for (int i = 0; i < nb && !dead; ++i) {
-      const uint32_t st = sm_base + slot * St::BYTES;
-      const int slot_next = (slot + 1 == NSTB) ? 0 : slot + 1;
-      const int slot_prev = (slot == 0) ? NSTB - 1 : slot - 1;
-      const int tok = (b0 + i) * BT + tid;  // this thread's token (keys, softmax)
-      const bool valid = tok < p.n_q;
-      const int gidx = i * NGRP + my_gl;     // its key group within this CTA's range
+  int slot = 0;  // ring slot of batch i
+  for (int i = 0; i < nb && !dead; ++i) {
+    const uint32_t st = sm_base + slot * St::BYTES;
+    const int slot_next = (slot + 1 == NSTB) ? 0 : slot + 1;
+    const int slot_prev = (slot == 0) ? NSTB - 1 : slot - 1;
+    const int tok = (b0 + i) * BT + tid;  // this thread's token (keys, softmax)
+    const bool valid = tok < p.n_q;
+    const int gidx = i * NGRP + my_gl;     // its key group within this CTA's range
 
-      // 1. logits of batch i; the A buffer is free again
-      if (!mbar_wait_or_dead(barS, phS, &dead_sm)) dead_sm = 1;
-      phS ^= 1;
-      tc_fence_after();
-      float x[GP];
-      tmem_ld_row<GP>(lane_base + COL_S + my_gl * GP, x);
-      tc_wait_ld();
-      bool raise = false;
+    // 1. logits of batch i
+    bool lost = !mbar_wait(barS, phS);
+    phS ^= 1;
+    tc_fence_after();
+    float x[GP];
+    tmem_ld_row<GP>(lane_base + COL_S + my_gl * GP, x);
+    tc_wait_ld();
+    bool raise = false;
 #pragma unroll
-      for (int h = 0; h < GP; ++h) {
-        x[h] = (valid && h < G) ? fmaf(x[h], c1, bias_sm[gidx * 8 + h]) : -CUDART_INF_F;
-        raise |= x[h] > m[h] + TAU;
-      }
-      // 2. barrier of the compute warps: does any token want the softmax reference raised (or has a wait given up)?
-      const bool gave_up = dead_sm != 0;
-      bool any_raise = bar_or_compute(raise || gave_up);
-      if (any_raise && bar_or_compute(gave_up)) {  // second vote only on the rare path: everyone leaves together
-        dead = true;
-        break;
-      }
-      // every compute thread is done with batch i - 1: its slot is refilled
-      issue_batch(i + NSTB - 1, slot_prev);
-      cp_async_commit();
-      // 3. raise the softmax reference (rare): CTA-wide maximum per head, rescale O, L, the zero-point sums
-      if (any_raise) {
-        float xm[GP];
-#pragma unroll
-        for (int h = 0; h < GP; ++h) {
-          xm[h] = x[h];
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) xm[h] = fmaxf(xm[h], __shfl_xor_sync(0xffffffffu, xm[h], o));
-          if (lane == 0) red[warp * 32 + h] = xm[h];
-        }
-        bar_sync_compute();
-        float f[GP];
-#pragma unroll
-        for (int h = 0; h < GP; ++h) {
-          const float mn = fmaxf(fmaxf(m[h], fmaxf(red[h], red[32 + h])), fmaxf(red[64 + h], red[96 + h]));
-          f[h] = ex2(m[h] - mn);  // 0 on the first batch (m = -inf); padded heads: -inf - -inf = NaN, never used
-          m[h] = mn;
-          L[h] *= f[h];
-#pragma unroll
-          for (int gi = 0; gi < NG; ++gi) zacc[gi][h] *= f[h];
-        }
-        if (i > 0) {  // this thread's channel row of O (its MMAs are complete): the columns of its own channel group
-          const uint32_t oaddr = lane_base + COL_O + ((warp * 32) / GS) * GP;
-          float o[GP];
-          tmem_ld_row<GP>(oaddr, o);
-          tc_wait_ld();
-#pragma unroll
-          for (int h = 0; h < GP; ++h) o[h] *= f[h];
-          tmem_st_row<GP>(oaddr, o);
-        }
-        bar_sync_compute();  // `red` may be reused
-      }
-
-      // 4. numerators of batch i, P' rows, zero-point and normaliser sums; values of batch i into the A buffer
-      {
-        uint32_t sv[NG / 2], zv[NG / 2];  // this token's value scales and zero-points, fp16 pairs
-        if (NG == 4) {
-          uint4 mt = lds128(st + St::OFF_VM + tid * 16);
-          sv[0] = mt.x; sv[NG / 2 - 1] = mt.y; zv[0] = mt.z; zv[NG / 2 - 1] = mt.w;
-        } else {
-          uint2 mt = lds64(st + St::OFF_VM + tid * 8);
-          sv[0] = mt.x; zv[0] = mt.y;
-        }
-        if (!valid) {
-#pragma unroll
-          for (int i2 = 0; i2 < NG / 2; ++i2) sv[i2] = zv[i2] = 0u;
-        }
-        float pe[GP];
-#pragma unroll
-        for (int h = 0; h < GP; ++h) {
-          pe[h] = (valid && h < G) ? ex2(x[h] - m[h]) * vw : 0.f;  // carries 2^-weight of the token's value slot
-          L[h] += pe[h];
-        }
-#pragma unroll
-        for (int g2 = 0; g2 < NG / 2; ++g2) {
-          const float2 zf = half2_to_float2(zv[g2]);
-#pragma unroll
-          for (int h = 0; h < GP; ++h) {
-            zacc[2 * g2][h] = fmaf(pe[h], zf.x, zacc[2 * g2][h]);
-            zacc[2 * g2 + 1][h] = fmaf(pe[h], zf.y, zacc[2 * g2 + 1][h]);
-          }
-        }
-        uint32_t ph[GP / 2];
-#pragma unroll
-        for (int h = 0; h < GP / 2; ++h) ph[h] = pack_half2(pe[2 * h], pe[2 * h + 1]);
-        // row `tid` of B_P: columns gi * GP + h, 8 columns per 16-byte chunk
-        const uint32_t prow = sm_base + Pl::OFF_BP + (tid >> 3) * LBO_P + (tid & 7) * 16;
-#pragma unroll
-        for (int gi = 0; gi < NG; ++gi) {
-          const uint32_t sb = __byte_perm(sv[gi >> 1], 0u, (gi & 1) ? 0x3232 : 0x1010);  // (s, s)
-          if (GP == 4) {
-            if ((gi & 1) == 0) {
-              const uint32_t sb1 = __byte_perm(sv[gi >> 1], 0u, 0x3232);
-              sts128(prow + (gi >> 1) * 128, hmul2_u(ph[0], sb), hmul2_u(ph[1], sb), hmul2_u(ph[0], sb1), hmul2_u(ph[1], sb1));
-            }
-          } else {
-            sts128(prow + gi * 128, hmul2_u(ph[0], sb), hmul2_u(ph[1], sb), hmul2_u(ph[GP / 2 - 2], sb),
-                   hmul2_u(ph[GP / 2 - 1], sb));
-          }
-        }
-      }
-      expand_values<BV>(st + St::OFF_VC, tid, lane_base + COL_AV);
+    for (int h = 0; h < GP; ++h) {
+      x[h] = (valid && h < G) ? fmaf(x[h], c1, bias_sm[gidx * 8 + h]) : -CUDART_INF_F;
+      raise |= x[h] > m[h] + TAU;
+    }
+    // 2. keys of batch i + 1 (their stage became visible at the previous barrier)
+    if (i + 1 < nb) {
+      const uint32_t sn = sm_base + slot_next * St::BYTES;
+      expand_keys<BK>(sn + warp * St::KU, lane, lane_base + COL_AK);
+      build_bk(sn);
       tc_wait_st();
       proxy_fence();
-      tc_fence_before();
-      mbar_arrive(barVR);  // the MMA warp takes it from here
-      // 5. keys of batch i + 1: B_K while the value MMAs run, then A once they are done
-      const bool more = i + 1 < nb;
-      const uint32_t sn = sm_base + slot_next * St::BYTES;
-      cp_async_wait<NSTB - 2>();  // batch i + 1 has landed (for this thread)
-      bar_sync_compute();          // ... for every compute thread
-      if (more) build_bk(sn);
-      if (!mbar_wait_or_dead(barO, phO, &dead_sm)) dead_sm = 1;
-      phO ^= 1;
-      tc_fence_after();
-      if (more) {
-        expand_keys<BK>(sn + warp * St::KU, lane, lane_base + COL_AK);
-        tc_wait_st();
-        proxy_fence();
-        tc_fence_before();
-        mbar_arrive(barKR);
-      }
-      slot = slot_next;
-    }
-
-    // ---- epilogue of the compute warps ----
-    cp_async_wait<0>();
-    dead = bar_or_compute(dead || dead_sm != 0);
-    tc_fence_after();
-    if (!dead) {
-      // L and the zero-point sums were accumulated with the per-lane factor 2^-weight; undo it, then reduce
-      const float uw = __int_as_float((127 + v_weight_log2<BV>(lane)) << 23);
-      float* wsum = reinterpret_cast<float*>(smem + Pl::OFF_BK);  // [warp][64]; B_K is dead
-#pragma unroll
-      for (int r = 0; r <= NG; ++r) {
-#pragma unroll
-        for (int h = 0; h < GP; ++h) {
-          float v = ((r < NG) ? zacc[r < NG ? r : 0][h] : L[h]) * uw;
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-          if (lane == 0) wsum[warp * 64 + r * GP + h] = v;
-        }
-      }
-    }
-    bar_sync_compute();  // all stages are dead: the memory becomes the merge buffer
-    if (!dead) {
-      const float* wsum = reinterpret_cast<const float*>(smem + Pl::OFF_BK);
-      const int gi = (warp * 32) / GS;  // channel group of this thread's channel
-      float o[GP];
-      tmem_ld_row<GP>(lane_base + COL_O + gi * GP, o);
-      tc_wait_ld();
-#pragma unroll
-      for (int h = 0; h < GP; ++h) {
-        if (h < G) {
-          const float z = wsum[gi * GP + h] + wsum[64 + gi * GP + h] + wsum[128 + gi * GP + h] + wsum[192 + gi * GP + h];
-          mb[h * MS + tid] = fmaf(o[h], 16777216.0f, z);  // the code operands carried 2^-24
-          if (tid == 0) {
-            mb[h * MS + HD] = m[h];
-            mb[h * MS + HD + 1] = wsum[NG * GP + h] + wsum[64 + NG * GP + h] + wsum[128 + NG * GP + h] + wsum[192 + NG * GP + h];
-          }
-        }
-      }
-    } else {  // leave a neutral partial so that the merge stays finite; the status word tells the host
-      if (tid == 0) atomicExch(p.status, 1);
-      for (int a = 0; a < G; ++a) {
-        mb[a * MS + tid] = 0.f;
-        if (tid == 0) {
-          mb[a * MS + HD] = -CUDART_INF_F;
-          mb[a * MS + HD + 1] = 0.f;
-        }
-      }
     }
     tc_fence_before();
+    // 3. barrier: S has been read by everyone, A_K / B_K of batch i + 1 are complete
+    const int votes = __syncthreads_or((raise ? 1 : 0) | (lost ? 2 : 0));
+    if (votes & 2) {
+      dead = true;
+      break;
+    }
+    if (tid == 0 && i + 1 < nb) issue_key_mmas();
+    // the slot of batch i - 1 is free now: refill it
+    issue_batch(i + NSTB - 1, slot_prev);
+    cp_async_commit();
+
+    // the value MMAs of batch i - 1 must be done before A_V, B_P (and O, when rescaling) are touched
+    if (i > 0) {
+      lost = !mbar_wait(barO, phO);
+      phO ^= 1;
+      tc_fence_after();
+    }
+    // 4. raise the softmax reference (rare): CTA-wide maximum per head, rescale O, L, the zero-point sums
+    if (votes & 1) {
+      float xm[GP];
+#pragma unroll
+      for (int h = 0; h < GP; ++h) {
+        xm[h] = x[h];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) xm[h] = fmaxf(xm[h], __shfl_xor_sync(0xffffffffu, xm[h], o));
+        if (lane == 0) red[warp * 32 + h] = xm[h];
+      }
+      __syncthreads();
+      float f[GP];
+#pragma unroll
+      for (int h = 0; h < GP; ++h) {
+        const float mn = fmaxf(fmaxf(m[h], fmaxf(red[h], red[32 + h])), fmaxf(red[64 + h], red[96 + h]));
+        f[h] = ex2(m[h] - mn);  // 0 on the first batch (m = -inf); padded heads: -inf - -inf = NaN, never used
+        m[h] = mn;
+        L[h] *= f[h];
+#pragma unroll
+        for (int gi = 0; gi < NG; ++gi) zacc[gi][h] *= f[h];
+      }
+      if (i > 0) {  // this thread's channel row of O: the columns of its own channel group
+        const uint32_t oaddr = lane_base + COL_O + ((warp * 32) / GS) * GP;
+        float o[GP];
+        tmem_ld_row<GP>(oaddr, o);
+        tc_wait_ld();
+#pragma unroll
+        for (int h = 0; h < GP; ++h) o[h] *= f[h];
+        tmem_st_row<GP>(oaddr, o);
+      }
+      __syncthreads();  // `red` may be reused
+    }
+
+    // 5. numerators of batch i, P' rows, zero-point and normaliser sums; values of batch i
+    {
+      uint32_t sv[NG / 2], zv[NG / 2];  // this token's value scales and zero-points, fp16 pairs
+      if (NG == 4) {
+        uint4 mt = lds128(st + St::OFF_VM + tid * 16);
+        sv[0] = mt.x; sv[NG / 2 - 1] = mt.y; zv[0] = mt.z; zv[NG / 2 - 1] = mt.w;
+      } else {
+        uint2 mt = lds64(st + St::OFF_VM + tid * 8);
+        sv[0] = mt.x; zv[0] = mt.y;
+      }
+      if (!valid) {
+#pragma unroll
+        for (int i2 = 0; i2 < NG / 2; ++i2) sv[i2] = zv[i2] = 0u;
+      }
+      float pe[GP];
+#pragma unroll
+      for (int h = 0; h < GP; ++h) {
+        pe[h] = (valid && h < G) ? ex2(x[h] - m[h]) * vw : 0.f;  // carries 2^-weight of the token's value slot
+        L[h] += pe[h];
+      }
+#pragma unroll
+      for (int g2 = 0; g2 < NG / 2; ++g2) {
+        const float2 zf = half2_to_float2(zv[g2]);
+#pragma unroll
+        for (int h = 0; h < GP; ++h) {
+          zacc[2 * g2][h] = fmaf(pe[h], zf.x, zacc[2 * g2][h]);
+          zacc[2 * g2 + 1][h] = fmaf(pe[h], zf.y, zacc[2 * g2 + 1][h]);
+        }
+      }
+      uint32_t ph[GP / 2];
+#pragma unroll
+      for (int h = 0; h < GP / 2; ++h) ph[h] = pack_half2(pe[2 * h], pe[2 * h + 1]);
+      // row `tid` of B_P: columns gi * GP + h, 8 columns per 16-byte chunk
+      const uint32_t prow = sm_base + Pl::OFF_BP + (tid >> 3) * LBO_P + (tid & 7) * 16;
+#pragma unroll
+      for (int gi = 0; gi < NG; ++gi) {
+        const uint32_t sb = __byte_perm(sv[gi >> 1], 0u, (gi & 1) ? 0x3232 : 0x1010);  // (s, s)
+        if (GP == 4) {
+          if ((gi & 1) == 0) {
+            const uint32_t sb1 = __byte_perm(sv[gi >> 1], 0u, 0x3232);
+            sts128(prow + (gi >> 1) * 128, hmul2_u(ph[0], sb), hmul2_u(ph[1], sb), hmul2_u(ph[0], sb1), hmul2_u(ph[1], sb1));
+          }
+        } else {
+          sts128(prow + gi * 128, hmul2_u(ph[0], sb), hmul2_u(ph[1], sb), hmul2_u(ph[GP / 2 - 2], sb),
+                 hmul2_u(ph[GP / 2 - 1], sb));
+        }
+      }
+    }
+    expand_values<BV>(st + St::OFF_VC, tid, lane_base + COL_AV);
+    tc_wait_st();
+    proxy_fence();
+    tc_fence_before();
+    cp_async_wait<NSTB - 3>();  // batch i + 2 has landed (for this thread); visible to all after the barrier
+    // 6. barrier: A_V and B_P are complete
+    if (__syncthreads_or(lost ? 1 : 0)) {
+      dead = true;
+      break;
+    }
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        umma_ts(tbase + COL_O, tbase + COL_AV + 8 * ks, smem_desc(sm_base + Pl::OFF_BP + ks * 2 * LBO_P, LBO_P, 128), idescO,
+                (i > 0 || ks > 0) ? 1u : 0u);
+      umma_commit(barO);
+    }
+    slot = slot_next;
   }
-  __syncthreads();  // all five warps: tensor memory is no longer used
-  if (warp == UW) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tbase), "r"(TM_COLS) : "memory");
-  if (warp < UW) write_partial(p, mb, nullptr, split, ns + 1, hk, b);
-  ticket_merge(p, ns + 1, hk, b, &s_flag);
+
+  // ---- epilogue ----
+  cp_async_wait<0>();
+  if (!dead) dead = !mbar_wait(barO, phO);  // the last value MMAs
+  dead = __syncthreads_or(dead ? 1 : 0) != 0;
+  tc_fence_after();
+  if (dead && tid == 0) atomicExch(p.status, 1);
+  if (!dead) {
+    // L and the zero-point sums were accumulated with the per-lane factor 2^-weight; undo it, then reduce
+    const float uw = __int_as_float((127 + v_weight_log2<BV>(lane)) << 23);
+    float* wsum = reinterpret_cast<float*>(smem + Pl::OFF_BK);  // [warp][64]; B_K is dead
+#pragma unroll
+    for (int r = 0; r <= NG; ++r) {
+#pragma unroll
+      for (int h = 0; h < GP; ++h) {
+        float v = ((r < NG) ? zacc[r < NG ? r : 0][h] : L[h]) * uw;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) wsum[warp * 64 + r * GP + h] = v;
+      }
+    }
+  }
+  __syncthreads();  // all stages are dead: the memory becomes the merge buffer
+  if (!dead) {
+    const float* wsum = reinterpret_cast<const float*>(smem + Pl::OFF_BK);
+    const int gi = (warp * 32) / GS;  // channel group of this thread's channel
+    float o[GP];
+    tmem_ld_row<GP>(lane_base + COL_O + gi * GP, o);
+    tc_wait_ld();
+#pragma unroll
+    for (int h = 0; h < GP; ++h) {
+      if (h < G) {
+        const float z = wsum[gi * GP + h] + wsum[64 + gi * GP + h] + wsum[128 + gi * GP + h] + wsum[192 + gi * GP + h];
+        mb[h * MS + tid] = fmaf(o[h], 16777216.0f, z);  // the code operands carried 2^-24
+        if (tid == 0) {
+          mb[h * MS + HD] = m[h];
+          mb[h * MS + HD + 1] = wsum[NG * GP + h] + wsum[64 + NG * GP + h] + wsum[128 + NG * GP + h] + wsum[192 + NG * GP + h];
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tbase), "r"(TM_COLS) : "memory");
+  if (dead) {  // leave a neutral partial so that the merge stays finite; the status word tells the host
+    for (int a = 0; a < G; ++a) {
+      mb[a * MS + tid] = 0.f;
+      if (tid == 0) {
+        mb[a * MS + HD] = -CUDART_INF_F;
+        mb[a * MS + HD + 1] = 0.f;
+      }
+    }
+    __syncthreads();
+  }
+  write_partial(p, mb, ws, split, ns, hk, b);
+  ticket_merge(p, ns, hk, b, &s_flag);
 }
 
 template <int BK, int BV, int GS, int GP>
 int smem_bytes(int G) {
-  (void)G;
-  return Plan<BK, BV, GS, GP>::TOTAL;
+  return Plan<BK, BV, GS, GP>::OFF_WS + wstate_bytes(G);
 }
 
 template <int BK, int BV, int GS, int GP>
@@ -997,8 +964,9 @@ cudaError_t launch_t(const DecodeParams& p, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     configured = smem;
   }
-  dim3 grid(p.ns_q + p.ns_w, p.dm.Hkv, p.dm.B);  // packed-region splits, then the window CTA(s)
-  decode_umma_kernel<BK, BV, GS, GP><<<grid, UT_ALL, smem, st>>>(p);
+  const int ns = p.ns_q > 0 ? p.ns_q : p.ns_w;
+  dim3 grid(ns, p.dm.Hkv, p.dm.B);
+  decode_umma_kernel<BK, BV, GS, GP><<<grid, UT, smem, st>>>(p);
   return cudaGetLastError();
 }
 
@@ -1011,11 +979,11 @@ int ctas_per_sm_t(int G) {
     return 0;
   }
   int n = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_umma_kernel<BK, BV, GS, GP>, UT_ALL, smem) != cudaSuccess) {
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_umma_kernel<BK, BV, GS, GP>, UT, smem) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
-  return n < 4 ? n : 4;  // 512 tensor-memory columns per SM, 128 per CTA
+  return n < 2 ? n : 2;  // 512 tensor-memory columns per SM, 256 per CTA
 }
 
 }  // namespace

@@ -187,7 +187,7 @@ int mma_ctas_per_sm(const xq_cache* c, int l) {
   int& slot = const_cast<xq_cache*>(c)->mma_ctas[bk - 1][bv - 1];
   if (slot == 0) {
     slot = decode_mma_ctas_per_sm(c->plan.dm, bk, bv);
-    if (slot <= 0) slot = 4;  // no device to ask
+    if (slot <= 0) slot = 2;  // no device to ask
   }
   return slot;
 }
@@ -210,7 +210,7 @@ void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w) {
       if (ns_w < 1) ns_w = 1;
       return;
     }
-    ns_w = 1;  // one more CTA per stream takes the 16-bit window
+    ns_w = 0;
     // the tensor-core kernel works in 128-token batches; a CTA takes at most decode_mma_max_batches of them
     const int nb = (nq + 127) / 128;
     const int cap = decode_mma_max_batches(dm);
@@ -218,14 +218,13 @@ void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w) {
     if (c->cfg.n_splits > 0) {
       ns_q = c->cfg.n_splits < nb ? c->cfg.n_splits : nb;
       if (ns_q < ns_min) ns_q = ns_min;  // n_splits is a request; ranges longer than the kernel's limit are cut
-      if (ns_q > XQ_MAX_SPLITS - 1) ns_q = XQ_MAX_SPLITS - 1;
       return;
     }
     const double slots = (double)c->sm_count * mma_ctas_per_sm(c, l);
     int best = ns_min;
     double best_score = -1.0;
-    for (int ns = ns_min; ns < XQ_MAX_SPLITS && ns <= nb; ++ns) {
-      double ctas = (double)(ns + 1) * streams;
+    for (int ns = ns_min; ns <= XQ_MAX_SPLITS && ns <= nb; ++ns) {
+      double ctas = (double)ns * streams;
       double waves = ceil(ctas / slots);
       double fill = ctas / (waves * slots);
       double bpc = ceil((double)nb / ns);          // batches of the longest CTA
