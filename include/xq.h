@@ -47,7 +47,6 @@ extern "C" {
 #define XQ_ERR_ORDER (-4)    /* a code-borrowing layer is ahead of the layer owning codes */
 #define XQ_ERR_CUDA (-5)     /* a CUDA call failed; xq_last_cuda_error gives the code     */
 #define XQ_ERR_NOMEM (-6)    /* host allocation failed                                    */
-#define XQ_ERR_DEVICE (-7)   /* a kernel gave up a bounded wait (xq_check_device)         */
 
 #define XQ_BF16 0
 
@@ -208,14 +207,6 @@ long long xq_launch_count(const xq_cache* c);
  * append kernel), the launch count and total milliseconds. */
 int xq_timing_enable(xq_cache* c, int on);
 int xq_timing_read(xq_cache* c, int kind, int* launches, double* total_ms);
-
-/* Kernels of this library never wait without a limit: a CTA whose tensor-core
- * work does not complete within the limit sets a status word in the workspace,
- * releases what it holds and writes a neutral partial (the output is then
- * meaningless).  This call synchronizes `stream` (the one exception to "never
- * synchronizes"), reads that word and returns XQ_OK, XQ_ERR_DEVICE if it was set
- * (the word is cleared), or XQ_ERR_CUDA. */
-int xq_check_device(xq_cache* c, void* stream);
 
 /* CUDA error code (cudaError_t) of the last XQ_ERR_CUDA on this handle, else 0. */
 int xq_last_cuda_error(const xq_cache* c);

@@ -14,7 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libxq.so")
 
 XQ_OK = 0
-XQ_ERR_CONFIG, XQ_ERR_ARG, XQ_ERR_CAPACITY, XQ_ERR_ORDER, XQ_ERR_CUDA, XQ_ERR_NOMEM, XQ_ERR_DEVICE = -1, -2, -3, -4, -5, -6, -7
+XQ_ERR_CONFIG, XQ_ERR_ARG, XQ_ERR_CAPACITY, XQ_ERR_ORDER, XQ_ERR_CUDA, XQ_ERR_NOMEM = -1, -2, -3, -4, -5, -6
 XQ_BF16 = 0
 XQ_KERNEL_AUTO, XQ_KERNEL_GENERIC, XQ_KERNEL_MMA = 0, 1, 2
 XQ_MEM_DEVICE, XQ_MEM_HOST = 0, 1
@@ -62,7 +62,6 @@ _SIGNATURES = {
     "xq_timing_enable": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
     "xq_timing_read": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int),
                                       ctypes.POINTER(ctypes.c_double)]),
-    "xq_check_device": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "xq_last_cuda_error": (ctypes.c_int, [ctypes.c_void_p]),
     "xq_strerror": (ctypes.c_char_p, [ctypes.c_int]),
 }
@@ -189,10 +188,6 @@ def xq_timing_read(handle, kind: int):
     return rc, n.value, ms.value
 
 
-def xq_check_device(handle, stream: int = 0) -> int:
-    return lib().xq_check_device(handle, stream)
-
-
 def xq_last_cuda_error(handle) -> int:
     return lib().xq_last_cuda_error(handle)
 
@@ -269,11 +264,6 @@ class Cache:
         if rc:
             raise XQError(rc, "xq_decode_step")
         return out
-
-    def check_device(self):
-        rc = xq_check_device(self.handle, self._stream())
-        if rc:
-            raise XQError(rc, "xq_check_device")
 
     def seq_len(self, layer):
         return xq_seq_len(self.handle, layer)

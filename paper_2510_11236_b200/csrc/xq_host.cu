@@ -30,7 +30,7 @@ struct LayerRegions {
 struct Plan {
   Dims dm;
   std::vector<LayerRegions> layers;
-  size_t part_acc, part_ml, tickets, status, staging, total;
+  size_t part_acc, part_ml, tickets, staging, total;
   size_t staging_kv_bytes, staging_q_bytes;
 };
 
@@ -88,7 +88,6 @@ void make_plan(const xq_config* c, Plan& pl) {
   pl.part_acc = take((size_t)dm.B * dm.Hq * XQ_MAX_SPLITS * dm.D * 4);
   pl.part_ml = take((size_t)dm.B * dm.Hq * XQ_MAX_SPLITS * 2 * 4);
   pl.tickets = take(BH * 4);
-  pl.status = take(4);
   pl.staging_kv_bytes = (size_t)c->n_layers * BH * dm.D * 2;
   pl.staging_q_bytes = (size_t)c->n_layers * dm.B * dm.Hq * dm.D * 2;
   pl.staging = take(2 * align_up(pl.staging_kv_bytes, 256) + 2 * align_up(pl.staging_q_bytes, 256));
@@ -187,7 +186,7 @@ int mma_ctas_per_sm(const xq_cache* c, int l) {
   int& slot = const_cast<xq_cache*>(c)->mma_ctas[bk - 1][bv - 1];
   if (slot == 0) {
     slot = decode_mma_ctas_per_sm(c->plan.dm, bk, bv);
-    if (slot <= 0) slot = 2;  // no device to ask
+    if (slot <= 0) slot = 3;  // no device to ask
   }
   return slot;
 }
@@ -211,26 +210,20 @@ void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w) {
       return;
     }
     ns_w = 0;
-    // the tensor-core kernel works in 128-token batches; a CTA takes at most decode_mma_max_batches of them
-    const int nb = (nq + 127) / 128;
-    const int cap = decode_mma_max_batches(dm);
-    const int ns_min = (nb + cap - 1) / cap;
     if (c->cfg.n_splits > 0) {
-      ns_q = c->cfg.n_splits < nb ? c->cfg.n_splits : nb;
-      if (ns_q < ns_min) ns_q = ns_min;  // n_splits is a request; ranges longer than the kernel's limit are cut
+      ns_q = c->cfg.n_splits < units ? c->cfg.n_splits : units;
       return;
     }
     const double slots = (double)c->sm_count * mma_ctas_per_sm(c, l);
-    int best = ns_min;
+    int best = 1;
     double best_score = -1.0;
-    for (int ns = ns_min; ns <= XQ_MAX_SPLITS && ns <= nb; ++ns) {
+    for (int ns = 1; ns <= 64 && ns <= units; ++ns) {
       double ctas = (double)ns * streams;
       double waves = ceil(ctas / slots);
       double fill = ctas / (waves * slots);
-      double bpc = ceil((double)nb / ns);          // batches of the longest CTA
-      double score = fill * ((double)nb / ns) / (bpc + 3.0);  // ~3 batches' worth of fixed cost per CTA
+      double upc = (double)units / ns;          // units per CTA
+      double score = fill * upc / (upc + 12.0);  // ~12 units' worth of fixed cost per CTA
       if (score > best_score) { best_score = score; best = ns; }
-      if (ctas > 4 * slots) break;
     }
     ns_q = best;
     return;
@@ -316,11 +309,10 @@ int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, c
   p.out = out;
   p.out_f32 = out_f32;
   p.tickets = (unsigned int*)(c->ws + c->plan.tickets);
-  p.status = (int*)(c->ws + c->plan.status);
   cudaError_t e;
   if (use_mma) {
     if (!c->tickets_clean) {
-      e = cudaMemsetAsync(p.tickets, 0, c->plan.status + 4 - c->plan.tickets, st);  // tickets and the status word
+      e = cudaMemsetAsync(p.tickets, 0, (size_t)dm.B * dm.Hkv * 4, st);
       if (e != cudaSuccess) return fail_cuda(c, e);
       c->tickets_clean = true;
     }
@@ -497,7 +489,7 @@ int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out,
   const size_t ns = (size_t)p.ns_q + (size_t)p.ns_w;
   const size_t acc_bytes = align_up((size_t)dm.B * dm.Hq * ns * dm.D * 4, 256);
   const size_t ml_bytes = align_up((size_t)dm.B * dm.Hq * ns * 2 * 4, 256);
-  const size_t ticket_bytes = align_up((size_t)dm.B * dm.Hkv * 4, 16) + 16;  // tickets, then the status word
+  const size_t ticket_bytes = (size_t)dm.B * dm.Hkv * 4;
   if (acc_bytes + ml_bytes + ticket_bytes > (size_t)XQ_STATIC_SCRATCH_BYTES) return XQ_ERR_CAPACITY;
   uint8_t* base = nullptr;
   cudaError_t e = static_scratch_address(&base);
@@ -505,7 +497,6 @@ int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out,
   p.part_acc = (float*)base;
   p.part_ml = (float*)(base + acc_bytes);
   p.tickets = (unsigned int*)(base + acc_bytes + ml_bytes);
-  p.status = (int*)(base + acc_bytes + ml_bytes + ticket_bytes - 16);
   if (use_mma) {
     // the array keeps whatever the previous call (of any handle) left: tickets must start at zero
     e = cudaMemsetAsync(p.tickets, 0, ticket_bytes, st);
@@ -663,21 +654,6 @@ int xq_timing_read(xq_cache* c, int kind, int* launches, double* total_ms) {
   return XQ_OK;
 }
 
-int xq_check_device(xq_cache* c, void* stream) {
-  if (!c) return XQ_ERR_ARG;
-  cudaStream_t st = (cudaStream_t)stream;
-  cudaError_t e = cudaStreamSynchronize(st);
-  if (e != cudaSuccess) return fail_cuda(c, e);
-  if (!c->tickets_clean) return XQ_OK;  // no kernel that could set the word has run yet
-  int word = 0;
-  e = cudaMemcpy(&word, c->ws + c->plan.status, 4, cudaMemcpyDeviceToHost);
-  if (e != cudaSuccess) return fail_cuda(c, e);
-  if (word == 0) return XQ_OK;
-  e = cudaMemset(c->ws + c->plan.status, 0, 4);
-  if (e != cudaSuccess) return fail_cuda(c, e);
-  return XQ_ERR_DEVICE;
-}
-
 int xq_last_cuda_error(const xq_cache* c) { return c ? c->last_cuda : 0; }
 
 const char* xq_strerror(int code) {
@@ -689,7 +665,6 @@ const char* xq_strerror(int code) {
     case XQ_ERR_ORDER: return "code-owning layer is behind the layer that borrows its codes";
     case XQ_ERR_CUDA: return "CUDA error (see xq_last_cuda_error)";
     case XQ_ERR_NOMEM: return "out of host memory";
-    case XQ_ERR_DEVICE: return "a kernel gave up a bounded wait; its output is invalid";
     default: return "unknown error";
   }
 }

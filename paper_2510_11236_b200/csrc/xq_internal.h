@@ -61,7 +61,6 @@ struct DecodeParams {
   void* out;              // [B,Hq,D] bf16 or f32
   int out_f32;
   unsigned int* tickets;  // [B*Hkv], zero between launches
-  int* status;            // set to 1 by a CTA that gave up a bounded wait
 };
 
 struct MergeParams {
@@ -79,7 +78,6 @@ cudaError_t launch_decode_generic(const DecodeParams& p, cudaStream_t st);
 cudaError_t launch_decode_mma(const DecodeParams& p, cudaStream_t st);
 bool decode_mma_supported(const Dims& dm, int bk, int bv);
 int decode_mma_ctas_per_sm(const Dims& dm, int bk, int bv);
-int decode_mma_max_batches(const Dims& dm);  // 128-token batches one CTA of the tensor-core kernel may take
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t st);
 
 }  // namespace xq
