@@ -204,54 +204,50 @@ def merge_codes_weighted(e0: np.ndarray, e1: np.ndarray, gamma0: float) -> np.nd
 # --------------------------------------------------------------------------
 # Packed layouts (this build's choice; the paper does not discuss packing)
 # --------------------------------------------------------------------------
-# Codes are packed into little-endian 32-bit words.  Inside a word, code number r
-# (r = 0 .. 32/bits - 1) sits in the low 16-bit half if r is even and in the high
-# half if r is odd, at bit bits * (r // 2) of that half.
-#
-# Keys: the D codes of one token fill W = D*bits/32 words, word j holding channels
-# j*cpw .. (j+1)*cpw - 1 (cpw = 32/bits).  The words of a 32-token unit are stored
-# as [W/CW][32 tokens][CW] with CW = min(4, W).
-# Values: per 128-token block and channel, WB = 128*bits/32 words, word j holding
-# tokens j*cpw .. (j+1)*cpw - 1 of the block; stored per block as [WB/4][D][4].
-
-K_PERIOD = 32    # tokens after which the key layout repeats
-V_PERIOD = 128   # tokens after which the value layout repeats
+# A code tile is 128 little-endian 32-bit words.  Each 16-bit half of a word is
+# cut into 16/bits slots of `bits` bits, slot 0 in the least significant bits.
+# D/16 channel blocks share the slots of a word; if slots remain, consecutive
+# 16-token sub-tiles fill them, so one tile spans 16 * (16/bits) / (D/16) tokens.
 
 
-def _bit_in_word(r: int, bits: int) -> int:
-    return 16 * (r % 2) + bits * (r // 2)
+def tokens_per_code_tile(bits: int, D: int) -> int:
+    return 16 * ((16 // bits) // (D // 16))
 
 
 def k_code_position(t: int, d: int, bits: int, D: int):
     """(word index, bit offset) of key code (token t, channel d) in one (batch,
-    kv head) stream."""
-    W = D * bits // 32
-    cpw = 32 // bits
-    CW = min(4, W)
-    j, r = divmod(d, cpw)
-    unit, tl = divmod(t, 32)
-    word = unit * 32 * W + ((j // CW) * 32 + tl) * CW + (j % CW)
-    return word, _bit_in_word(r, bits)
+    kv head) stream.  Within a 16x16 sub-block the token is the row and the
+    channel the column."""
+    cb_n = D // 16
+    tpt = tokens_per_code_tile(bits, D)
+    tile, tl = divmod(t, tpt)
+    tt, row = divmod(tl, 16)
+    cb, kk = divmod(d, 16)
+    lane = (row % 8) * 4 + (kk % 8) // 2
+    i = (row // 8) + 2 * (kk // 8)
+    slot = tt * cb_n + cb
+    return tile * 128 + lane * 4 + i, 16 * (kk % 2) + bits * slot
 
 
 def v_code_position(t: int, d: int, bits: int, D: int):
-    """(word index, bit offset) of value code (token t, channel d)."""
-    WB = 128 * bits // 32
-    cpw = 32 // bits
-    blk, tb = divmod(t, 128)
-    j, r = divmod(tb, cpw)
-    word = blk * D * WB + ((j // 4) * D + d) * 4 + (j % 4)
-    return word, _bit_in_word(r, bits)
+    """(word index, bit offset) of value code (token t, channel d): as for keys
+    with the roles swapped, the channel is the row and the token the column."""
+    cb_n = D // 16
+    tpt = tokens_per_code_tile(bits, D)
+    tile, tl = divmod(t, tpt)
+    tt, tk = divmod(tl, 16)
+    cb, cc = divmod(d, 16)
+    lane = (cc % 8) * 4 + (tk % 8) // 2
+    i = (cc // 8) + 2 * (tk // 8)
+    slot = tt * cb_n + cb
+    return tile * 128 + lane * 4 + i, 16 * (tk % 2) + bits * slot
 
 
-def _n_words(T: int, D: int, bits: int, period: int) -> int:
-    n_periods = -(-T // period)
-    return n_periods * period * D * bits // 32
-
-
-def _pack(codes: np.ndarray, bits: int, pos_fn, period: int) -> np.ndarray:
+def _pack(codes: np.ndarray, bits: int, pos_fn) -> np.ndarray:
     T, D = codes.shape
-    words = np.zeros(_n_words(T, D, bits, period), dtype=np.uint32)
+    tpt = tokens_per_code_tile(bits, D)
+    assert T % tpt == 0
+    words = np.zeros((T // tpt) * 128, dtype=np.uint32)
     for t in range(T):
         for d in range(D):
             w, b = pos_fn(t, d, bits, D)
@@ -259,46 +255,44 @@ def _pack(codes: np.ndarray, bits: int, pos_fn, period: int) -> np.ndarray:
     return words
 
 
+def _position_tables(T: int, D: int, bits: int, pos_fn):
+    w = np.empty((T, D), dtype=np.int64)
+    b = np.empty((T, D), dtype=np.int64)
+    for t in range(T):
+        for d in range(D):
+            w[t, d], b[t, d] = pos_fn(t, d, bits, D)
+    return w, b
+
+
 _TABLE_CACHE: dict = {}
 
 
-def _tables(D: int, bits: int, pos_fn, period: int):
+def _pack_fast(codes: np.ndarray, bits: int, pos_fn) -> np.ndarray:
+    """Same result as _pack; the (word, bit) table of one tile is built by calling
+    the position function for every element of that tile and then reused for
+    every tile (the position function is periodic in the tile by construction;
+    tests check _pack_fast == _pack)."""
+    T, D = codes.shape
+    tpt = tokens_per_code_tile(bits, D)
+    assert T % tpt == 0
     key = (pos_fn.__name__, bits, D)
     if key not in _TABLE_CACHE:
-        w = np.empty((period, D), dtype=np.int64)
-        b = np.empty((period, D), dtype=np.int64)
-        for t in range(period):
-            for d in range(D):
-                w[t, d], b[t, d] = pos_fn(t, d, bits, D)
-        _TABLE_CACHE[key] = (w, b)
-    return _TABLE_CACHE[key]
-
-
-def _pack_fast(codes: np.ndarray, bits: int, pos_fn, period: int) -> np.ndarray:
-    """Same result as _pack; the (word, bit) table of one period is built by
-    calling the position function for every element of that period and reused for
-    every period (tests check _pack_fast == _pack)."""
-    T, D = codes.shape
-    w, b = _tables(D, bits, pos_fn, period)
-    n_periods = -(-T // period)
-    wpp = period * D * bits // 32
-    padded = np.zeros((n_periods * period, D), dtype=np.uint32)
-    padded[:T] = codes
-    c = padded.reshape(n_periods, period, D) << b.astype(np.uint32)[None]
-    words = np.zeros((n_periods, wpp), dtype=np.uint32)
-    for i in range(n_periods):
-        np.bitwise_or.at(words[i], w.reshape(-1), c[i].reshape(-1))
+        _TABLE_CACHE[key] = _position_tables(tpt, D, bits, pos_fn)
+    w, b = _TABLE_CACHE[key]
+    n_tiles = T // tpt
+    c = codes.reshape(n_tiles, tpt, D).astype(np.uint32) << b.astype(np.uint32)[None]
+    words = np.zeros((n_tiles, 128), dtype=np.uint32)
+    for tile in range(n_tiles):
+        np.bitwise_or.at(words[tile], w.reshape(-1), c[tile].reshape(-1))
     return words.reshape(-1)
 
 
 def pack_k_codes(codes: np.ndarray, bits: int, fast: bool = True) -> np.ndarray:
-    """[T, D] codes -> words of ceil(T/32) units (a ragged tail is padded with zero codes)."""
-    return (_pack_fast if fast else _pack)(codes, bits, k_code_position, K_PERIOD)
+    return (_pack_fast if fast else _pack)(codes, bits, k_code_position)
 
 
 def pack_v_codes(codes: np.ndarray, bits: int, fast: bool = True) -> np.ndarray:
-    """[T, D] codes -> words of ceil(T/128) blocks (a ragged tail is padded with zero codes)."""
-    return (_pack_fast if fast else _pack)(codes, bits, v_code_position, V_PERIOD)
+    return (_pack_fast if fast else _pack)(codes, bits, v_code_position)
 
 
 def _unpack(words: np.ndarray, T: int, D: int, bits: int, pos_fn) -> np.ndarray:
@@ -319,16 +313,48 @@ def unpack_v_codes(words, T, D, bits):
     return _unpack(words, T, D, bits, v_code_position)
 
 
+def k_meta_position(d: int, D: int) -> int:
+    """Index of channel d inside the D-entry scale (or zero-point) block of one
+    key token-group: 8-entry chunks, chunk 4*(d//32) + ((d%16)%8)//2, and inside
+    the chunk the entry ((d//16)%2)*4 + ((d%16)//8)*2 + d%2."""
+    cb, kk = divmod(d, 16)
+    chunk = (cb // 2) * 4 + (kk % 8) // 2
+    return chunk * 8 + (cb % 2) * 4 + (kk // 8) * 2 + (kk % 2)
+
+
 def pack_k_meta(s_hat: np.ndarray, z_hat: np.ndarray) -> np.ndarray:
     """[n_groups, D] fp16 scale and zero -> uint16 [2, n_groups, D]: the plane of
-    scale blocks, then the plane of zero-point blocks, channels in order."""
-    return np.stack([s_hat.astype(np.float16).view(np.uint16), z_hat.astype(np.float16).view(np.uint16)])
+    permuted scale blocks, then the plane of permuted zero-point blocks."""
+    n, D = s_hat.shape
+    out = np.zeros((2, n, D), dtype=np.uint16)
+    su = s_hat.astype(np.float16).view(np.uint16)
+    zu = z_hat.astype(np.float16).view(np.uint16)
+    for d in range(D):
+        p = k_meta_position(d, D)
+        out[0, :, p] = su[:, d]
+        out[1, :, p] = zu[:, d]
+    return out
+
+
+def v_meta_position(tk: int, gi: int, n_g: int) -> int:
+    """Index of (token tk of a 16-token tile, channel group gi) inside the
+    16*n_g-entry scale (or zero-point) block of that tile."""
+    return ((tk % 8) // 2) * (n_g * 4) + gi * 4 + (tk // 8) * 2 + (tk % 2)
 
 
 def pack_v_meta(s_hat: np.ndarray, z_hat: np.ndarray) -> np.ndarray:
-    """[T, n_g] fp16 scale and zero -> uint16 [T, 2, n_g]: per token its scales,
-    then its zero-points."""
-    return np.stack([s_hat.astype(np.float16).view(np.uint16), z_hat.astype(np.float16).view(np.uint16)], axis=1)
+    """[T, n_g] fp16 scale and zero -> uint16 [T/16, 2, 16*n_g]."""
+    T, n_g = s_hat.shape
+    assert T % 16 == 0
+    out = np.zeros((T // 16, 2, 16 * n_g), dtype=np.uint16)
+    su = s_hat.astype(np.float16).view(np.uint16).reshape(T // 16, 16, n_g)
+    zu = z_hat.astype(np.float16).view(np.uint16).reshape(T // 16, 16, n_g)
+    for tk in range(16):
+        for gi in range(n_g):
+            p = v_meta_position(tk, gi, n_g)
+            out[:, 0, p] = su[:, tk, gi]
+            out[:, 1, p] = zu[:, tk, gi]
+    return out
 
 
 # --------------------------------------------------------------------------

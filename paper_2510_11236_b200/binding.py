@@ -217,7 +217,7 @@ class Cache:
             raise XQError(XQ_ERR_CONFIG, "xq_workspace_bytes")
         self.nbytes = nbytes
         with torch.cuda.device(self.device):
-            self.workspace = torch.zeros(nbytes, dtype=torch.uint8, device=self.device)
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
             assert self.workspace.data_ptr() % 256 == 0
             rc, self.handle = xq_create(cfg, self.workspace, nbytes)
         if rc != XQ_OK:

@@ -11,7 +11,6 @@
 
 #include "../../include/xq.h"
 #include "xq_internal.h"
-#include "xq_layout.cuh"
 
 using namespace xq;
 
@@ -65,7 +64,7 @@ void make_plan(const xq_config* c, Plan& pl) {
   Dims& dm = pl.dm;
   dm.B = c->batch; dm.Hq = c->n_q_heads; dm.Hkv = c->n_kv_heads; dm.G = dm.Hq / dm.Hkv;
   dm.D = c->head_dim; dm.g = c->group_size; dm.R = c->residual_len; dm.NG = dm.D / dm.g;
-  dm.nq_cap = c->max_seq > 1 ? round_up_128(((c->max_seq - 1) / dm.R) * dm.R) : 0;
+  dm.nq_cap = c->max_seq > 1 ? ((c->max_seq - 1) / dm.R) * dm.R : 0;
   const size_t BH = (size_t)dm.B * dm.Hkv;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
@@ -77,7 +76,7 @@ void make_plan(const xq_config* c, Plan& pl) {
     r.win_k = take(BH * r.stride[4]);
     r.win_v = take(BH * r.stride[5]);
     r.stride[2] = (size_t)(dm.nq_cap / dm.g) * 2 * dm.D * 2;
-    r.stride[3] = (size_t)dm.nq_cap * 2 * dm.NG * 2;
+    r.stride[3] = (size_t)(dm.nq_cap / 16) * 2 * 16 * dm.NG * 2;
     r.k_meta = take(BH * r.stride[2]);
     r.v_meta = take(BH * r.stride[3]);
     r.stride[0] = (size_t)dm.nq_cap * dm.D * bk / 8;

@@ -7,7 +7,7 @@ namespace xq {
 
 struct Dims {
   int B, Hq, Hkv, G, D, g, R, NG;
-  int nq_cap;  // capacity of the quantized region in tokens (whole 128-token blocks)
+  int nq_cap;  // capacity of the quantized region in tokens (multiple of R)
 };
 
 // Device addresses of one layer's regions (codes: of the layer that owns them).
@@ -15,7 +15,7 @@ struct LayerPtrs {
   uint16_t* win_k;   // [B,Hkv,R,D] bf16
   uint16_t* win_v;
   uint16_t* k_meta;  // [B,Hkv,2,nq_cap/g,D] fp16 (scale plane, zero-point plane)
-  uint16_t* v_meta;  // [B,Hkv,nq_cap,2,NG] fp16 (per token: scales, zero-points)
+  uint16_t* v_meta;  // [B,Hkv,nq_cap/16,2,16*NG] fp16
   uint32_t* k_codes; // [B,Hkv,nq_cap*D*bk/32]
   uint32_t* v_codes;
   int bk, bv;

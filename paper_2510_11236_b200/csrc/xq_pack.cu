@@ -87,10 +87,11 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
       group_params(mn, mx, bits, eta, z, s, zh, sh);
       z_arr[item] = z;
       s_arr[item] = s;
-      const size_t cap_g = (size_t)(dm.nq_cap / g);  // nq_cap is a multiple of 128, hence of g
+      const size_t cap_g = (size_t)(dm.nq_cap / g);
       size_t grp = (size_t)bh * 2 * cap_g + (tq0 / g + gl);  // scale plane, then zero-point plane
-      meta[grp * D + d] = sh;
-      meta[(grp + cap_g) * D + d] = zh;
+      int pos = k_meta_position(d, D);
+      meta[grp * D + pos] = sh;
+      meta[(grp + cap_g) * D + pos] = zh;
     }
   } else {
     // values: one group per (token, run of g channels)
@@ -110,48 +111,48 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
       z_arr[item] = z;
       s_arr[item] = s;
       int tabs = tq0 + tl;
-      const size_t base = (size_t)bh * dm.nq_cap * (2 * NG);
-      meta[base + v_meta_index(tabs, gi, 0, NG)] = sh;
-      meta[base + v_meta_index(tabs, gi, 1, NG)] = zh;
+      size_t t16 = (size_t)bh * (dm.nq_cap / 16) + tabs / 16;
+      int pos = v_meta_position(tabs % 16, gi, NG);
+      meta[(t16 * 2 + 0) * (16 * NG) + pos] = sh;
+      meta[(t16 * 2 + 1) * (16 * NG) + pos] = zh;
     }
   }
   if (!own) return;  // PseudoQuantize: parameters only
   __syncthreads();
 
   // codes: each thread assembles whole 32-bit words of the packed layout
-  const int cpw = 32 / bits;  // codes per word
+  const int nslot = 16 / bits;
+  const int CB = D / 16;
+  const int tpt = tokens_per_code_tile(bits, D);
+  const int words_per_token_x32 = D * bits;  // words per 32 tokens
+  const int n_words = tb * D * bits / 32;
   uint32_t* codes = kind ? p.L.v_codes : p.L.k_codes;
   const size_t stream_words = (size_t)dm.nq_cap * D * bits / 32;
-  uint32_t* dst = codes + (size_t)bh * stream_words;
-  const int n_words = tb * D / cpw;
-  if (kind == 0) {
-    // a key word: cpw consecutive channels of one token
-    const int W = k_words_per_token(bits, D);
-    for (int wl = tid; wl < n_words; wl += PACK_THREADS) {
-      const int tl = wl / W, j = wl % W;
-      uint32_t word = 0;
-      for (int r = 0; r < cpw; ++r) {
-        const int d = j * cpw + r;
-        const float x = bf16_bits(tile[tl * D + d]);
-        const int gidx = (tl / g) * D + d;
-        word |= code_of(x, z_arr[gidx], s_arr[gidx], qmax) << (16 * (r & 1) + bits * (r >> 1));
+  uint32_t* dst = codes + (size_t)bh * stream_words + (size_t)(tq0 / 32) * words_per_token_x32;
+  for (int wl = tid; wl < n_words; wl += PACK_THREADS) {
+    int tile_l = wl >> 7, w = wl & 127;
+    int lane = w >> 2, i = w & 3;
+    uint32_t word = 0;
+    for (int hf = 0; hf < 2; ++hf) {
+      int row = (lane >> 2) + 8 * (i & 1);
+      int col = 2 * (lane & 3) + hf + 8 * (i >> 1);
+      for (int slot = 0; slot < nslot; ++slot) {
+        int tt = slot / CB, cb = slot % CB;
+        int tl, d;
+        if (kind == 0) {
+          tl = tile_l * tpt + tt * 16 + row;
+          d = cb * 16 + col;
+        } else {
+          tl = tile_l * tpt + tt * 16 + col;
+          d = cb * 16 + row;
+        }
+        float x = bf16_bits(tile[tl * D + d]);
+        int gidx = (kind == 0) ? (tl / g) * D + d : tl * NG + d / g;
+        uint32_t c = code_of(x, z_arr[gidx], s_arr[gidx], qmax);
+        word |= c << (16 * hf + bits * slot);
       }
-      dst[k_code_position(tq0 + tl, j * cpw, bits, D).word] = word;
     }
-  } else {
-    // a value word: cpw consecutive tokens of one channel
-    const int wpc = tb / cpw;  // words per channel in this tile
-    for (int wl = tid; wl < n_words; wl += PACK_THREADS) {
-      const int d = wl / wpc, jl = wl % wpc;
-      uint32_t word = 0;
-      for (int r = 0; r < cpw; ++r) {
-        const int tl = jl * cpw + r;
-        const float x = bf16_bits(tile[tl * D + d]);
-        const int gidx = tl * NG + d / g;
-        word |= code_of(x, z_arr[gidx], s_arr[gidx], qmax) << (16 * (r & 1) + bits * (r >> 1));
-      }
-      dst[v_code_position(tq0 + jl * cpw, d, bits, D).word] = word;
-    }
+    dst[wl] = word;
   }
 }
 

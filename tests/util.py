@@ -45,14 +45,14 @@ def compare_regions(cache, oc, layer, b, hk):
     got = cache.region(layer, 0)[bh].cpu().numpy().view(np.uint32)[: nq * D * bk // 32]
     want = O.pack_k_codes(kc[0, 0], bk)
     assert np.array_equal(got, want), f"key codes differ in {np.count_nonzero(got != want)} words"
-    want = O.pack_v_codes(vc[0, 0], bv)  # whole 128-token blocks; the workspace starts zeroed, as the padding
-    got = cache.region(layer, 1)[bh].cpu().numpy().view(np.uint32)[: want.size]
+    got = cache.region(layer, 1)[bh].cpu().numpy().view(np.uint32)[: nq * D * bv // 32]
+    want = O.pack_v_codes(vc[0, 0], bv)
     assert np.array_equal(got, want), f"value codes differ in {np.count_nonzero(got != want)} words"
     got = cache.region(layer, 2)[bh].cpu().numpy().view(np.uint16).reshape(2, -1, D)[:, : nq // g]
     want = O.pack_k_meta(ks[0, 0], kz[0, 0])
     assert np.array_equal(got, want), f"key scale/zero differ in {np.count_nonzero(got != want)} entries"
     n_g = D // g
-    got = cache.region(layer, 3)[bh].cpu().numpy().view(np.uint16)[: nq * 2 * n_g]
+    got = cache.region(layer, 3)[bh].cpu().numpy().view(np.uint16)[: (nq // 16) * 2 * 16 * n_g]
     want = O.pack_v_meta(vs[0, 0], vz[0, 0]).reshape(-1)
     assert np.array_equal(got, want), f"value scale/zero differ in {np.count_nonzero(got != want)} entries"
 
