@@ -20,8 +20,8 @@
 // Work split: grid (split, kv head, sequence), sized by the host to one wave of
 // long-lived CTAs.  Every split takes a contiguous range of 32-token units of the
 // packed region, cut into four contiguous warp ranges, plus an equal share of the
-// 16-bit window tokens (scalar fp32 path, its loads issued together, done while
-// the first packed stages are in flight).  Each warp stages its own units in
+// 16-bit window tokens, which one of its warps takes as tiles of 16 tokens (bf16
+// tensor-core operands loaded with ldmatrix) before its packed units.  Each warp stages its own units in
 // shared memory with cp.async (a ring of NST stages: key codes, key scales, value
 // codes, value scale / zero-point of one unit) and, once per 16 units, the key
 // zero-point rows of the next 16 units, from which the q . z biases of those
@@ -168,7 +168,6 @@ constexpr int ZTAB_BYTES = ZROWS * 8 * 4;  // q . z biases [unit][head], fp32, l
 constexpr int MS = HD + 4;                 // state row: acc[HD], m, l, padding (keeps rows 16-byte aligned)
 constexpr int MERGE_BYTES = MMA_WARPS * 8 * MS * 4;
 constexpr int Q_BYTES = 32 * 64;
-__host__ __device__ inline int wstate_bytes(int G) { return MMA_WARPS * G * MS * 4; }
 
 // dynamic shared memory:
 //   [per warp: NST stages | zero-point rows | bias table]   (the merge buffer aliases the start after the loop)
@@ -284,6 +283,109 @@ __device__ __forceinline__ void window_tokens(const DecodeParams& p, int t0, int
         row[HD + 1] = l[a];
       }
     }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// window tiles on the tensor cores: 16 tokens of the 16-bit window are staged
+// row by row (rows padded to WROW bytes against bank conflicts) and enter the
+// same softmax state as the packed units, as bf16 operands.
+// ---------------------------------------------------------------------------
+constexpr int WROW = 2 * HD + 16;        // bytes per staged window row
+constexpr int WIN_BYTES = 2 * 16 * WROW;  // 16 key rows, then 16 value rows
+
+__device__ __forceinline__ void mma16816_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// One warp stages window tokens [tb, tb + 16) (rows at or beyond t1 are zero-filled); no commit.
+__device__ __forceinline__ void window_stage(const DecodeParams& p, int tb, int t1, int hk, int b, uint32_t wbuf, int lane) {
+  const Dims& dm = p.dm;
+  const size_t row0 = (size_t)(b * dm.Hkv + hk) * dm.R;
+  const uint8_t* wk = reinterpret_cast<const uint8_t*>(p.L.win_k);
+  const uint8_t* wv = reinterpret_cast<const uint8_t*>(p.L.win_v);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int chunk = lane + 32 * i, row = chunk >> 4, c = chunk & 15;
+    const uint32_t dk = wbuf + row * WROW + c * 16, dv = dk + 16 * WROW;
+    if (tb + row < t1) {
+      const size_t off = (row0 + tb + row) * (2 * HD) + c * 16;
+      cp_async16(dk, wk + off);
+      cp_async16(dv, wv + off);
+    } else {
+      asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};\n" ::"r"(dk), "r"(0u) : "memory");
+      asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};\n" ::"r"(dv), "r"(0u) : "memory");
+    }
+  }
+}
+
+// One warp folds the staged tile (n_valid of its 16 tokens exist) into its softmax state.  accO is kept in true
+// units here (the caller applies the slot weights of the packed path once all window tiles are in).
+// qb: q of head gid as bf16 pairs in B-operand order (as loaded), scale2: softmax scale in log2 units.
+__device__ __forceinline__ void window_tile(uint32_t wbuf, int n_valid, const uint32_t (&qb)[16], float scale2,
+                                            float (&accO)[8][4], float (&accZ)[4], float& m0, float& m1, int lane) {
+  const int gid = lane >> 2;
+  float s[4] = {0.f, 0.f, 0.f, 0.f};  // rows = tokens gid, gid + 8; cols = heads 2 tig, 2 tig + 1
+  const uint32_t ka = wbuf + ((lane & 7) + 8 * ((lane >> 3) & 1)) * WROW + (lane >> 4) * 16;
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    uint32_t a0, a1, a2, a3;
+    ldmatrix_x4(ka + ks * 32, a0, a1, a2, a3);
+    mma16816_bf16(s, a0, a1, a2, a3, qb[2 * ks], qb[2 * ks + 1]);
+  }
+  const bool va = gid < n_valid, vb = gid + 8 < n_valid;
+  const float x00 = va ? s[0] * scale2 : -CUDART_INF_F, x01 = va ? s[1] * scale2 : -CUDART_INF_F;
+  const float x10 = vb ? s[2] * scale2 : -CUDART_INF_F, x11 = vb ? s[3] * scale2 : -CUDART_INF_F;
+  float r0 = fmaxf(x00, x10), r1 = fmaxf(x01, x11);
+#pragma unroll
+  for (int o = 4; o < 32; o <<= 1) {
+    r0 = fmaxf(r0, __shfl_xor_sync(0xffffffffu, r0, o));
+    r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, o));
+  }
+  const float mn0 = fmaxf(m0, r0), mn1 = fmaxf(m1, r1);  // finite: token 0 of the tile exists
+  const float f0 = ex2(m0 - mn0), f1 = ex2(m1 - mn1);
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt) {
+    accO[mt][0] *= f0; accO[mt][1] *= f1; accO[mt][2] *= f0; accO[mt][3] *= f1;
+  }
+  accZ[0] *= f0; accZ[1] *= f1; accZ[2] *= f0; accZ[3] *= f1;
+  m0 = mn0; m1 = mn1;
+  const float p00 = ex2(x00 - m0), p01 = ex2(x01 - m1), p10 = ex2(x10 - m0), p11 = ex2(x11 - m1);
+  // numerators as bf16 hi + lo (16 bits of precision), transposed into B-operand order
+  const uint32_t h0 = pack_bf16x2(p00, p01), h1 = pack_bf16x2(p10, p11);
+  const uint32_t l0 = pack_bf16x2(p00 - bf16_to_f(h0 & 0xffff), p01 - bf16_to_f(h0 >> 16));
+  const uint32_t l1 = pack_bf16x2(p10 - bf16_to_f(h1 & 0xffff), p11 - bf16_to_f(h1 >> 16));
+  const uint32_t bh0 = movmatrix_trans(h0), bh1 = movmatrix_trans(h1), bl0 = movmatrix_trans(l0), bl1 = movmatrix_trans(l1);
+  const uint32_t ones = (gid == 0) ? 0x3F803F80u : 0u;  // row 8 of the sums tile: sum_t p_t
+  mma16816_bf16(accZ, 0u, ones, 0u, ones, bh0, bh1);
+  mma16816_bf16(accZ, 0u, ones, 0u, ones, bl0, bl1);
+  // O^T += V^T P: A fragments are transposed 8x8 blocks of the row-major value rows
+  const int mi = lane >> 3;
+  const uint32_t va_addr = wbuf + 16 * WROW + ((lane & 7) + 8 * (mi >> 1)) * WROW + (mi & 1) * 16;
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt) {
+    uint32_t a0, a1, a2, a3;
+    ldmatrix_x4_trans(va_addr + mt * 32, a0, a1, a2, a3);
+    mma16816_bf16(accO[mt], a0, a1, a2, a3, bh0, bh1);
+    mma16816_bf16(accO[mt], a0, a1, a2, a3, bl0, bl1);
   }
 }
 
@@ -488,7 +590,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   __shared__ int s_flag;
   float* mb = reinterpret_cast<float*>(smem);                   // merge buffer (after the loop)
   uint32_t* q_sm = reinterpret_cast<uint32_t*>(smem + PIPE);     // [4 chunks][lane][4] half2
-  float* ws = reinterpret_cast<float*>(smem + PIPE + Q_BYTES);  // window states
+  float* ws = reinterpret_cast<float*>(smem);                  // window states of the window-only path
 
   const Dims& dm = p.dm;
   const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
@@ -569,10 +671,12 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
 #pragma unroll
     for (int i = 0; i < 16; ++i) raw[i] = real ? *reinterpret_cast<const uint32_t*>(qp + 16 * (i >> 1) + 8 * (i & 1)) : 0u;
   }
-  WindowRegs wr;
-  window_preload(p, wt0, wt1, hk, b, wr);
+  // the CTA's share of the window, in tiles of 16 tokens, goes to one warp (rotating with the split index)
+  const int ww = split & (MMA_WARPS - 1);
+  const uint32_t wbuf = sm_base + PIPE + Q_BYTES;
+  if (warp == ww && wt0 < wt1) window_stage(p, wt0, wt1, hk, b, wbuf, lane);
 
-  // start the pipeline (group jj holds unit jj; group 0 also the first zero-point rows)
+  // start the pipeline (group jj holds unit jj; group 0 also the first zero-point rows and the first window tile)
 #pragma unroll
   for (int jj = 0; jj < NST - 1; ++jj) {
     issue_unit(jj, jj * St::BYTES);
@@ -591,7 +695,6 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
       qe[2 * s + j] = pack_half2(lo * sc, hi * sc);
     }
   }
-  window_tokens(p, wt0, wt1, hk, b, ws, wr);  // while the copies fly
   __syncthreads();
 
   const float scale2 = p.scale * 1.4426950408889634f;
@@ -605,11 +708,28 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;  // softmax reference (log2 units) of heads 2 tig, 2 tig + 1
   float accS[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 
-  if (n_my > 0) {
-    cp_async_wait<NST - 2>();  // unit 0 and the first zero-point rows have landed
-    __syncwarp();
-    unit_logits<BK, BV, GS>(my, qe, accS, lane, tig);
+  cp_async_wait<NST - 2>();  // unit 0, the first zero-point rows and the first window tile have landed
+  __syncwarp();
+  if (warp == ww && wt0 < wt1) {
+    // window tokens first (the accumulators are empty): true units, then the slot weights of the packed path
+    for (int tb = wt0; tb < wt1; tb += 16) {
+      if (tb > wt0) {  // a share of more than 16 tokens (few splits): stage the next tile and wait for it
+        __syncwarp();
+        window_stage(p, tb, wt1, hk, b, wbuf, lane);
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncwarp();
+      }
+      window_tile(wbuf, wt1 - tb, raw, scale2, accO, accZ, m0, m1, lane);
+    }
+#pragma unroll
+    for (int mt = 0; mt < 8; ++mt) {
+      const float wgt = 1.0f / (float)(1u << (24 - Slots<BV>::e(mt)));
+#pragma unroll
+      for (int i = 0; i < 4; ++i) accO[mt][i] *= wgt;
+    }
   }
+  if (n_my > 0) unit_logits<BK, BV, GS>(my, qe, accS, lane, tig);
 
   // One iteration: bias table every ZROWS units, refill of the stage unit j - 1 used, softmax reference,
   // numerators of unit j, then (MORE) logits of unit j + 1 next to the value product of unit j.
@@ -726,13 +846,14 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     }
   }
   __syncthreads();
-  write_partial(p, mb, ws, split, ns, hk, b);
+  write_partial(p, mb, nullptr, split, ns, hk, b);
   ticket_merge(p, ns, hk, b, &s_flag);
 }
 
 template <int BK, int BV, int GS>
 int smem_bytes(int G) {
-  return pipe_bytes<BK, BV, GS>() + Q_BYTES + wstate_bytes(G);
+  (void)G;
+  return pipe_bytes<BK, BV, GS>() + Q_BYTES + WIN_BYTES;
 }
 
 template <int BK, int BV, int GS>
