@@ -183,3 +183,54 @@ def test_decode_step_device_and_host():
             ref = a.decode_attention(l, q[l])
             assert torch.equal(ref, out_d[l])
     assert xq.xq_launch_count(a.handle) > 0
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4"])
+def test_full_size_configs_sampled(name):
+    """The benchmark's shapes and launch configuration (library-chosen splits, tensor-core kernel), one layer
+    pair at the full context: codes, scales and zero-points of sampled streams bit for bit, attention of the
+    sampled streams' query heads against the oracle."""
+    w = dict(W.CONFIGS[name], n_layers=2)
+    w["kq"], w["vq"] = min(w["kq"], 2), min(w["vq"], 2)
+    cfg = W.make_xq_config(w)  # n_splits as the workload names it (0 = library's choice, c4: 64)
+    cache = xq.Cache(cfg, DEV)
+    S, B, Hkv = w["seq"], w["batch"], w["n_kv_heads"]
+    streams = sorted({(0, 0), (B - 1, Hkv - 1), (B // 2, Hkv // 3)})
+    kv = {0: {}, 1: {}}  # per layer, per stream: the tokens of that stream only (host side)
+    parts = {s: [[], [], [], []] for s in streams}
+    for c0 in range(0, S, W.CHUNK):
+        k0, v0, k1, v1 = W.pair_tokens(w, 0, c0, min(S, c0 + W.CHUNK), DEV)
+        cache.append_kv(0, k0, v0)
+        cache.append_kv(1, k1, v1)
+        for (b, h) in streams:
+            for lst, t in zip(parts[(b, h)], (k0, v0, k1, v1)):
+                lst.append(t[b:b + 1, h:h + 1].cpu())
+    torch.cuda.synchronize()
+    assert cache.seq_len(1) == S and cache.quantized_len(1) == S - w["residual_len"]
+    rc, nsq, nsw = xq.xq_split_plan(cache.handle, 0)
+    assert rc == 0 and nsq >= 1
+    if name == "c4":
+        assert nsq == 64
+    G = w["n_q_heads"] // Hkv
+    worst = 0.0
+    for layer in (0, 1):
+        q = W.queries(w, layer, 0, DEV)
+        o32 = cache.decode_attention(layer, q, f32=True)
+        o16 = cache.decode_attention(layer, q)
+        torch.cuda.synchronize()
+        for (b, h) in streams:
+            k0, v0, k1, v1 = (torch.cat(x, dim=2) for x in parts[(b, h)])
+            one = {0: (k0, v0), 1: (k1, v1)}
+            oc = util.oracle_for_stream(cfg, [0, 1], 0, 0, one)
+            # the oracle holds this one stream as (sequence 0, kv head 0): compare its regions with stream (b, h)
+            util.compare_regions(cache, oc, layer, b, h)
+            qs = q[b:b + 1, h * G:(h + 1) * G]
+            ref = oc.decode(layer, util.bits_of(qs))[0]
+            got = o32[b, h * G:(h + 1) * G].double().cpu().numpy()
+            err = np.abs(got - ref).max()
+            assert err <= util.ATTN_TOL, f"{name} layer {layer} stream {(b, h)}: fp32 attention error {err}"
+            got16 = o16[b, h * G:(h + 1) * G].double().cpu().numpy()
+            assert (np.abs(got16 - ref) <= util.ATTN_TOL + 2.0 ** -8 * np.abs(ref)).all()
+            worst = max(worst, err)
+    print(f"{name}: splits {nsq}+{nsw}, worst fp32 attention error over sampled streams {worst:.2e}")
+    cache.close()
