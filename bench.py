@@ -193,6 +193,7 @@ def main():
     import torch
     import torch.distributed as dist
     import paper_2510_11236_b200 as xq
+    from paper_2510_11236_b200 import sharding
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -201,7 +202,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
-    w["seed"] = w["seed"] + 101 * rank  # every rank holds its own sequences
+    w = sharding.rank_workload(w, rank)  # every rank holds its own sequences
 
     L, B, Hq, Hkv, D, S = w["n_layers"], w["batch"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"], w["seq"]
     K, Wm = args.steps, args.warmup
@@ -275,12 +276,9 @@ def main():
     clocks = sampler.stop() if sampler else None
     launches = xq.xq_launch_count(cache.handle) - launches_before
     bytes_pass1 = step_bytes(seq_before + 1, K)
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_max = float(t.item())
-    value = world * bytes_pass1 / (ms_max * 1e-3) / 1e9
-    tokens_per_s = world * B * sum(seq_before + 1 + i for i in range(K)) * L / (ms_max * 1e-3) / L
+    ms_max = sharding.max_over_ranks(ms, dev)
+    value = sharding.aggregate_rate(bytes_pass1, ms_max, world) / 1e9
+    tokens_per_s = sharding.aggregate_rate(B * sum(seq_before + 1 + i for i in range(K)), ms_max, world)
 
     # ---- pass 2: the same steps with CUDA events around every kernel (roofline of the dominant kernel)
     xq.xq_timing_enable(cache.handle, 1)
@@ -314,10 +312,8 @@ def main():
     e1.record()
     barrier()
     ms3 = e0.elapsed_time(e1)
-    t = torch.tensor([ms3], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_val = world * step_bytes(seq_before3 + 1, K) / (float(t.item()) * 1e-3) / 1e9
+    ms3_max = sharding.max_over_ranks(ms3, dev)
+    e2e_val = sharding.aggregate_rate(step_bytes(seq_before3 + 1, K), ms3_max, world) / 1e9
 
     if rank == 0:
         nsq = nsw = None
@@ -341,7 +337,7 @@ def main():
             "gpu_launches": int(launches),
             "clocks": clocks,
             "e2e": {"value": e2e_val, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": float(t.item()) / K},
+                    "ms_per_step": ms3_max / K},
             "roofline": {"bound": "hbm", "kernel": "decode split kernel", "achieved": achieved, "peak": peak,
                          "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                          "frac_of_8TBps": achieved / 8000.0, "traffic": None,
