@@ -801,16 +801,11 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     unit_values<BK, BV, GS>(my + off_cur, pb, accO, accZ, lane, gid, tig);
   };
 
-  // main loop, unrolled over the ring so that every stage address is a constant offset
-  static_assert(NST == 4, "the loop below is unrolled for a ring of four stages");
-  int j = 0;
-  for (; j + NST < n_my; j += NST) {
-    step(j + 0, true, 3 * St::BYTES, 0 * St::BYTES, 1 * St::BYTES);
-    step(j + 1, true, 0 * St::BYTES, 1 * St::BYTES, 2 * St::BYTES);
-    step(j + 2, true, 1 * St::BYTES, 2 * St::BYTES, 3 * St::BYTES);
-    step(j + 3, true, 2 * St::BYTES, 3 * St::BYTES, 0 * St::BYTES);
-  }
-  for (; j < n_my; ++j)  // the last one to four units; the very last has no successor
+  // main loop: one copy of the body (four unrolled copies with constant stage offsets save address arithmetic
+  // but cost more in instruction-cache misses than they save)
+  static_assert(NST == 4, "ring of four stages");
+#pragma unroll 1
+  for (int j = 0; j < n_my; ++j)  // the very last unit has no successor
     step(j, j + 1 < n_my, ((j + 3) & 3) * St::BYTES, (j & 3) * St::BYTES, ((j + 1) & 3) * St::BYTES);
   cp_async_wait<0>();
   __syncthreads();  // all warps are done with their stages: the memory becomes the merge buffer
