@@ -30,6 +30,10 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "decode-attention GB/s at 32k ctx"
+APPEND_BLOCKS = 6  # window blocks quantized per layer in the append pass
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the decode kernel (ncu, same launch shape as the
+# timed one; see profiles/).  Valid only for the kernel version the counters were taken on.
+NCU_TRAFFIC_BYTES = {"c2": 84.05e6 + 2.95e6}
 
 
 def _peaks():
@@ -206,7 +210,8 @@ def main():
 
     L, B, Hq, Hkv, D, S = w["n_layers"], w["batch"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"], w["seq"]
     K, Wm = args.steps, args.warmup
-    n_total = Wm + 3 * K + 8  # warm-up, then three timed passes (device, per-kernel events, host buffers)
+    R = w["residual_len"]
+    n_total = Wm + 3 * K + 8 + (APPEND_BLOCKS + 1) * R  # warm-up, three timed passes, then the append pass
     cfg = W.make_xq_config(w, max_seq=S + n_total + 1, eta1=args.eta1, eta2=args.eta2, kernel=args.kernel,
                            n_splits=args.splits)
     cache = xq.Cache(cfg, dev)
@@ -315,6 +320,31 @@ def main():
     ms3_max = sharding.max_over_ranks(ms3, dev)
     e2e_val = sharding.aggregate_rate(step_bytes(seq_before3 + 1, K), ms3_max, world) / 1e9
 
+    # ---- pass 4: the quantize-and-pack path: every layer receives whole window blocks (R tokens per call), so each
+    # ---- call quantizes and packs the block that filled the window (code-owning layers: codes + scale / zero-point;
+    # ---- borrowing layers: scale / zero-point only)
+    gk = torch.Generator(device=dev).manual_seed(99 + rank)
+    blk = [torch.randn(B, Hkv, R, D, generator=gk, device=dev).to(torch.bfloat16) for _ in range(4)]
+    fill = R - (cache.seq_len(0) % R)  # top the window up so that the next R tokens flush exactly one block
+    for l in range(L):
+        cache.append_kv(l, blk[0][:, :, :fill].contiguous(), blk[1][:, :, :fill].contiguous())
+    xq.xq_timing_enable(cache.handle, 1)
+    barrier()
+    for i in range(APPEND_BLOCKS):
+        for l in range(L):
+            cache.append_kv(l, blk[(i + l) % 4], blk[(i + l + 1) % 4])
+    barrier()
+    _, n_pack, ms_pack = xq.xq_timing_read(cache.handle, 2)
+    _, n_wapp, ms_wapp = xq.xq_timing_read(cache.handle, 3)
+    xq.xq_timing_enable(cache.handle, 0)
+    block_in_bytes = 2 * B * Hkv * R * D * 2  # 16-bit K and V of one block
+    append = {"block_tokens": R, "blocks_per_layer": APPEND_BLOCKS, "pack_launches": n_pack,
+              "pack_avg_us": ms_pack / n_pack * 1e3 if n_pack else None,
+              "pack_input_gbs": block_in_bytes / (ms_pack / n_pack * 1e-3) / 1e9 if n_pack else None,
+              "pack_frac_of_measured_hbm": (block_in_bytes / (ms_pack / n_pack * 1e-3) / 1e9 / peak) if n_pack else None,
+              "window_append_avg_us": ms_wapp / n_wapp * 1e3 if n_wapp else None,
+              "input_bytes_per_block": block_in_bytes}
+
     if rank == 0:
         nsq = nsw = None
         rc, nsq, nsw = xq.xq_split_plan(cache.handle, 0)
@@ -340,9 +370,12 @@ def main():
                     "ms_per_step": ms3_max / K},
             "roofline": {"bound": "hbm", "kernel": "decode split kernel", "achieved": achieved, "peak": peak,
                          "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                         "frac_of_8TBps": achieved / 8000.0, "traffic": None,
+                         "frac_of_8TBps": achieved / 8000.0,
+                         "traffic": NCU_TRAFFIC_BYTES.get(args.config) if not (args.layers or args.seq or args.splits) else None,
+                         "algorithmic_bytes_per_launch": bytes_pass2 / dec["launches"] if dec["launches"] else None,
                          "avg_launch_us": dec["avg_us"], "launches": dec["launches"]},
             "kernels": kinds,
+            "append": append,
         }
         if not args.no_cpu_baseline and world == 1:
             n_streams = min(B * Hkv, 32)
