@@ -11,6 +11,7 @@
 
 #include "../../include/xq.h"
 #include "xq_internal.h"
+#include "xq_layout.cuh"
 
 using namespace xq;
 
@@ -422,7 +423,11 @@ int xq_append_kv(xq_cache* c, int layer, const void* K, const void* V, int n_tok
     p.own_k = owns_codes(layer, c->cfg.km); p.own_v = owns_codes(layer, c->cfg.vm);
     p.eta_k = L.bk == 1 ? c->cfg.eta1 : c->cfg.eta2;
     p.eta_v = L.bv == 1 ? c->cfg.eta1 : c->cfg.eta2;
-    p.tb = (dm.R % 64 == 0) ? 64 : 32;  // g = 64 implies R % 64 == 0
+    // tokens per CTA: whole key groups and whole code tiles of both kinds; the
+    // configuration check makes the window a multiple of 64 whenever this is 64
+    p.tb = dm.g > 32 ? dm.g : 32;
+    if (tokens_per_code_tile(L.bk, dm.D) > p.tb) p.tb = tokens_per_code_tile(L.bk, dm.D);
+    if (tokens_per_code_tile(L.bv, dm.D) > p.tb) p.tb = tokens_per_code_tile(L.bv, dm.D);
     cudaError_t e;
     {
       Timer t(c, st, 2);
