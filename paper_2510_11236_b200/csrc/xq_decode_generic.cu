@@ -40,13 +40,15 @@ __global__ void __launch_bounds__(GEN_WARPS * 32) decode_generic_kernel(DecodePa
   int t0, t1;
   if (quant) {
     int units = p.n_q / 32;
-    t0 = (int)(((long long)split * units) / p.ns_q) * 32;
-    t1 = (int)(((long long)(split + 1) * units) / p.ns_q) * 32;
+    share_of(units, p.ns_q, split, t0, t1);
+    t0 *= 32;
+    t1 *= 32;
   } else {
     int sw = split - p.ns_q;
     int tiles = (p.r + 15) / 16;
-    t0 = (int)(((long long)sw * tiles) / p.ns_w) * 16;
-    t1 = min((int)(((long long)(sw + 1) * tiles) / p.ns_w) * 16, p.r);
+    share_of(tiles, p.ns_w, sw, t0, t1);
+    t0 *= 16;
+    t1 = min(t1 * 16, p.r);
   }
 
   const int bk = p.L.bk, bv = p.L.bv;

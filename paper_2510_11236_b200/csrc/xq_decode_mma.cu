@@ -599,10 +599,14 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   const int G = dm.G;
 
   if (p.ns_q == 0) {  // nothing is quantized yet: window-only splits
+    grid_dependents_go();
+    grid_dependency_wait();
     const int ns = p.ns_w;
     const int tiles = (p.r + 15) / 16;
-    const int t0 = (int)(((long long)split * tiles) / ns) * 16;
-    const int t1 = min((int)(((long long)(split + 1) * tiles) / ns) * 16, p.r);
+    int t0, t1;
+    share_of(tiles, ns, split, t0, t1);
+    t0 *= 16;
+    t1 = min(t1 * 16, p.r);
     WindowRegs wr;
     window_preload(p, t0, t1, hk, b, wr);
     window_tokens(p, t0, t1, hk, b, ws, wr);
@@ -614,8 +618,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
 
   const int ns = p.ns_q;
   const int units = p.n_q / 32;
-  const int u0 = (int)(((long long)split * units) / ns);
-  const int u1 = (int)(((long long)(split + 1) * units) / ns);
+  int u0, u1;
+  share_of(units, ns, split, u0, u1);
   const int n_cta = u1 - u0;
   const int uw = u0 + (warp * n_cta) / MMA_WARPS;  // this warp's units: [uw, uw + n_my)
   const int n_my = u0 + ((warp + 1) * n_cta) / MMA_WARPS - uw;
@@ -661,9 +665,31 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
       if (i * 512 + lane * 16 < bytes) cp_async16(zbuf + i * 512 + lane * 16, src + i * 512);
   };
 
-  // Loads the prologue waits for go out first: q in B-operand order, q and the first rows of this split's
-  // share of the window.  Then the packed stream's copies are queued behind them.
-  const int wt0 = (int)(((long long)split * p.r) / ns), wt1 = (int)(((long long)(split + 1) * p.r) / ns);
+  // The first units of the packed streams may be on their way while the preceding kernel in the stream (which
+  // wrote q and the newest window rows, and whose predecessors may still use the split-K scratch) is finishing:
+  // with early_fetch the whole ring is queued before this kernel waits for that one (groups 0, 1, 2 = units 0, 1,
+  // 2; the window tile gets a group of its own).  Without it, group 0 holds unit 0, the first zero-point rows and
+  // the window tile, and the rest of the ring follows once q is here: a launch-wide burst of three units per warp
+  // would sit in the memory queues in front of the q loads.
+  const bool early = p.early_fetch != 0;
+  grid_dependents_go();
+  if (!early) grid_dependency_wait();
+  issue_unit(0, 0);
+  if (n_my > 0) issue_zero_rows(0);
+  if (early) {
+    cp_async_commit();
+#pragma unroll
+    for (int jj = 1; jj < NST - 1; ++jj) {
+      issue_unit(jj, jj * St::BYTES);
+      cp_async_commit();
+    }
+    grid_dependency_wait();
+  }
+
+  // Loads the prologue waits for go out next: q in B-operand order and the first rows of this split's share of
+  // the window.
+  int wt0, wt1;
+  share_of(p.r, ns, split, wt0, wt1);
   uint32_t raw[16];  // q of head gid: (q[16s + 2tig + 8j], q[16s + 2tig + 8j + 1]), j = 0, 1
   {
     const bool real = gid < G;
@@ -676,13 +702,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   const uint32_t wbuf = sm_base + PIPE + Q_BYTES;
   if (warp == ww && wt0 < wt1) window_stage(p, wt0, wt1, hk, b, wbuf, lane);
 
-  // start the pipeline (group jj holds unit jj; group 0 also the first zero-point rows and the first window tile)
-#pragma unroll
-  for (int jj = 0; jj < NST - 1; ++jj) {
-    issue_unit(jj, jj * St::BYTES);
-    if (jj == 0 && n_my > 0) issue_zero_rows(0);
-    cp_async_commit();
-  }
+  cp_async_commit();  // group 0, or the window tile's group (empty for the other warps)
 
   uint32_t qe[16];  // q as fp16 B operand, pre-scaled by 2^-e(s), the weight the code's slot carries
 #pragma unroll
@@ -696,6 +716,13 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     }
   }
   __syncthreads();
+  if (!early) {  // q is here: the rest of the ring (group jj holds unit jj)
+#pragma unroll
+    for (int jj = 1; jj < NST - 1; ++jj) {
+      issue_unit(jj, jj * St::BYTES);
+      cp_async_commit();
+    }
+  }
 
   const float scale2 = p.scale * 1.4426950408889634f;
   const float c1 = scale2 * 16777216.0f;  // undoes the 2^-24 of the subnormal code operand
@@ -708,7 +735,13 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;  // softmax reference (log2 units) of heads 2 tig, 2 tig + 1
   float accS[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 
-  cp_async_wait<NST - 2>();  // unit 0, the first zero-point rows and the first window tile have landed
+  // unit 0, the first zero-point rows and (for its warp) the first window tile have landed
+  if (!early)
+    cp_async_wait<NST - 2>();
+  else if (warp == ww && wt0 < wt1)
+    cp_async_wait<0>();
+  else
+    cp_async_wait<NST - 1>();
   __syncwarp();
   if (warp == ww && wt0 < wt1) {
     // window tokens first (the accumulators are empty): true units, then the slot weights of the packed path
@@ -862,8 +895,7 @@ cudaError_t launch_t(const DecodeParams& p, cudaStream_t st) {
   }
   const int ns = p.ns_q > 0 ? p.ns_q : p.ns_w;
   dim3 grid(ns, p.dm.Hkv, p.dm.B);
-  decode_mma_kernel<BK, BV, GS><<<grid, MMA_THREADS, smem, st>>>(p);
-  return cudaGetLastError();
+  return launch_dependent(decode_mma_kernel<BK, BV, GS>, grid, dim3(MMA_THREADS), (size_t)smem, st, p);
 }
 
 template <int BK, int BV, int GS>

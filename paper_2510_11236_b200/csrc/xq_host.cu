@@ -143,6 +143,7 @@ struct xq_cache {
   float scale;
   int sm_count;
   bool tickets_clean;  // the ticket counters have been zeroed on a stream
+  std::vector<uint8_t> repacked;  // per layer: codes or parameters it reads were written since its last decode
   int mma_ctas[2][2];  // resident CTAs per SM of the tensor-core kernel by (key bits - 1, value bits - 1); 0 = not asked yet
   // timing
   bool timing;
@@ -295,6 +296,7 @@ int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, c
     if (nqo < nq) return XQ_ERR_ORDER;
   }
   DecodeParams p;
+  p.early_fetch = 0;
   p.dm = dm;
   p.L = layer_ptrs(c, layer);
   p.q = (const uint16_t*)q;
@@ -316,6 +318,10 @@ int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, c
       if (e != cudaSuccess) return fail_cuda(c, e);
       c->tickets_clean = true;
     }
+    // the packed streams may be fetched ahead of the preceding kernel unless a pack kernel wrote them since
+    // this layer's last decode (then that kernel may be the writer, or only just behind it)
+    p.early_fetch = c->repacked[layer] ? 0 : 1;
+    c->repacked[layer] = 0;
     {
       Timer t(c, st, 0);
       e = launch_decode_mma(p, st);  // merges the partials itself
@@ -371,6 +377,7 @@ int xq_create(const xq_config* cfg, void* dev_workspace, size_t bytes, xq_cache*
   if (bytes < c->plan.total) { delete c; return XQ_ERR_CAPACITY; }
   c->ws = (uint8_t*)dev_workspace;
   c->seq.assign(cfg->n_layers, 0);
+  c->repacked.assign(cfg->n_layers, 1);
   c->launches = 0;
   c->last_cuda = 0;
   c->scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.0f / sqrtf((float)cfg->head_dim);
@@ -435,6 +442,8 @@ int xq_append_kv(xq_cache* c, int layer, const void* K, const void* V, int n_tok
     }
     c->launches++;
     if (e != cudaSuccess) return fail_cuda(c, e);
+    c->repacked[layer] = 1;
+    if (layer + 1 < c->cfg.n_layers) c->repacked[layer + 1] = 1;  // it may read this layer's codes
   }
   {
     WindowParams w;
@@ -480,6 +489,7 @@ int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out,
   const bool use_mma = layer_uses_mma(c, layer);
   if (c->cfg.kernel == XQ_KERNEL_MMA && !use_mma) return XQ_ERR_CONFIG;
   DecodeParams p;
+  p.early_fetch = 0;
   p.dm = dm;
   p.L = layer_ptrs(c, layer);
   p.q = (const uint16_t*)q;

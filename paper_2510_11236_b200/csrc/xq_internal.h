@@ -61,6 +61,9 @@ struct DecodeParams {
   void* out;              // [B,Hq,D] bf16 or f32
   int out_f32;
   unsigned int* tickets;  // [B*Hkv], zero between launches
+  // 1: the packed streams were complete before the preceding kernel in the stream started, so their first
+  // copies may be issued before this kernel has waited for that kernel (programmatic dependent launch)
+  int early_fetch;
 };
 
 struct MergeParams {
@@ -71,6 +74,38 @@ struct MergeParams {
   void* out;
   int out_f32;
 };
+
+// Part `part` of `parts` nearly equal shares of n items: [lo, hi), sizes differ by at most one.
+// (32-bit arithmetic: a 64-bit division costs a device thread hundreds of instructions.)
+__host__ __device__ inline void share_of(int n, int parts, int part, int& lo, int& hi) {
+  const unsigned base = (unsigned)n / (unsigned)parts, rem = (unsigned)n - base * (unsigned)parts;
+  lo = (int)((unsigned)part * base + ((unsigned)part < rem ? (unsigned)part : rem));
+  hi = lo + (int)base + ((unsigned)part < rem ? 1 : 0);
+}
+
+// Programmatic dependent launch (sm_90 and later).  A kernel launched with launch_dependent() may start while
+// the preceding kernel in the stream is still running, provided that kernel has called grid_dependents_go() (or
+// when it ends); it must call grid_dependency_wait() before it touches anything the preceding kernels wrote or
+// still read.  After the wait all earlier work in the stream is complete and visible, as at a kernel boundary.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void grid_dependents_go() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
+template <typename P>
+cudaError_t launch_dependent(void (*kernel)(P), dim3 grid, dim3 block, size_t smem, cudaStream_t st, const P& params) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, params);
+}
+#endif
 
 cudaError_t launch_pack(const PackParams& p, cudaStream_t st);
 cudaError_t launch_window_append(const WindowParams& p, cudaStream_t st);

@@ -274,6 +274,8 @@ __global__ void __launch_bounds__(256) window_append_kernel(WindowParams p) {
   const int vec_per_row = dm.D / 8;
   const size_t per_kind = (size_t)dm.B * dm.Hkv * p.count * vec_per_row;
   size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  grid_dependents_go();    // the next kernel may get its CTAs placed; it waits for this one before it reads the window
+  grid_dependency_wait();  // the inputs come from the preceding kernel, and earlier kernels may still read the window
   if (idx >= 2 * per_kind) return;
   int kind = idx >= per_kind;
   size_t r = idx - (kind ? per_kind : 0);
@@ -292,8 +294,7 @@ __global__ void __launch_bounds__(256) window_append_kernel(WindowParams p) {
 cudaError_t launch_window_append(const WindowParams& p, cudaStream_t st) {
   size_t total = 2 * (size_t)p.dm.B * p.dm.Hkv * p.count * (p.dm.D / 8);
   unsigned blocks = (unsigned)((total + 255) / 256);
-  window_append_kernel<<<blocks, 256, 0, st>>>(p);
-  return cudaGetLastError();
+  return launch_dependent(window_append_kernel, dim3(blocks), dim3(256), 0, st, p);
 }
 
 }  // namespace xq
