@@ -328,13 +328,29 @@ __device__ __forceinline__ void window_stage(const DecodeParams& p, int tb, int 
     const uint32_t dk = wbuf + row * WROW + c * 16, dv = dk + 16 * WROW;
     if (tb + row < t1) {
       const size_t off = (row0 + tb + row) * (2 * HD) + c * 16;
-      cp_async16(dk, wk + off);
-      cp_async16(dv, wv + off);
+      if (p.K_new != nullptr && tb + row == p.r - 1) {  // the token of this step: not in the window yet
+        const size_t noff = (size_t)(b * dm.Hkv + hk) * (2 * HD) + c * 16;
+        cp_async16(dk, reinterpret_cast<const uint8_t*>(p.K_new) + noff);
+        cp_async16(dv, reinterpret_cast<const uint8_t*>(p.V_new) + noff);
+      } else {
+        cp_async16(dk, wk + off);
+        cp_async16(dv, wv + off);
+      }
     } else {
       asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};\n" ::"r"(dk), "r"(0u) : "memory");
       asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};\n" ::"r"(dv), "r"(0u) : "memory");
     }
   }
+}
+
+// Fused append: the staged tile [tb, tb + 16) holds the token of this step (row r - 1); one warp stores it into
+// the window, keys by lanes 0..15, values by lanes 16..31.
+__device__ __forceinline__ void window_store_new(const DecodeParams& p, int tb, int hk, int b, uint32_t wbuf, int lane) {
+  const Dims& dm = p.dm;
+  const int row = p.r - 1 - tb, c = lane & 15;
+  const uint4 v = lds128(wbuf + (lane >> 4) * 16 * WROW + row * WROW + c * 16);
+  uint8_t* win = reinterpret_cast<uint8_t*>(lane < 16 ? p.L.win_k : p.L.win_v);
+  *reinterpret_cast<uint4*>(win + ((size_t)(b * dm.Hkv + hk) * dm.R + (p.r - 1)) * (2 * HD) + c * 16) = v;
 }
 
 // One warp folds the staged tile (n_valid of its 16 tokens exist) into its softmax state.  accO is kept in true
@@ -753,6 +769,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
         cp_async_wait<0>();
         __syncwarp();
       }
+      if (p.K_new != nullptr && tb + 16 > p.r - 1 && wt1 == p.r) window_store_new(p, tb, hk, b, wbuf, lane);
       window_tile(wbuf, wt1 - tb, raw, scale2, accO, accZ, m0, m1, lane);
     }
 #pragma unroll

@@ -280,7 +280,10 @@ struct Timer {
 
 int fail_cuda(xq_cache* c, cudaError_t e) { c->last_cuda = (int)e; return XQ_ERR_CUDA; }
 
-int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, cudaStream_t st) {
+// K_new / V_new: one new token per stream that the tensor-core kernel appends itself (see append_fuses); the
+// layer's length already counts it.
+int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, cudaStream_t st,
+                const void* K_new = nullptr, const void* V_new = nullptr) {
   if (!c || !q || !out) return XQ_ERR_ARG;
   if (layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
   if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return XQ_ERR_ARG;
@@ -297,6 +300,7 @@ int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, c
   }
   DecodeParams p;
   p.early_fetch = 0;
+  p.K_new = p.V_new = nullptr;
   p.dm = dm;
   p.L = layer_ptrs(c, layer);
   p.q = (const uint16_t*)q;
@@ -311,6 +315,9 @@ int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, c
   p.out = out;
   p.out_f32 = out_f32;
   p.tickets = (unsigned int*)(c->ws + c->plan.tickets);
+  p.K_new = (const uint16_t*)K_new;
+  p.V_new = (const uint16_t*)V_new;
+  if (K_new && !(use_mma && nq > 0)) return XQ_ERR_ARG;
   cudaError_t e;
   if (use_mma) {
     if (!c->tickets_clean) {
@@ -490,6 +497,7 @@ int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out,
   if (c->cfg.kernel == XQ_KERNEL_MMA && !use_mma) return XQ_ERR_CONFIG;
   DecodeParams p;
   p.early_fetch = 0;
+  p.K_new = p.V_new = nullptr;
   p.dm = dm;
   p.L = layer_ptrs(c, layer);
   p.q = (const uint16_t*)q;
@@ -580,9 +588,20 @@ int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void
   }
   for (int i = 0; i < L; ++i) {
     const int l = layer_order ? layer_order[i] : i;
-    int rc = xq_append_kv(c, l, dk + l * kv_layer, dv + l * kv_layer, 1, stream);
-    if (rc != XQ_OK) return rc;
-    rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st);
+    // One token that neither fills a window block nor is the layer's first quantized step goes into the window
+    // inside the tensor-core decode kernel; every other case appends with its own kernels first.
+    const int s_old = c->seq[l];
+    const int nq_old = s_old - residual_count(s_old, dm.R), nq_new = s_old + 1 - residual_count(s_old + 1, dm.R);
+    int rc;
+    if (nq_new == nq_old && nq_old > 0 && layer_uses_mma(c, l)) {
+      c->seq[l] = s_old + 1;
+      rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st, dk + l * kv_layer, dv + l * kv_layer);
+      if (rc != XQ_OK) c->seq[l] = s_old;
+    } else {
+      rc = xq_append_kv(c, l, dk + l * kv_layer, dv + l * kv_layer, 1, stream);
+      if (rc != XQ_OK) return rc;
+      rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st);
+    }
     if (rc != XQ_OK) return rc;
   }
   if (mem == XQ_MEM_HOST) {

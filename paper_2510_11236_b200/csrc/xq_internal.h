@@ -64,6 +64,11 @@ struct DecodeParams {
   // 1: the packed streams were complete before the preceding kernel in the stream started, so their first
   // copies may be issued before this kernel has waited for that kernel (programmatic dependent launch)
   int early_fetch;
+  // Fused append of one token per stream (tensor-core kernel with quantized tokens only; else null): the newest
+  // window row, index r - 1, is not in the window yet but here, [B,Hkv,D] bf16.  The CTA whose share of the
+  // window holds that row reads it from here and stores it into the window.
+  const uint16_t* K_new;
+  const uint16_t* V_new;
 };
 
 struct MergeParams {

@@ -185,6 +185,54 @@ def test_decode_step_device_and_host():
     assert xq.xq_launch_count(a.handle) > 0
 
 
+def test_decode_step_appends_inside_the_decode_kernel():
+    """Steps of one token on the tensor-core kernel's shape: the token goes into the window inside the decode
+    kernel except on the steps that quantize a full window first.  Every step's output equals, bit for bit, what
+    xq_decode_attention returns afterwards (the kernels that append first); after every few steps the windows,
+    codes, scales and zero-points equal the oracle's bit for bit and the attention is close to the oracle's.
+
+    Tolerance: at ~100 tokens with key outlier channels ten times the rest, one or two tokens carry the softmax,
+    so the result follows the logits' error instead of averaging it away as it does over the benchmark's
+    contexts.  The kernel rounds q_d * s_d to fp16 (relative 2^-12) before the tensor-core product; a channel
+    whose codes span 60 units of q_d s_d / sqrt(D) moves a logit by up to 2e-3, three such channels by 6e-3, and
+    a two-token softmax hands a quarter of that, times the distance of two value rows (~4), to the output."""
+    short_context_tol = 6e-3
+    L, B, Hq, Hkv, D, R = 2, 2, 8, 2, 128, 32
+    w = dict(n_layers=L, batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, seq=70, residual_len=R,
+             group_size=32, kq=2, vq=0, km=0, vm=0, n_outliers=3, outlier_scale=10.0, seed=5, n_splits=0)
+    cfg = W.make_xq_config(w, max_seq=256)
+    cache = xq.Cache(cfg, DEV)
+    kv = _fill(cache, w, [0, 1], 70)
+    gen = torch.Generator(device="cpu").manual_seed(17)
+    launches = xq.xq_launch_count(cache.handle)
+    for step in range(62):  # lengths 71 .. 132: flushes at 97 and 129
+        kn = torch.randn(L, B, Hkv, 1, D, generator=gen).to(torch.bfloat16).to(DEV)
+        vn = torch.randn(L, B, Hkv, 1, D, generator=gen).to(torch.bfloat16).to(DEV)
+        q = torch.randn(L, B, Hq, D, generator=gen).to(torch.bfloat16).to(DEV)
+        out = torch.empty_like(q)
+        cache.decode_step(kn, vn, q, out)
+        torch.cuda.synchronize()
+        S = 71 + step
+        flush = (S - 1) % R == 0
+        now = xq.xq_launch_count(cache.handle)
+        assert now - launches == (L * 3 if flush else L)  # pack + window append + decode, or the decode alone
+        launches = now
+        for l in range(L):
+            kv[l] = (torch.cat([kv[l][0], kn[l]], dim=2), torch.cat([kv[l][1], vn[l]], dim=2))
+            assert cache.seq_len(l) == S
+            assert torch.equal(out[l], cache.decode_attention(l, q[l]))
+        launches = xq.xq_launch_count(cache.handle)
+        if step % 7 == 0 or flush or step == 61:
+            o32 = [cache.decode_attention(l, q[l], f32=True) for l in range(L)]
+            launches = xq.xq_launch_count(cache.handle)
+            for b in range(B):
+                for hk in range(Hkv):
+                    oc = util.oracle_for_stream(cfg, [0, 1], b, hk, kv)
+                    for l in range(L):
+                        util.compare_regions(cache, oc, l, b, hk)
+                        util.check_attention(cache, oc, l, q[l], b, hk, o32[l], None, tol=short_context_tol)
+
+
 @pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4"])
 def test_full_size_configs_sampled(name):
     """The benchmark's shapes and launch configuration (library-chosen splits, tensor-core kernel), one layer
