@@ -473,20 +473,37 @@ __device__ __forceinline__ void ticket_merge(const DecodeParams& p, int ns, int 
     const size_t hq = (size_t)b * dm.Hq + hk * dm.G + a;
     const float* ml = p.part_ml + hq * ns * 2;
     const float* pa = p.part_acc + hq * ns * HD + lane * 4;
+    // every load of a round is issued before anything waits for one: the merge costs one L2 round trip per 16
+    // partials instead of one per partial
+    float4 v[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = (i < ns) ? ld_cg4(pa + (size_t)i * HD) : make_float4(0.f, 0.f, 0.f, 0.f);
     float M = -CUDART_INF_F;
     for (int s = lane; s < ns; s += 32) M = fmaxf(M, ld_cg(ml + 2 * s));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float Ls = 0.f;
-#pragma unroll 4
-    for (int s = 0; s < ns; ++s) {
-      float f = ex2(ld_cg(ml + 2 * s) - M);
-      Ls = fmaf(ld_cg(ml + 2 * s + 1), f, Ls);
-      float4 v = ld_cg4(pa + (size_t)s * HD);
-      acc.x = fmaf(v.x, f, acc.x); acc.y = fmaf(v.y, f, acc.y);
-      acc.z = fmaf(v.z, f, acc.z); acc.w = fmaf(v.w, f, acc.w);
+    for (int s0 = 0; s0 < ns; s0 += 16) {
+      if (s0 > 0) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          v[i] = (s0 + i < ns) ? ld_cg4(pa + (size_t)(s0 + i) * HD) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      float f = 0.f;  // lane i < 16: weight of partial s0 + i
+      if (lane < 16 && s0 + lane < ns) {
+        f = ex2(ld_cg(ml + 2 * (s0 + lane)) - M);
+        Ls = fmaf(ld_cg(ml + 2 * (s0 + lane) + 1), f, Ls);
+      }
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const float fi = __shfl_sync(0xffffffffu, f, i);
+        acc.x = fmaf(v[i].x, fi, acc.x); acc.y = fmaf(v[i].y, fi, acc.y);
+        acc.z = fmaf(v[i].z, fi, acc.z); acc.w = fmaf(v[i].w, fi, acc.w);
+      }
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) Ls += __shfl_xor_sync(0xffffffffu, Ls, o);
     const float inv = 1.0f / Ls;
     acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
     if (p.out_f32) {
