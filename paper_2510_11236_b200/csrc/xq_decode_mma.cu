@@ -356,6 +356,7 @@ __device__ __forceinline__ void window_store_new(const DecodeParams& p, int tb, 
 // One warp folds the staged tile (n_valid of its 16 tokens exist) into its softmax state.  accO is kept in true
 // units here (the caller applies the slot weights of the packed path once all window tiles are in).
 // qb: q of head gid as bf16 pairs in B-operand order (as loaded), scale2: softmax scale in log2 units.
+template <bool SP>
 __device__ __forceinline__ void window_tile(uint32_t wbuf, int n_valid, const uint32_t (&qb)[16], float scale2,
                                             float (&accO)[8][4], float (&accZ)[4], float& m0, float& m1, int lane) {
   const int gid = lane >> 2;
@@ -368,23 +369,27 @@ __device__ __forceinline__ void window_tile(uint32_t wbuf, int n_valid, const ui
     mma16816_bf16(s, a0, a1, a2, a3, qb[2 * ks], qb[2 * ks + 1]);
   }
   const bool va = gid < n_valid, vb = gid + 8 < n_valid;
-  const float x00 = va ? s[0] * scale2 : -CUDART_INF_F, x01 = va ? s[1] * scale2 : -CUDART_INF_F;
-  const float x10 = vb ? s[2] * scale2 : -CUDART_INF_F, x11 = vb ? s[3] * scale2 : -CUDART_INF_F;
+  // SP: the odd columns are padding (q = 0 there): they keep reference 0 and numerators 0
+  const float x00 = va ? s[0] * scale2 : -CUDART_INF_F, x01 = SP ? 0.f : (va ? s[1] * scale2 : -CUDART_INF_F);
+  const float x10 = vb ? s[2] * scale2 : -CUDART_INF_F, x11 = SP ? 0.f : (vb ? s[3] * scale2 : -CUDART_INF_F);
   float r0 = fmaxf(x00, x10), r1 = fmaxf(x01, x11);
 #pragma unroll
   for (int o = 4; o < 32; o <<= 1) {
     r0 = fmaxf(r0, __shfl_xor_sync(0xffffffffu, r0, o));
-    r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, o));
+    if (!SP) r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, o));
   }
-  const float mn0 = fmaxf(m0, r0), mn1 = fmaxf(m1, r1);  // finite: token 0 of the tile exists
-  const float f0 = ex2(m0 - mn0), f1 = ex2(m1 - mn1);
+  const float mn0 = fmaxf(m0, r0), mn1 = SP ? m1 : fmaxf(m1, r1);  // finite: token 0 of the tile exists
+  const float f0 = ex2(m0 - mn0), f1 = SP ? 1.f : ex2(m1 - mn1);
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
-    accO[mt][0] *= f0; accO[mt][1] *= f1; accO[mt][2] *= f0; accO[mt][3] *= f1;
+    accO[mt][0] *= f0; accO[mt][2] *= f0;
+    if (!SP) { accO[mt][1] *= f1; accO[mt][3] *= f1; }
   }
-  accZ[0] *= f0; accZ[1] *= f1; accZ[2] *= f0; accZ[3] *= f1;
+  accZ[0] *= f0; accZ[2] *= f0;
+  if (!SP) { accZ[1] *= f1; accZ[3] *= f1; }
   m0 = mn0; m1 = mn1;
-  const float p00 = ex2(x00 - m0), p01 = ex2(x01 - m1), p10 = ex2(x10 - m0), p11 = ex2(x11 - m1);
+  const float p00 = ex2(x00 - m0), p10 = ex2(x10 - m0);
+  const float p01 = SP ? 0.f : ex2(x01 - m1), p11 = SP ? 0.f : ex2(x11 - m1);
   // numerators as bf16 hi + lo (16 bits of precision), transposed into B-operand order
   const uint32_t h0 = pack_bf16x2(p00, p01), h1 = pack_bf16x2(p10, p11);
   const uint32_t l0 = pack_bf16x2(p00 - bf16_to_f(h0 & 0xffff), p01 - bf16_to_f(h0 >> 16));
@@ -613,7 +618,9 @@ __device__ __forceinline__ void unit_values(uint32_t st, const uint32_t (&pb)[2]
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
-template <int BK, int BV, int GS>
+// SP ("spread"): groups of at most 4 query heads put head h in column 2h of the N = 8 tiles and leave the odd
+// columns as padding, so that each thread's accumulator pairs hold one real head: half the softmax work.
+template <int BK, int BV, int GS, bool SP>
 __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams p) {
   using St = Stage<BK, BV, GS>;
   constexpr int NG = St::NG;
@@ -725,8 +732,9 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   share_of(p.r, ns, split, wt0, wt1);
   uint32_t raw[16];  // q of head gid: (q[16s + 2tig + 8j], q[16s + 2tig + 8j + 1]), j = 0, 1
   {
-    const bool real = gid < G;
-    const uint16_t* qp = p.q + ((size_t)b * dm.Hq + hk * G + (real ? gid : 0)) * HD + 2 * tig;
+    const int hcol = SP ? (gid >> 1) : gid;  // the head of column gid
+    const bool real = SP ? ((gid & 1) == 0 && hcol < G) : (gid < G);
+    const uint16_t* qp = p.q + ((size_t)b * dm.Hq + hk * G + (real ? hcol : 0)) * HD + 2 * tig;
 #pragma unroll
     for (int i = 0; i < 16; ++i) raw[i] = real ? *reinterpret_cast<const uint32_t*>(qp + 16 * (i >> 1) + 8 * (i & 1)) : 0u;
   }
@@ -765,7 +773,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   for (int mt = 0; mt < 8; ++mt)
 #pragma unroll
     for (int i = 0; i < 4; ++i) accO[mt][i] = 0.f;
-  float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F;  // softmax reference (log2 units) of heads 2 tig, 2 tig + 1
+  // softmax reference (log2 units) of columns 2 tig, 2 tig + 1 (SP: the odd column is padding, reference 0)
+  float m0 = -CUDART_INF_F, m1 = SP ? 0.f : -CUDART_INF_F;
   float accS[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 
   // unit 0, the first zero-point rows and (for its warp) the first window tile have landed
@@ -787,7 +796,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
         __syncwarp();
       }
       if (p.K_new != nullptr && tb + 16 > p.r - 1 && wt1 == p.r) window_store_new(p, tb, hk, b, wbuf, lane);
-      window_tile(wbuf, wt1 - tb, raw, scale2, accO, accZ, m0, m1, lane);
+      window_tile<SP>(wbuf, wt1 - tb, raw, scale2, accO, accZ, m0, m1, lane);
     }
 #pragma unroll
     for (int mt = 0; mt < 8; ++mt) {
@@ -832,21 +841,23 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     const float2 bz = lds64f(ztab + jr * 32 + tig * 8);
     {
       const float lm0 = fmaxf(fmaxf(accS[0][0], accS[0][2]), fmaxf(accS[1][0], accS[1][2]));
-      const float lm1 = fmaxf(fmaxf(accS[0][1], accS[0][3]), fmaxf(accS[1][1], accS[1][3]));
-      float x0 = fmaf(lm0, c1, bz.x), x1 = fmaf(lm1, c1, bz.y);
-      if (__any_sync(0xffffffffu, (x0 > m0 + TAU) | (x1 > m1 + TAU))) {
+      const float lm1 = SP ? 0.f : fmaxf(fmaxf(accS[0][1], accS[0][3]), fmaxf(accS[1][1], accS[1][3]));
+      float x0 = fmaf(lm0, c1, bz.x), x1 = SP ? 0.f : fmaf(lm1, c1, bz.y);
+      if (__any_sync(0xffffffffu, SP ? (x0 > m0 + TAU) : ((x0 > m0 + TAU) | (x1 > m1 + TAU)))) {
 #pragma unroll
         for (int o = 4; o < 32; o <<= 1) {
           x0 = fmaxf(x0, __shfl_xor_sync(0xffffffffu, x0, o));
-          x1 = fmaxf(x1, __shfl_xor_sync(0xffffffffu, x1, o));
+          if (!SP) x1 = fmaxf(x1, __shfl_xor_sync(0xffffffffu, x1, o));
         }
-        const float mn0 = fmaxf(m0, x0), mn1 = fmaxf(m1, x1);
-        const float f0 = ex2(m0 - mn0), f1 = ex2(m1 - mn1);
+        const float mn0 = fmaxf(m0, x0), mn1 = SP ? m1 : fmaxf(m1, x1);
+        const float f0 = ex2(m0 - mn0), f1 = SP ? 1.f : ex2(m1 - mn1);
 #pragma unroll
         for (int mt = 0; mt < 8; ++mt) {
-          accO[mt][0] *= f0; accO[mt][1] *= f1; accO[mt][2] *= f0; accO[mt][3] *= f1;
+          accO[mt][0] *= f0; accO[mt][2] *= f0;
+          if (!SP) { accO[mt][1] *= f1; accO[mt][3] *= f1; }
         }
-        accZ[0] *= f0; accZ[1] *= f1; accZ[2] *= f0; accZ[3] *= f1;
+        accZ[0] *= f0; accZ[2] *= f0;
+        if (!SP) { accZ[1] *= f1; accZ[3] *= f1; }
         m0 = mn0; m1 = mn1;
       }
     }
@@ -859,8 +870,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     uint32_t pb[2][2];
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
-      float p0 = ex2(fmaf(accS[mt][0], c1, t0)), p1 = ex2(fmaf(accS[mt][1], c1, t1));
-      float p2 = ex2(fmaf(accS[mt][2], c1, t0)), p3 = ex2(fmaf(accS[mt][3], c1, t1));
+      float p0 = ex2(fmaf(accS[mt][0], c1, t0)), p1 = SP ? 0.f : ex2(fmaf(accS[mt][1], c1, t1));
+      float p2 = ex2(fmaf(accS[mt][2], c1, t0)), p3 = SP ? 0.f : ex2(fmaf(accS[mt][3], c1, t1));
       pb[mt][0] = movmatrix_trans(pack_half2(p0, p1));
       pb[mt][1] = movmatrix_trans(pack_half2(p2, p3));
     }
@@ -886,23 +897,25 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     const float z0 = __shfl_sync(0xffffffffu, accZ[0], 4 * gi + tig), z1 = __shfl_sync(0xffffffffu, accZ[1], 4 * gi + tig);
     const float wgt = (float)(1u << (24 - Slots<BV>::e(mt)));
     const int ch = 16 * mt + gid;
-    if (2 * tig < G) {
-      float* row = mine + (2 * tig) * MS;
+    const int h0 = SP ? tig : 2 * tig;  // the head of this thread's even column
+    if (h0 < G) {
+      float* row = mine + h0 * MS;
       row[ch] = fmaf(accO[mt][0], wgt, z0);
       row[ch + 8] = fmaf(accO[mt][2], wgt, z0);
     }
-    if (2 * tig + 1 < G) {
+    if (!SP && 2 * tig + 1 < G) {
       float* row = mine + (2 * tig + 1) * MS;
       row[ch] = fmaf(accO[mt][1], wgt, z1);
       row[ch + 8] = fmaf(accO[mt][3], wgt, z1);
     }
   }
   if (gid == 0) {
-    if (2 * tig < G) {
-      mine[(2 * tig) * MS + HD] = m0;
-      mine[(2 * tig) * MS + HD + 1] = l0;
+    const int h0 = SP ? tig : 2 * tig;
+    if (h0 < G) {
+      mine[h0 * MS + HD] = m0;
+      mine[h0 * MS + HD + 1] = l0;
     }
-    if (2 * tig + 1 < G) {
+    if (!SP && 2 * tig + 1 < G) {
       mine[(2 * tig + 1) * MS + HD] = m1;
       mine[(2 * tig + 1) * MS + HD + 1] = l1;
     }
@@ -918,34 +931,45 @@ int smem_bytes(int G) {
   return pipe_bytes<BK, BV, GS>() + Q_BYTES + WIN_BYTES;
 }
 
-template <int BK, int BV, int GS>
-cudaError_t launch_t(const DecodeParams& p, cudaStream_t st) {
+template <int BK, int BV, int GS, bool SP>
+cudaError_t launch_sp(const DecodeParams& p, cudaStream_t st) {
   const int smem = smem_bytes<BK, BV, GS>(p.dm.G);
   static int configured = 0;
   if (configured < smem) {
-    cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<BK, BV, GS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<BK, BV, GS, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     configured = smem;
   }
   const int ns = p.ns_q > 0 ? p.ns_q : p.ns_w;
   dim3 grid(ns, p.dm.Hkv, p.dm.B);
-  return launch_dependent(decode_mma_kernel<BK, BV, GS>, grid, dim3(MMA_THREADS), (size_t)smem, st, p);
+  return launch_dependent(decode_mma_kernel<BK, BV, GS, SP>, grid, dim3(MMA_THREADS), (size_t)smem, st, p);
 }
 
 template <int BK, int BV, int GS>
-int ctas_per_sm_t(int G) {
+cudaError_t launch_t(const DecodeParams& p, cudaStream_t st) {
+  return p.dm.G <= 4 ? launch_sp<BK, BV, GS, true>(p, st) : launch_sp<BK, BV, GS, false>(p, st);
+}
+
+template <int BK, int BV, int GS, bool SP>
+int ctas_per_sm_sp(int G) {
   const int smem = smem_bytes<BK, BV, GS>(G);
-  if (cudaFuncSetAttribute(decode_mma_kernel<BK, BV, GS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+  if (cudaFuncSetAttribute(decode_mma_kernel<BK, BV, GS, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
       cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
   int n = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_mma_kernel<BK, BV, GS>, MMA_THREADS, smem) != cudaSuccess) {
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_mma_kernel<BK, BV, GS, SP>, MMA_THREADS, smem) !=
+      cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
   return n;
+}
+
+template <int BK, int BV, int GS>
+int ctas_per_sm_t(int G) {
+  return G <= 4 ? ctas_per_sm_sp<BK, BV, GS, true>(G) : ctas_per_sm_sp<BK, BV, GS, false>(G);
 }
 
 }  // namespace
