@@ -25,6 +25,12 @@
  *     synchronizes the device, except where a function says otherwise.  All
  *     kernels are launched asynchronously on the given stream
  *     (a cudaStream_t passed as void*; NULL is the default stream).
+ *     The decode and window-append kernels are launched as programmatic
+ *     dependents: their thread blocks may be placed, and packed cache data that
+ *     earlier calls completed may be fetched, while the preceding kernel in the
+ *     stream is still running; they wait for that kernel to complete before
+ *     they touch q, new tokens, the window, the split scratch or any output, so
+ *     stream order holds for everything a caller can observe.
  *   - Every function returns XQ_OK (0) or a negative XQ_ERR_* code; a failing
  *     call leaves the cache unchanged.  Nothing is thrown across the boundary.
  *   - A cache handle is not thread-safe; use one host thread per handle.
@@ -167,7 +173,12 @@ int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out,
  * mem = XQ_MEM_HOST: host pointers (pinned memory for the copies to be
  * asynchronous); inputs are copied to the workspace's staging area on `stream`,
  * the result is copied back to `out` on `stream`; the caller synchronizes the
- * stream before reading `out` or reusing the host buffers. */
+ * stream before reading `out` or reusing the host buffers.
+ * The result equals xq_append_kv followed by xq_decode_attention per layer, bit
+ * for bit; where the tensor-core kernel serves the layer and the token fills no
+ * window block, that kernel stores the token into the window itself (one launch
+ * per layer).  K_new and V_new must stay unchanged until the step's kernels
+ * have run. */
 int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void* q, void* out,
                    const int32_t* layer_order, int mem, void* stream);
 
