@@ -1,5 +1,5 @@
 // Quantize-and-pack of residual-window blocks (Eq. 1, 2, 12; Algorithm 2) and
-// the window append.  One CTA quantizes a tile of `tb` tokens x D channels of
+// the window append.  One CTA quantizes a tile of T (32 or 64) tokens x D channels of
 // one (sequence, kv head) for keys or for values.
 //
 // The fp32 arithmetic uses the *_rn intrinsics so that no multiply-add is ever
@@ -39,52 +39,49 @@ __device__ __forceinline__ uint32_t code_of(float x, float z, float s, float qma
 }
 
 constexpr int PACK_THREADS = 128;
-constexpr int PACK_MAX_TB = 64;
 constexpr int PACK_ROW_PAD = 16;  // bytes added to each staged row: 8 consecutive rows then fall in 8 different bank groups
+constexpr float PACK_MAGIC = 12582912.0f;  // 1.5 * 2^23: x + MAGIC has rint(x) in its low mantissa bits for |x| < 2^22
 
-// The quantizer's parameters of one group as the code loop wants them.
-struct GroupPar {
-  float z, s, inv, unused;  // inv = 1/s rounded to nearest (0 for a constant group)
-};
+__device__ __forceinline__ float rcp_or_zero(float s) { return (s == 0.0f) ? 0.0f : __frcp_rn(s); }
 
-__device__ __forceinline__ GroupPar make_par(float z, float s) {
-  GroupPar r;
-  r.z = z;
-  r.s = s;
-  r.inv = (s == 0.0f) ? 0.0f : __frcp_rn(s);
-  r.unused = 0.0f;
-  return r;
+// Eq. 2 for two elements through the reciprocals.  (x - z) * inv differs from the correctly rounded quotient
+// (x - z) / s by at most three roundings of a value below 2^B, i.e. by less than 6e-7, so both round to the same
+// integer unless the product lies within 1e-5 of a tie; `doubt` collects that case (and any non-finite product
+// of a subnormal scale), and the caller then recomputes the word with the division.  The fused multiply-add
+// with MAGIC rounds the exact product to the nearest integer, ties to even, and leaves it in the low mantissa
+// bits; 0 <= (x - z) / s < 2^B - 1/2 holds for every member of the group, so this path needs no clamp.
+// Returns code(x0) | code(x1) << 16.
+template <int BITS>
+__device__ __forceinline__ uint32_t code_pair(float x0, float x1, float z0, float inv0, float z1, float inv1, bool& doubt) {
+  const float a0 = __fsub_rn(x0, z0), a1 = __fsub_rn(x1, z1);
+  const float u0 = __fmaf_rn(a0, inv0, PACK_MAGIC), u1 = __fmaf_rn(a1, inv1, PACK_MAGIC);
+  const float d0 = __fmaf_rn(a0, inv0, -__fsub_rn(u0, PACK_MAGIC)), d1 = __fmaf_rn(a1, inv1, -__fsub_rn(u1, PACK_MAGIC));
+  doubt |= !(fabsf(d0) <= 0.49999f) | !(fabsf(d1) <= 0.49999f);
+  constexpr uint32_t QM = (1u << BITS) - 1u;
+  return __byte_perm(__float_as_uint(u0), __float_as_uint(u1), 0x0400) & (QM | (QM << 16));
 }
 
-// Eq. 2 through the reciprocal.  (x - z) * inv differs from the correctly
-// rounded quotient (x - z) / s by at most three roundings of a value below
-// 2^B, i.e. by less than 6e-7, so both round to the same integer unless the
-// product lies within 1e-5 of a tie; `doubt` collects that case (and any
-// non-finite product of a subnormal scale), and the caller then recomputes the
-// word with the division.  0 <= (x - z) / s < 2^B - 1/2 holds for every member
-// of the group, so the fast path needs no clamp.
-__device__ __forceinline__ uint32_t code_fast(float x, const GroupPar& g, bool& doubt) {
-  float t = __fmul_rn(__fsub_rn(x, g.z), g.inv);
-  float c = rintf(t);
-  doubt |= !(fabsf(__fsub_rn(t, c)) <= 0.49999f);
-  return (uint32_t)(int)c;
-}
-
-// One CTA: T = p.tb tokens x D channels of one (sequence, kv head), keys
-// (blockIdx.x even) or values (odd).  Staged rows are padded; the statistics
-// and the codes read them without bank conflicts; the packed words are
-// collected in shared memory and leave in 16-byte vectors.
-template <int D, int G>
+// One CTA: T tokens x D channels of one (sequence, kv head), keys (blockIdx.x even) or values (odd).  Staged
+// rows are padded; the statistics and the codes read them without bank conflicts; thread (lane, i) builds word
+// 4 * lane + i of every code tile of the CTA, the words are collected in shared memory and leave in 16-byte
+// vectors.  G: group size; T = p.tb: a multiple of G and of both kinds' tokens per code tile.
+template <int D, int G, int T>
 __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
   constexpr int ROWB = D * 2 + PACK_ROW_PAD;
   constexpr int NG = D / G;
   constexpr int CB = D / 16;
-  __shared__ __align__(16) uint8_t tile[PACK_MAX_TB * ROWB];
-  __shared__ __align__(16) GroupPar par[PACK_MAX_TB * NG > (PACK_MAX_TB / G) * D ? PACK_MAX_TB * NG : (PACK_MAX_TB / G) * D];
-  __shared__ __align__(16) uint32_t wbuf[PACK_MAX_TB * D * 2 / 32];
+  constexpr int NPAR = (T * NG > (T / G) * D) ? T * NG : (T / G) * D;  // groups of the tile, either kind
+  constexpr int KP = PACK_THREADS / ((T / G) * (D / 2));               // token parts of a key group in the statistics
+  static_assert(KP >= 1 && G % KP == 0, "key statistics: 128 threads over (group, channel pair, token part)");
+  __shared__ __align__(16) uint8_t tile[T * ROWB];
+  __shared__ __align__(16) float2 par_zi[NPAR];  // (z, 1/s) of a group; keys: [group][channel], values: [channel group][token]
+  __shared__ float par_s[NPAR];
+  // packed words (at most T * D * 2 / 32); before that, the key statistics' partial (min, max) pairs, two words per thread
+  constexpr int NWBUF = (T * D * 2 / 32) > 2 * PACK_THREADS ? (T * D * 2 / 32) : 2 * PACK_THREADS;
+  __shared__ __align__(16) uint32_t wbuf[NWBUF];
 
   const Dims& dm = p.dm;
-  const int R = dm.R, T = p.tb;
+  const int R = dm.R;
   const int kind = blockIdx.x & 1;  // 0 keys, 1 values
   const int tile_idx = blockIdx.x >> 1;
   const int h = blockIdx.y, b = blockIdx.z;
@@ -96,9 +93,11 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
     const uint16_t* win = kind ? p.L.win_v : p.L.win_k;
     const uint16_t* in = kind ? p.V_in : p.K_in;
     constexpr int VPR = D / 8;
-    for (int idx = tid; idx < T * VPR; idx += PACK_THREADS) {
-      int tl = idx / VPR, c8 = idx % VPR;
-      int pabs = tq0 + tl;
+#pragma unroll
+    for (int k = 0; k < T * VPR / PACK_THREADS; ++k) {
+      const int idx = tid + k * PACK_THREADS;
+      const int tl = idx / VPR, c8 = idx % VPR;
+      const int pabs = tq0 + tl;
       const uint16_t* src = (pabs < p.s_old) ? win + ((size_t)bh * R + (pabs - p.nq_old)) * D
                                              : in + ((size_t)bh * p.n_in + (pabs - p.s_old)) * D;
       *reinterpret_cast<uint4*>(tile + tl * ROWB + c8 * 16) = reinterpret_cast<const uint4*>(src)[c8];
@@ -111,141 +110,161 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
   const int own = kind ? p.own_v : p.own_k;
 
   if (kind == 0) {
-    // keys: one group per (channel, run of G tokens); consecutive threads take consecutive channels
+    // keys: one group per (channel, run of G tokens).  First bf16x2 min / max of a channel pair over a part of the
+    // group's tokens (consecutive threads take consecutive pairs), then one thread per (group, channel).
+    {
+      const int dp = tid % (D / 2), rest = tid / (D / 2);
+      const int gl = rest / KP, part = rest % KP;
+      const uint8_t* col = tile + (gl * G + part * (G / KP)) * ROWB + dp * 4;
+      __nv_bfloat162 mn2 = *reinterpret_cast<const __nv_bfloat162*>(col), mx2 = mn2;
+#pragma unroll
+      for (int j = 1; j < G / KP; ++j) {
+        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(col + j * ROWB);
+        mn2 = __hmin2(mn2, v);
+        mx2 = __hmax2(mx2, v);
+      }
+      wbuf[(rest * (D / 2) + dp) * 2] = *reinterpret_cast<uint32_t*>(&mn2);
+      wbuf[(rest * (D / 2) + dp) * 2 + 1] = *reinterpret_cast<uint32_t*>(&mx2);
+    }
+    __syncthreads();
     __half* meta = reinterpret_cast<__half*>(p.L.k_meta);
     const size_t cap_g = (size_t)(dm.nq_cap / G);
-    for (int item = tid; item < (T / G) * D; item += PACK_THREADS) {
-      int gl = item / D, d = item % D;
-      const uint8_t* col = tile + (gl * G) * ROWB + d * 2;
-      float mn = bf16_bits(*reinterpret_cast<const uint16_t*>(col)), mx = mn;
-#pragma unroll 8
-      for (int j = 1; j < G; ++j) {
-        float x = bf16_bits(*reinterpret_cast<const uint16_t*>(col + j * ROWB));
-        mn = fminf(mn, x);
-        mx = fmaxf(mx, x);
+#pragma unroll
+    for (int k = 0; k < ((T / G) * D + PACK_THREADS - 1) / PACK_THREADS; ++k) {
+      const int item = tid + k * PACK_THREADS;
+      if (item < (T / G) * D) {
+        const int gl = item / D, d = item % D;
+        float mn = 0.f, mx = 0.f;
+#pragma unroll
+        for (int part = 0; part < KP; ++part) {
+          const uint32_t a2 = wbuf[((gl * KP + part) * (D / 2) + d / 2) * 2], b2 = wbuf[((gl * KP + part) * (D / 2) + d / 2) * 2 + 1];
+          const float lo = __uint_as_float((d & 1) ? (a2 & 0xffff0000u) : (a2 << 16));
+          const float hi = __uint_as_float((d & 1) ? (b2 & 0xffff0000u) : (b2 << 16));
+          mn = part == 0 ? lo : fminf(mn, lo);
+          mx = part == 0 ? hi : fmaxf(mx, hi);
+        }
+        float z, sc;
+        __half zh, sh;
+        group_params(mn, mx, bits, eta, z, sc, zh, sh);
+        par_zi[item] = make_float2(z, rcp_or_zero(sc));
+        par_s[item] = sc;
+        const size_t grp = (size_t)bh * 2 * cap_g + (tq0 / G + gl);  // scale plane, then zero-point plane
+        const int pos = k_meta_position(d, D);
+        meta[grp * D + pos] = sh;
+        meta[(grp + cap_g) * D + pos] = zh;
       }
-      float z, s;
-      __half zh, sh;
-      group_params(mn, mx, bits, eta, z, s, zh, sh);
-      par[item] = make_par(z, s);
-      size_t grp = (size_t)bh * 2 * cap_g + (tq0 / G + gl);  // scale plane, then zero-point plane
-      int pos = k_meta_position(d, D);
-      meta[grp * D + pos] = sh;
-      meta[(grp + cap_g) * D + pos] = zh;
     }
   } else {
     // values: one group per (token, run of G channels); consecutive threads take consecutive tokens
     __half* meta = reinterpret_cast<__half*>(p.L.v_meta);
-    for (int item = tid; item < T * NG; item += PACK_THREADS) {
-      int tl = item % T, gi = item / T;
-      const uint4* row = reinterpret_cast<const uint4*>(tile + tl * ROWB + gi * G * 2);
-      __nv_bfloat162 mn2, mx2;
-      {
-        uint4 v = row[0];
-        const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&v);
-        mn2 = __hmin2(__hmin2(e[0], e[1]), __hmin2(e[2], e[3]));
-        mx2 = __hmax2(__hmax2(e[0], e[1]), __hmax2(e[2], e[3]));
-      }
 #pragma unroll
-      for (int j = 1; j < G / 8; ++j) {
-        uint4 v = row[j];
-        const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&v);
-        mn2 = __hmin2(mn2, __hmin2(__hmin2(e[0], e[1]), __hmin2(e[2], e[3])));
-        mx2 = __hmax2(mx2, __hmax2(__hmax2(e[0], e[1]), __hmax2(e[2], e[3])));
+    for (int k = 0; k < (T * NG + PACK_THREADS - 1) / PACK_THREADS; ++k) {
+      const int item = tid + k * PACK_THREADS;
+      if (item < T * NG) {
+        const int tl = item % T, gi = item / T;
+        const uint4* row = reinterpret_cast<const uint4*>(tile + tl * ROWB + gi * G * 2);
+        __nv_bfloat162 mn2, mx2;
+        {
+          uint4 v = row[0];
+          const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&v);
+          mn2 = __hmin2(__hmin2(e[0], e[1]), __hmin2(e[2], e[3]));
+          mx2 = __hmax2(__hmax2(e[0], e[1]), __hmax2(e[2], e[3]));
+        }
+#pragma unroll
+        for (int j = 1; j < G / 8; ++j) {
+          uint4 v = row[j];
+          const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&v);
+          mn2 = __hmin2(mn2, __hmin2(__hmin2(e[0], e[1]), __hmin2(e[2], e[3])));
+          mx2 = __hmax2(mx2, __hmax2(__hmax2(e[0], e[1]), __hmax2(e[2], e[3])));
+        }
+        const float mn = fminf(__low2float(mn2), __high2float(mn2));
+        const float mx = fmaxf(__low2float(mx2), __high2float(mx2));
+        float z, sc;
+        __half zh, sh;
+        group_params(mn, mx, bits, eta, z, sc, zh, sh);
+        par_zi[gi * T + tl] = make_float2(z, rcp_or_zero(sc));
+        par_s[gi * T + tl] = sc;
+        const int tabs = tq0 + tl;
+        const size_t t16 = (size_t)bh * (dm.nq_cap / 16) + tabs / 16;
+        const int pos = v_meta_position(tabs % 16, gi, NG);
+        meta[(t16 * 2 + 0) * (16 * NG) + pos] = sh;
+        meta[(t16 * 2 + 1) * (16 * NG) + pos] = zh;
       }
-      float mn = fminf(__low2float(mn2), __high2float(mn2));
-      float mx = fmaxf(__low2float(mx2), __high2float(mx2));
-      float z, s;
-      __half zh, sh;
-      group_params(mn, mx, bits, eta, z, s, zh, sh);
-      par[tl * NG + gi] = make_par(z, s);
-      int tabs = tq0 + tl;
-      size_t t16 = (size_t)bh * (dm.nq_cap / 16) + tabs / 16;
-      int pos = v_meta_position(tabs % 16, gi, NG);
-      meta[(t16 * 2 + 0) * (16 * NG) + pos] = sh;
-      meta[(t16 * 2 + 1) * (16 * NG) + pos] = zh;
     }
   }
   if (!own) return;  // PseudoQuantize: parameters only
   __syncthreads();
 
-  // codes: thread -> (tile, fragment lane, word of the lane); lanes of a warp
-  // differ in the fragment lane, so they read 8 rows x 4 column pairs (keys)
-  // or 4 token pairs x 8 channels (values) of the padded tile
-  const int n_words = T * D * bits / 32;
+  // codes: thread (lane, i) = word 4 * lane + i of every tile: rows (lane / 4) + 8 (i % 2), columns 2 (lane % 4) +
+  // 8 (i / 2) and the next one of each 16 x 16 block (keys: row = token, column = channel; values: the reverse)
+  const int lane = tid & 31, i = tid >> 5;
+  const int row = (lane >> 2) + 8 * (i & 1), col = 2 * (lane & 3) + 8 * (i >> 1);
   auto build = [&](auto bits_c) {
     constexpr int BITS = decltype(bits_c)::value;
     constexpr int NSLOT = 16 / BITS;
     constexpr int TPT = 16 * (NSLOT / CB);
+    constexpr int NT = T >= TPT ? T / TPT : 1;  // code tiles of the CTA (the host never launches a T below TPT)
     constexpr float QMAX = (float)((1 << BITS) - 1);
-    for (int it = tid; it < n_words; it += PACK_THREADS) {
-      const int lane = it & 31, i = (it >> 5) & 3, tile_l = it >> 7;
-      const int row = (lane >> 2) + 8 * (i & 1);
-      const int col = 2 * (lane & 3) + 8 * (i >> 1);
-      uint32_t word = 0;
-      bool doubt = false;
-      if (kind == 0) {
+    uint32_t word[NT];
+    bool doubt[NT];
 #pragma unroll
-        for (int slot = 0; slot < NSLOT; ++slot) {
-          const int tt = slot / CB, cb = slot % CB;
-          const int tl = tile_l * TPT + tt * 16 + row, d = cb * 16 + col;
-          uint32_t xx = *reinterpret_cast<const uint32_t*>(tile + tl * ROWB + d * 2);
-          const GroupPar* gp = par + ((tile_l * TPT + tt * 16) / G) * D + d;
-          GroupPar g0 = gp[0], g1 = gp[1];
-          uint32_t c0 = code_fast(__uint_as_float(xx << 16), g0, doubt);
-          uint32_t c1 = code_fast(__uint_as_float(xx & 0xffff0000u), g1, doubt);
-          word |= (c0 | (c1 << 16)) << (BITS * slot);
-        }
-        if (doubt) {
-          word = 0;
-#pragma unroll 1
-          for (int slot = 0; slot < NSLOT; ++slot) {
-            const int tt = slot / CB, cb = slot % CB;
-            const int tl = tile_l * TPT + tt * 16 + row, d = cb * 16 + col;
-            uint32_t xx = *reinterpret_cast<const uint32_t*>(tile + tl * ROWB + d * 2);
-            const GroupPar* gp = par + ((tile_l * TPT + tt * 16) / G) * D + d;
-            uint32_t c0 = code_of(__uint_as_float(xx << 16), gp[0].z, gp[0].s, QMAX);
-            uint32_t c1 = code_of(__uint_as_float(xx & 0xffff0000u), gp[1].z, gp[1].s, QMAX);
-            word |= (c0 | (c1 << 16)) << (BITS * slot);
-          }
-        }
-      } else {
+    for (int t = 0; t < NT; ++t) { word[t] = 0u; doubt[t] = false; }
+    if (kind == 0) {
 #pragma unroll
-        for (int slot = 0; slot < NSLOT; ++slot) {
-          const int tt = slot / CB, cb = slot % CB;
-          const int tl = tile_l * TPT + tt * 16 + col, d = cb * 16 + row;
-          const uint8_t* src = tile + tl * ROWB + d * 2;
-          float x0 = bf16_bits(*reinterpret_cast<const uint16_t*>(src));
-          float x1 = bf16_bits(*reinterpret_cast<const uint16_t*>(src + ROWB));
-          const GroupPar* gp = par + tl * NG + (cb * 16) / G;
-          GroupPar g0 = gp[0], g1 = gp[NG];
-          uint32_t c0 = code_fast(x0, g0, doubt);
-          uint32_t c1 = code_fast(x1, g1, doubt);
-          word |= (c0 | (c1 << 16)) << (BITS * slot);
-        }
-        if (doubt) {
-          word = 0;
-#pragma unroll 1
-          for (int slot = 0; slot < NSLOT; ++slot) {
-            const int tt = slot / CB, cb = slot % CB;
-            const int tl = tile_l * TPT + tt * 16 + col, d = cb * 16 + row;
-            const uint8_t* src = tile + tl * ROWB + d * 2;
-            float x0 = bf16_bits(*reinterpret_cast<const uint16_t*>(src));
-            float x1 = bf16_bits(*reinterpret_cast<const uint16_t*>(src + ROWB));
-            const GroupPar* gp = par + tl * NG + (cb * 16) / G;
-            uint32_t c0 = code_of(x0, gp[0].z, gp[0].s, QMAX);
-            uint32_t c1 = code_of(x1, gp[NG].z, gp[NG].s, QMAX);
-            word |= (c0 | (c1 << 16)) << (BITS * slot);
-          }
+      for (int slot = 0; slot < NSLOT; ++slot) {
+        const int tt = slot / CB, cb = slot % CB, d = cb * 16 + col;
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+          const int tl = t * TPT + tt * 16 + row, gl = (t * TPT + tt * 16) / G;
+          const float4 zi = *reinterpret_cast<const float4*>(&par_zi[gl * D + d]);  // channels d, d + 1
+          const uint32_t xx = *reinterpret_cast<const uint32_t*>(tile + tl * ROWB + d * 2);
+          word[t] |= code_pair<BITS>(__uint_as_float(xx << 16), __uint_as_float(xx & 0xffff0000u), zi.x, zi.y, zi.z, zi.w,
+                                     doubt[t]) << (BITS * slot);
         }
       }
-      wbuf[tile_l * 128 + lane * 4 + i] = word;
+    } else {
+#pragma unroll
+      for (int slot = 0; slot < NSLOT; ++slot) {
+        const int tt = slot / CB, cb = slot % CB, d = cb * 16 + row, gi = (cb * 16) / G;
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+          const int tl = t * TPT + tt * 16 + col;  // tokens tl, tl + 1
+          const float4 zi = *reinterpret_cast<const float4*>(&par_zi[gi * T + tl]);
+          const uint8_t* src = tile + tl * ROWB + d * 2;
+          const float x0 = bf16_bits(*reinterpret_cast<const uint16_t*>(src));
+          const float x1 = bf16_bits(*reinterpret_cast<const uint16_t*>(src + ROWB));
+          word[t] |= code_pair<BITS>(x0, x1, zi.x, zi.y, zi.z, zi.w, doubt[t]) << (BITS * slot);
+        }
+      }
     }
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+      if (doubt[t]) {  // rare: the word again, with the division
+        uint32_t w = 0u;
+#pragma unroll 1
+        for (int slot = 0; slot < NSLOT; ++slot) {
+          const int tt = slot / CB, cb = slot % CB;
+          uint32_t c0, c1;
+          if (kind == 0) {
+            const int tl = t * TPT + tt * 16 + row, d = cb * 16 + col, g0 = ((t * TPT + tt * 16) / G) * D + d;
+            const uint32_t xx = *reinterpret_cast<const uint32_t*>(tile + tl * ROWB + d * 2);
+            c0 = code_of(__uint_as_float(xx << 16), par_zi[g0].x, par_s[g0], QMAX);
+            c1 = code_of(__uint_as_float(xx & 0xffff0000u), par_zi[g0 + 1].x, par_s[g0 + 1], QMAX);
+          } else {
+            const int tl = t * TPT + tt * 16 + col, d = cb * 16 + row, g0 = ((cb * 16) / G) * T + tl;
+            const uint8_t* src = tile + tl * ROWB + d * 2;
+            c0 = code_of(bf16_bits(*reinterpret_cast<const uint16_t*>(src)), par_zi[g0].x, par_s[g0], QMAX);
+            c1 = code_of(bf16_bits(*reinterpret_cast<const uint16_t*>(src + ROWB)), par_zi[g0 + 1].x, par_s[g0 + 1], QMAX);
+          }
+          w |= (c0 | (c1 << 16)) << (BITS * slot);
+        }
+        word[t] = w;
+      }
+      wbuf[t * 128 + lane * 4 + i] = word[t];
+    }
+    return NT * 128;
   };
-  if (bits == 2)
-    build(std::integral_constant<int, 2>{});
-  else
-    build(std::integral_constant<int, 1>{});
+  const int n_words = (bits == 2) ? build(std::integral_constant<int, 2>{}) : build(std::integral_constant<int, 1>{});
   __syncthreads();
 
   uint32_t* codes = kind ? p.L.v_codes : p.L.k_codes;
@@ -257,14 +276,16 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
 cudaError_t launch_pack(const PackParams& p, cudaStream_t st) {
   int tiles = p.n_blocks * (p.dm.R / p.tb);
   dim3 grid(2 * tiles, p.dm.Hkv, p.dm.B);
-  if (p.dm.D == 128 && p.dm.g == 32)
-    pack_kernel<128, 32><<<grid, PACK_THREADS, 0, st>>>(p);
-  else if (p.dm.D == 128)
-    pack_kernel<128, 64><<<grid, PACK_THREADS, 0, st>>>(p);
-  else if (p.dm.g == 32)
-    pack_kernel<64, 32><<<grid, PACK_THREADS, 0, st>>>(p);
-  else
-    pack_kernel<64, 64><<<grid, PACK_THREADS, 0, st>>>(p);
+  const int key = p.dm.D * 10000 + p.dm.g * 100 + p.tb;
+  switch (key) {
+    case 1283232: pack_kernel<128, 32, 32><<<grid, PACK_THREADS, 0, st>>>(p); break;
+    case 1283264: pack_kernel<128, 32, 64><<<grid, PACK_THREADS, 0, st>>>(p); break;
+    case 1286464: pack_kernel<128, 64, 64><<<grid, PACK_THREADS, 0, st>>>(p); break;
+    case 643232: pack_kernel<64, 32, 32><<<grid, PACK_THREADS, 0, st>>>(p); break;
+    case 643264: pack_kernel<64, 32, 64><<<grid, PACK_THREADS, 0, st>>>(p); break;
+    case 646464: pack_kernel<64, 64, 64><<<grid, PACK_THREADS, 0, st>>>(p); break;
+    default: return cudaErrorInvalidValue;
+  }
   return cudaGetLastError();
 }
 
