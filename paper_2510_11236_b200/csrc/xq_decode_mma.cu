@@ -36,6 +36,8 @@
 // the partials and writes the output.  No thread ever spins on memory.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+
+#include <type_traits>
 #include <math_constants.h>
 
 #include "xq_internal.h"
@@ -694,6 +696,18 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     if (St::VC == 1024) cp_async16_if(s + St::OFF_VC + 512, v + 512, on);
     cp_async16_if(s + St::OFF_VM, gvm + (size_t)(uint32_t)jj * St::VM, on && lane * 16 < St::VM);
   };
+  // the same for a unit that is known to exist: no predicates beyond the two lane masks
+  auto issue_unit_always = [&](int jj, uint32_t soff) {
+    const uint32_t s = my + soff + lane * 16;
+    const uint8_t* k = gk + (size_t)(uint32_t)jj * St::KC;
+    cp_async16(s, k);
+    if (St::KC == 1024) cp_async16(s + 512, k + 512);
+    if (lane < 16) cp_async16(s + St::OFF_KS, gks + (size_t)(uint32_t)(((uw + jj) * 32) / GS) * 256);
+    const uint8_t* v = gv + (size_t)(uint32_t)jj * St::VC;
+    cp_async16(s + St::OFF_VC, v);
+    if (St::VC == 1024) cp_async16(s + St::OFF_VC + 512, v + 512);
+    if (lane * 16 < St::VM) cp_async16(s + St::OFF_VM, gvm + (size_t)(uint32_t)jj * St::VM);
+  };
   // stage the key zero-point rows of the groups of units [jb, jb + ZROWS) (no commit)
   auto issue_zero_rows = [&](int jb) {
     const int rows = min(ZROWS, n_my - jb);
@@ -810,7 +824,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   // One iteration: bias table every ZROWS units, refill of the stage unit j - 1 used, softmax reference,
   // numerators of unit j, then (MORE) logits of unit j + 1 next to the value product of unit j.
   // off_prev / off_cur / off_next: ring offsets of the stages of units j - 1 (free, refilled), j and j + 1.
-  auto step = [&](int j, bool more, uint32_t off_prev, uint32_t off_cur, uint32_t off_next) {
+  // refill: unit j + NST - 1 exists (then so does unit j + 1, and `more` is true)
+  auto step = [&](auto refill, int j, bool more, uint32_t off_prev, uint32_t off_cur, uint32_t off_next) {
     const int jr = j & (ZROWS - 1);
     if (jr == 0) {
       // bias table of units [j, j + 16): ztab[row][head] = scale * sum_d q_d z_d (log2 units)
@@ -834,8 +849,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     }
 
     __syncwarp();  // every lane is done with the stage of unit j - 1
-    issue_unit(j + NST - 1, off_prev);
-    cp_async_commit();
+    if (decltype(refill)::value) issue_unit_always(j + NST - 1, off_prev);
+    cp_async_commit();  // (an empty group once the stream's end is near: the waits below count groups)
 
     // ---- softmax reference: raise it only when a logit of unit j exceeds it by more than TAU ----
     const float2 bz = lds64f(ztab + jr * 32 + tig * 8);
@@ -882,9 +897,13 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   // main loop: one copy of the body (four unrolled copies with constant stage offsets save address arithmetic
   // but cost more in instruction-cache misses than they save)
   static_assert(NST == 4, "ring of four stages");
+  int j = 0;
 #pragma unroll 1
-  for (int j = 0; j < n_my; ++j)  // the very last unit has no successor
-    step(j, j + 1 < n_my, ((j + 3) & 3) * St::BYTES, (j & 3) * St::BYTES, ((j + 1) & 3) * St::BYTES);
+  for (; j + NST - 1 < n_my; ++j)  // steady state: every refill exists
+    step(std::true_type{}, j, true, ((j + 3) & 3) * St::BYTES, (j & 3) * St::BYTES, ((j + 1) & 3) * St::BYTES);
+#pragma unroll 1
+  for (; j < n_my; ++j)  // the last NST - 1 units: nothing left to fetch; the very last unit has no successor
+    step(std::false_type{}, j, j + 1 < n_my, ((j + 3) & 3) * St::BYTES, (j & 3) * St::BYTES, ((j + 1) & 3) * St::BYTES);
   cp_async_wait<0>();
   __syncthreads();  // all warps are done with their stages: the memory becomes the merge buffer
 
