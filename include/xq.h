@@ -59,6 +59,14 @@ extern "C" {
 #define XQ_KERNEL_AUTO 0    /* tensor-core kernel when the shape allows it, else generic   */
 #define XQ_KERNEL_GENERIC 1 /* scalar kernel: any supported shape, slow, used as cross-check */
 #define XQ_KERNEL_MMA 2     /* tensor-core kernel: head_dim 128, group of <= 8 query heads  */
+/* The tensor-core kernel rounds the products q_d * s_d (query times key scale) to
+ * fp16 before its matrix product: relative 2^-12 of every term of a logit.  Over
+ * contexts with spread-out attention that stays far below 2e-3 in the result; a
+ * query with very large logits on a few tokens (|logit| of tens) can see several
+ * 1e-3.  This variant (head_dim 128, groups of <= 4 query heads) carries each
+ * product as an fp16 pair (rounded value + what the rounding lost) and is about
+ * 5 % slower. */
+#define XQ_KERNEL_MMA_PRECISE 3
 
 #define XQ_MEM_DEVICE 0
 #define XQ_MEM_HOST 1

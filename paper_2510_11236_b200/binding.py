@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libxq.so")
 XQ_OK = 0
 XQ_ERR_CONFIG, XQ_ERR_ARG, XQ_ERR_CAPACITY, XQ_ERR_ORDER, XQ_ERR_CUDA, XQ_ERR_NOMEM = -1, -2, -3, -4, -5, -6
 XQ_BF16 = 0
-XQ_KERNEL_AUTO, XQ_KERNEL_GENERIC, XQ_KERNEL_MMA = 0, 1, 2
+XQ_KERNEL_AUTO, XQ_KERNEL_GENERIC, XQ_KERNEL_MMA, XQ_KERNEL_MMA_PRECISE = 0, 1, 2, 3
 XQ_MEM_DEVICE, XQ_MEM_HOST = 0, 1
 XQ_MAX_SPLITS = 256
 XQ_STATIC_SCRATCH_BYTES = 8 << 20

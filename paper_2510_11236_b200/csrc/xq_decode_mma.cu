@@ -107,6 +107,11 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   __half2 h = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&h);
 }
+// a * b - c in one rounding, per half
+__device__ __forceinline__ uint32_t hfms2_u(uint32_t a, uint32_t b, uint32_t c) {
+  __half2 r = __hfma2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<__half2*>(&b), __hneg2(*reinterpret_cast<__half2*>(&c)));
+  return *reinterpret_cast<uint32_t*>(&r);
+}
 __device__ __forceinline__ uint32_t hmul2_u(uint32_t a, uint32_t b) {
   __half2 r = __hmul2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<__half2*>(&b));
   return *reinterpret_cast<uint32_t*>(&r);
@@ -526,9 +531,12 @@ __device__ __forceinline__ void ticket_merge(const DecodeParams& p, int ns, int 
 
 // S^T = Kc (q s)^T for the 32 tokens of the unit staged at `st`:
 // accS[mt] rows = tokens 16 mt + gid (+8), cols = heads 2 tig (+1); values carry a factor 2^-24.
-template <int BK, int BV, int GS>
-__device__ __forceinline__ void unit_logits(uint32_t st, const uint32_t (&qe)[16], float (&accS)[2][4], int lane,
-                                            int tig) {
+// HP (with the spread column layout only): column 2h carries fp16(q_d s_d) of head h and column 2h + 1 what that
+// rounding lost, q_d s_d - fp16(q_d s_d) (one fused multiply-add; alpha is 1 in the odd columns and 0 in the even
+// ones, where the same instruction reproduces the rounded product).  The caller adds the two columns' sums.
+template <int BK, int BV, int GS, bool HP>
+__device__ __forceinline__ void unit_logits(uint32_t st, const uint32_t (&qe)[16], uint32_t alpha, float (&accS)[2][4],
+                                            int lane, int tig) {
   using St = Stage<BK, BV, GS>;
   uint4 w[2];
   if (BK == 2) {
@@ -546,8 +554,14 @@ __device__ __forceinline__ void unit_logits(uint32_t st, const uint32_t (&qe)[16
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const uint4 sv = lds128(st + St::OFF_KS + i * 64 + tig * 16);  // scales of k-steps 2i, 2i+1
-    const uint32_t bq[4] = {hmul2_u(qe[4 * i + 0], sv.x), hmul2_u(qe[4 * i + 1], sv.y),
-                            hmul2_u(qe[4 * i + 2], sv.z), hmul2_u(qe[4 * i + 3], sv.w)};
+    uint32_t bq[4] = {hmul2_u(qe[4 * i + 0], sv.x), hmul2_u(qe[4 * i + 1], sv.y),
+                      hmul2_u(qe[4 * i + 2], sv.z), hmul2_u(qe[4 * i + 3], sv.w)};
+    if (HP) {
+      bq[0] = hfms2_u(qe[4 * i + 0], sv.x, hmul2_u(bq[0], alpha));
+      bq[1] = hfms2_u(qe[4 * i + 1], sv.y, hmul2_u(bq[1], alpha));
+      bq[2] = hfms2_u(qe[4 * i + 2], sv.z, hmul2_u(bq[2], alpha));
+      bq[3] = hfms2_u(qe[4 * i + 3], sv.w, hmul2_u(bq[3], alpha));
+    }
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       const int s = 2 * i + h;
@@ -560,6 +574,13 @@ __device__ __forceinline__ void unit_logits(uint32_t st, const uint32_t (&qe)[16
         else
           mma16816(accS[mt], src.x & mk, src.y & mk, src.z & mk, src.w & mk, bq[2 * h], bq[2 * h + 1]);
       }
+    }
+  }
+  if (HP) {
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      accS[mt][0] += accS[mt][1];
+      accS[mt][2] += accS[mt][3];
     }
   }
 }
@@ -622,8 +643,10 @@ __device__ __forceinline__ void unit_values(uint32_t st, const uint32_t (&pb)[2]
 // ---------------------------------------------------------------------------
 // SP ("spread"): groups of at most 4 query heads put head h in column 2h of the N = 8 tiles and leave the odd
 // columns as padding, so that each thread's accumulator pairs hold one real head: half the softmax work.
-template <int BK, int BV, int GS, bool SP>
+// HP: q_d s_d as an fp16 pair in the two columns of a head (see unit_logits); needs SP.
+template <int BK, int BV, int GS, bool SP, bool HP>
 __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams p) {
+  static_assert(SP || !HP, "the residual column is the padding column of the spread layout");
   using St = Stage<BK, BV, GS>;
   constexpr int NG = St::NG;
   constexpr int WARP_BYTES = warp_bytes<BK, BV, GS>();
@@ -759,6 +782,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
 
   cp_async_commit();  // group 0, or the window tile's group (empty for the other warps)
 
+  const uint32_t alpha = (HP && (gid & 1)) ? 0x3C003C00u : 0u;  // (1, 1) in the residual columns
   uint32_t qe[16];  // q as fp16 B operand, pre-scaled by 2^-e(s), the weight the code's slot carries
 #pragma unroll
   for (int s = 0; s < 8; ++s) {
@@ -766,6 +790,13 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     for (int j = 0; j < 2; ++j) {
       float lo = bf16_to_f(raw[2 * s + j] & 0xffff), hi = bf16_to_f(raw[2 * s + j] >> 16);
       if (warp == 0) q_sm[((s >> 1) * 32 + lane) * 4 + (s & 1) * 2 + j] = pack_half2(lo, hi);
+      if (HP) {  // the odd column of a head multiplies the same q (its raw[] stays zero: bias and window use it)
+        const uint32_t left = __shfl_up_sync(0xffffffffu, raw[2 * s + j], 4);
+        if ((gid & 1) && (gid >> 1) < G) {
+          lo = bf16_to_f(left & 0xffff);
+          hi = bf16_to_f(left >> 16);
+        }
+      }
       const float sc = 1.0f / (float)(1 << Slots<BK>::e(s));
       qe[2 * s + j] = pack_half2(lo * sc, hi * sc);
     }
@@ -819,7 +850,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
       for (int i = 0; i < 4; ++i) accO[mt][i] *= wgt;
     }
   }
-  if (n_my > 0) unit_logits<BK, BV, GS>(my, qe, accS, lane, tig);
+  if (n_my > 0) unit_logits<BK, BV, GS, HP>(my, qe, alpha, accS, lane, tig);
 
   // One iteration: bias table every ZROWS units, refill of the stage unit j - 1 used, softmax reference,
   // numerators of unit j, then (MORE) logits of unit j + 1 next to the value product of unit j.
@@ -890,7 +921,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
       pb[mt][0] = movmatrix_trans(pack_half2(p0, p1));
       pb[mt][1] = movmatrix_trans(pack_half2(p2, p3));
     }
-    if (more) unit_logits<BK, BV, GS>(my + off_next, qe, accS, lane, tig);
+    if (more) unit_logits<BK, BV, GS, HP>(my + off_next, qe, alpha, accS, lane, tig);
     unit_values<BK, BV, GS>(my + off_cur, pb, accO, accZ, lane, gid, tig);
   };
 
@@ -950,35 +981,36 @@ int smem_bytes(int G) {
   return pipe_bytes<BK, BV, GS>() + Q_BYTES + WIN_BYTES;
 }
 
-template <int BK, int BV, int GS, bool SP>
+template <int BK, int BV, int GS, bool SP, bool HP>
 cudaError_t launch_sp(const DecodeParams& p, cudaStream_t st) {
   const int smem = smem_bytes<BK, BV, GS>(p.dm.G);
   static int configured = 0;
   if (configured < smem) {
-    cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<BK, BV, GS, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<BK, BV, GS, SP, HP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     configured = smem;
   }
   const int ns = p.ns_q > 0 ? p.ns_q : p.ns_w;
   dim3 grid(ns, p.dm.Hkv, p.dm.B);
-  return launch_dependent(decode_mma_kernel<BK, BV, GS, SP>, grid, dim3(MMA_THREADS), (size_t)smem, st, p);
+  return launch_dependent(decode_mma_kernel<BK, BV, GS, SP, HP>, grid, dim3(MMA_THREADS), (size_t)smem, st, p);
 }
 
 template <int BK, int BV, int GS>
 cudaError_t launch_t(const DecodeParams& p, cudaStream_t st) {
-  return p.dm.G <= 4 ? launch_sp<BK, BV, GS, true>(p, st) : launch_sp<BK, BV, GS, false>(p, st);
+  if (p.dm.G > 4) return p.precise ? cudaErrorInvalidValue : launch_sp<BK, BV, GS, false, false>(p, st);
+  return p.precise ? launch_sp<BK, BV, GS, true, true>(p, st) : launch_sp<BK, BV, GS, true, false>(p, st);
 }
 
-template <int BK, int BV, int GS, bool SP>
+template <int BK, int BV, int GS, bool SP, bool HP>
 int ctas_per_sm_sp(int G) {
   const int smem = smem_bytes<BK, BV, GS>(G);
-  if (cudaFuncSetAttribute(decode_mma_kernel<BK, BV, GS, SP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+  if (cudaFuncSetAttribute(decode_mma_kernel<BK, BV, GS, SP, HP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
       cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
   int n = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_mma_kernel<BK, BV, GS, SP>, MMA_THREADS, smem) !=
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_mma_kernel<BK, BV, GS, SP, HP>, MMA_THREADS, smem) !=
       cudaSuccess) {
     cudaGetLastError();
     return 0;
@@ -988,7 +1020,7 @@ int ctas_per_sm_sp(int G) {
 
 template <int BK, int BV, int GS>
 int ctas_per_sm_t(int G) {
-  return G <= 4 ? ctas_per_sm_sp<BK, BV, GS, true>(G) : ctas_per_sm_sp<BK, BV, GS, false>(G);
+  return G <= 4 ? ctas_per_sm_sp<BK, BV, GS, true, false>(G) : ctas_per_sm_sp<BK, BV, GS, false, false>(G);
 }
 
 }  // namespace

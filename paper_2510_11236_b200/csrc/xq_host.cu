@@ -50,7 +50,8 @@ bool check(const xq_config* c) {
   if (!(c->sm_scale >= 0.f) || isinf(c->sm_scale)) return false;
   if (c->n_splits < 0 || c->n_splits > XQ_MAX_SPLITS) return false;
   if (c->io_dtype != XQ_BF16) return false;
-  if (c->kernel < XQ_KERNEL_AUTO || c->kernel > XQ_KERNEL_MMA) return false;
+  if (c->kernel < XQ_KERNEL_AUTO || c->kernel > XQ_KERNEL_MMA_PRECISE) return false;
+  if (c->kernel == XQ_KERNEL_MMA_PRECISE && (c->head_dim != 128 || c->n_q_heads / c->n_kv_heads > 4)) return false;
   bool any_1bit = c->kq < c->n_layers || c->vq < c->n_layers;
   if (c->head_dim == 64 && any_1bit && c->residual_len % 64) return false;
   // both layers of a sharing pair must have the same bit-width
@@ -301,6 +302,7 @@ int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, c
   DecodeParams p;
   p.early_fetch = 0;
   p.K_new = p.V_new = nullptr;
+  p.precise = 0;
   p.dm = dm;
   p.L = layer_ptrs(c, layer);
   p.q = (const uint16_t*)q;
@@ -311,12 +313,13 @@ int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, c
   p.part_acc = (float*)(c->ws + c->plan.part_acc);
   p.part_ml = (float*)(c->ws + c->plan.part_ml);
   bool use_mma = layer_uses_mma(c, layer);
-  if (c->cfg.kernel == XQ_KERNEL_MMA && !use_mma) return XQ_ERR_CONFIG;
+  if (c->cfg.kernel >= XQ_KERNEL_MMA && !use_mma) return XQ_ERR_CONFIG;
   p.out = out;
   p.out_f32 = out_f32;
   p.tickets = (unsigned int*)(c->ws + c->plan.tickets);
   p.K_new = (const uint16_t*)K_new;
   p.V_new = (const uint16_t*)V_new;
+  p.precise = c->cfg.kernel == XQ_KERNEL_MMA_PRECISE;
   if (K_new && !(use_mma && nq > 0)) return XQ_ERR_ARG;
   cudaError_t e;
   if (use_mma) {
@@ -494,10 +497,11 @@ int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out,
     if (So - residual_count(So, dm.R) < nq) return XQ_ERR_ORDER;
   }
   const bool use_mma = layer_uses_mma(c, layer);
-  if (c->cfg.kernel == XQ_KERNEL_MMA && !use_mma) return XQ_ERR_CONFIG;
+  if (c->cfg.kernel >= XQ_KERNEL_MMA && !use_mma) return XQ_ERR_CONFIG;
   DecodeParams p;
   p.early_fetch = 0;
   p.K_new = p.V_new = nullptr;
+  p.precise = c->cfg.kernel == XQ_KERNEL_MMA_PRECISE;
   p.dm = dm;
   p.L = layer_ptrs(c, layer);
   p.q = (const uint16_t*)q;

@@ -69,6 +69,7 @@ struct DecodeParams {
   // window holds that row reads it from here and stores it into the window.
   const uint16_t* K_new;
   const uint16_t* V_new;
+  int precise;  // tensor-core kernel, groups of <= 4 query heads: carry q_d s_d as an fp16 pair (XQ_KERNEL_MMA_PRECISE)
 };
 
 struct MergeParams {

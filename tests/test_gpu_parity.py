@@ -233,6 +233,46 @@ def test_decode_step_appends_inside_the_decode_kernel():
                         util.check_attention(cache, oc, l, q[l], b, hk, o32[l], None, tol=short_context_tol)
 
 
+@pytest.mark.parametrize("S", [1000, 8192])
+def test_precise_kernel_on_queries_with_a_few_dominant_tokens(S):
+    """Queries built from the keys of one, two or four tokens, scaled up: logits of tens on those tokens, so the
+    result follows the logits' error.  XQ_KERNEL_MMA_PRECISE (q_d s_d as an fp16 pair) stays within the 2e-3 of
+    the other tests; the default tensor-core kernel (q_d s_d rounded to fp16: 2^-12 of every term of a logit)
+    is allowed the 2e-2 that 2^-12 of a logit magnitude of ~80 can cost, and must agree with the precise one
+    to that."""
+    w = dict(W.CONFIGS["c2"], n_layers=2, batch=1, n_kv_heads=1, n_q_heads=4, seq=S, kq=2, vq=0)
+    k0, v0, k1, v1 = W.pair_tokens(w, 0, 0, S, DEV)
+    kv = {0: (k0, v0), 1: (k1, v1)}
+    caches = {}
+    for kernel in (xq.XQ_KERNEL_MMA_PRECISE, xq.XQ_KERNEL_AUTO):
+        cfg = W.make_xq_config(w, kernel=kernel)
+        caches[kernel] = xq.Cache(cfg, DEV)
+        caches[kernel].append_kv(0, k0, v0)
+        caches[kernel].append_kv(1, k1, v1)
+    oc = util.oracle_for_stream(caches[xq.XQ_KERNEL_AUTO].cfg, [0, 1], 0, 0, kv)
+    gen = torch.Generator().manual_seed(3)
+    K = k0[0, 0].float().cpu()
+    worst = {xq.XQ_KERNEL_MMA_PRECISE: 0.0, xq.XQ_KERNEL_AUTO: 0.0}
+    for trial in range(6):
+        t = torch.randint(0, S - 200, (8,), generator=gen)
+        for layer in (0, 1):  # layer 1 borrows layer 0's codes: the same keys up to the second layer's noise
+            q = torch.zeros(1, 4, 128)
+            q[0, 0] = torch.randn(128, generator=gen)
+            q[0, 1] = K[t[0]] * 0.3
+            q[0, 2] = (K[t[1]] + K[t[2]]) * 0.21
+            q[0, 3] = (K[t[3]] + K[t[4]] + K[t[5]] + K[t[6]]) * 0.15
+            qb = q.to(torch.bfloat16).to(DEV)
+            ref = oc.decode(layer, util.bits_of(qb))[0]
+            for kernel, cache in caches.items():
+                got = cache.decode_attention(layer, qb, f32=True)[0].double().cpu().numpy()
+                worst[kernel] = max(worst[kernel], np.abs(got - ref).max())
+    print("peaked queries, S =", S, "fp32 error: precise %.2e, default %.2e" % (worst[xq.XQ_KERNEL_MMA_PRECISE], worst[xq.XQ_KERNEL_AUTO]))
+    assert worst[xq.XQ_KERNEL_MMA_PRECISE] <= util.ATTN_TOL
+    assert worst[xq.XQ_KERNEL_AUTO] <= 2e-2
+    for cache in caches.values():
+        cache.close()
+
+
 @pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4"])
 def test_full_size_configs_sampled(name):
     """The benchmark's shapes and launch configuration (library-chosen splits, tensor-core kernel), one layer
