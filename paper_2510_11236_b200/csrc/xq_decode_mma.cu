@@ -1,15 +1,16 @@
 // Tensor-core decode attention over the packed cache (head_dim 128, up to 8
 // query heads per kv head).
 //
-// Why mma.sync from registers and not tcgen05: the packed cache delivers
-// ~1.8e13 quantized elements/s at the HBM roofline.  tcgen05.mma takes its
-// operands from shared memory (or TMEM), so every dequantized element would
-// have to be written to and read back from on-chip memory at one byte or more
-// each -- more than the SMs' shared-memory bandwidth.  Here the codes never
-// leave registers in expanded form: the packed word layout is the A-fragment
-// layout of mma.sync.m16n8k16, so `word & mask` IS an fp16x2 operand register
-// (the code sits in the mantissa bits of an fp16 subnormal: value c * 2^(pos-24)),
-// and scale / zero-point are folded into the other operand:
+// Why mma.sync from registers: the packed cache delivers ~1.8e13 quantized
+// elements/s at the HBM roofline, so an element may cost about one instruction
+// per two elements and no trip through on-chip memory in expanded form.  The
+// packed word layout is the A-fragment layout of mma.sync.m16n8k16, so
+// `word & mask` IS an fp16x2 operand register (the code sits in the mantissa
+// bits of an fp16 subnormal: value c * 2^(pos-24)), and scale / zero-point are
+// folded into the other operand.  (tcgen05.mma takes A from shared or tensor
+// memory: the codes would have to be expanded there first -- the same masks plus
+// tcgen05.st -- and with N = 8..16 columns one tcgen05.mma costs its issuing
+// thread ~67 cycles on this part; a version built that way ran slower.)
 //
 //   q . k_hat_t = sum_d (q_d s_d) c_td + sum_d q_d z_d        (keys, per channel)
 //   sum_t p_t v_hat_td = sum_t (p_t s_tg) c_td + sum_t p_t z_tg  (values, per token)
@@ -34,6 +35,15 @@
 // partial (m, l, acc[D]) per query head.  The CTA that finishes last for a
 // (sequence, kv head) -- found with an atomic ticket, never by waiting -- merges
 // the partials and writes the output.  No thread ever spins on memory.
+//
+// Launch: programmatic dependent launch.  The kernel lets its successor start
+// at once and waits for its predecessor only after it has queued its first
+// packed units (when the host says that no pack kernel wrote them since the
+// layer's last decode), so its set-up hides under the predecessor's tail.
+// Variants: SP (groups of <= 4 heads in the even columns, odd columns padding),
+// HP (the padding column carries what the fp16 rounding of q_d s_d lost), and
+// the fused append of xq_decode_step (the newest window row comes from the
+// step's input and is stored into the window by the CTA that reads it).
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -925,8 +935,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     unit_values<BK, BV, GS>(my + off_cur, pb, accO, accZ, lane, gid, tig);
   };
 
-  // main loop: one copy of the body (four unrolled copies with constant stage offsets save address arithmetic
-  // but cost more in instruction-cache misses than they save)
+  // main loop: two copies of the body, one that refills and one that does not (four unrolled copies with constant
+  // stage offsets save address arithmetic but cost more in instruction-cache misses than they save)
   static_assert(NST == 4, "ring of four stages");
   int j = 0;
 #pragma unroll 1
