@@ -235,6 +235,41 @@ def test_decode_step_appends_inside_the_decode_kernel(kernel, oracle_tol):
                         util.check_attention(cache, oc, l, q[l], b, hk, o32[l], None, tol=short_context_tol)
 
 
+@pytest.mark.parametrize("G,kernel", [(1, xq.XQ_KERNEL_AUTO), (1, xq.XQ_KERNEL_MMA_PRECISE), (2, xq.XQ_KERNEL_AUTO),
+                                      (3, xq.XQ_KERNEL_MMA_PRECISE), (4, xq.XQ_KERNEL_MMA_PRECISE),
+                                      (5, xq.XQ_KERNEL_AUTO), (8, xq.XQ_KERNEL_MMA)])
+def test_decode_step_head_groupings(G, kernel):
+    """Every size of query-head group the tensor-core kernel takes (1..4: heads in the even columns, with and
+    without the residual column; 5..8: all columns), through xq_decode_step (in-kernel append) over a window
+    flush: regions bit for bit, attention against the oracle (700 tokens with x10 outlier channels: the default
+    kernel gets the short-context tolerance derived in test_decode_step_appends_inside_the_decode_kernel)."""
+    tol = util.ATTN_TOL if kernel == xq.XQ_KERNEL_MMA_PRECISE else 6e-3
+    L, B, Hkv, D, R = 2, 2, 2, 128, 64
+    w = dict(n_layers=L, batch=B, n_q_heads=G * Hkv, n_kv_heads=Hkv, head_dim=D, seq=700, residual_len=R,
+             group_size=32, kq=2, vq=2, km=0, vm=2, n_outliers=3, outlier_scale=10.0, seed=23 + G, n_splits=0)
+    cfg = W.make_xq_config(w, max_seq=800, kernel=kernel)
+    cache = xq.Cache(cfg, DEV)
+    kv = _fill(cache, w, [0, 1], 700, step=333)
+    gen = torch.Generator(device="cpu").manual_seed(G)
+    for step in range(6):  # lengths 701 .. 706; 705 quantizes the block 640 .. 703
+        kn = torch.randn(L, B, Hkv, 1, D, generator=gen).to(torch.bfloat16).to(DEV)
+        vn = torch.randn(L, B, Hkv, 1, D, generator=gen).to(torch.bfloat16).to(DEV)
+        q = torch.randn(L, B, G * Hkv, D, generator=gen).to(torch.bfloat16).to(DEV)
+        out = torch.empty_like(q)
+        cache.decode_step(kn, vn, q, out)
+        torch.cuda.synchronize()
+        for l in range(L):
+            kv[l] = (torch.cat([kv[l][0], kn[l]], dim=2), torch.cat([kv[l][1], vn[l]], dim=2))
+        o32 = [cache.decode_attention(l, q[l], f32=True) for l in range(L)]
+        for b in range(B):
+            for hk in range(Hkv):
+                oc = util.oracle_for_stream(cfg, [0, 1], b, hk, kv)
+                for l in range(L):
+                    util.compare_regions(cache, oc, l, b, hk)
+                    util.check_attention(cache, oc, l, q[l], b, hk, o32[l], out[l], tol=tol)
+    cache.close()
+
+
 @pytest.mark.parametrize("S", [1000, 8192])
 def test_precise_kernel_on_queries_with_a_few_dominant_tokens(S):
     """Queries built from the keys of one, two or four tokens, scaled up: logits of tens on those tokens, so the
