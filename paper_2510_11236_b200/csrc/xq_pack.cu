@@ -42,21 +42,33 @@ constexpr int PACK_THREADS = 128;
 constexpr int PACK_ROW_PAD = 16;  // bytes added to each staged row: 8 consecutive rows then fall in 8 different bank groups
 constexpr float PACK_MAGIC = 12582912.0f;  // 1.5 * 2^23: x + MAGIC has rint(x) in its low mantissa bits for |x| < 2^22
 
-__device__ __forceinline__ float rcp_or_zero(float s) { return (s == 0.0f) ? 0.0f : __frcp_rn(s); }
+// 1/s for the quotient sequence of code_pair: 0 for a constant group (every code 0), NaN where that sequence is
+// not known to round correctly -- a scale whose significand is all ones, or one so small or large that an
+// intermediate could leave the normal range -- which sends the word to the division.
+__device__ __forceinline__ float safe_rcp(float s) {
+  if (s == 0.0f) return 0.0f;
+  const uint32_t b = __float_as_uint(s);
+  const uint32_t e = (b >> 23) & 0xffu;
+  if ((b & 0x7fffffu) == 0x7fffffu || e < 40u || e > 210u) return __uint_as_float(0x7fc00000u);
+  return __frcp_rn(s);
+}
 
-// Eq. 2 for two elements through the reciprocals.  (x - z) * inv differs from the correctly rounded quotient
-// (x - z) / s by at most three roundings of a value below 2^B, i.e. by less than 6e-7, so both round to the same
-// integer unless the product lies within 1e-5 of a tie; `doubt` collects that case (and any non-finite product
-// of a subnormal scale), and the caller then recomputes the word with the division.  The fused multiply-add
-// with MAGIC rounds the exact product to the nearest integer, ties to even, and leaves it in the low mantissa
-// bits; 0 <= (x - z) / s < 2^B - 1/2 holds for every member of the group, so this path needs no clamp.
+// Eq. 2 for two elements without a division.  With y = RN(1/s): q = RN(a y), r = a - q s (exact in one fused
+// multiply-add), q' = RN(q + r y) is the correctly rounded quotient RN(a / s) (the classical correction step of
+// division by a correctly rounded reciprocal; the significands it can miss are excluded by safe_rcp), so
+// rint(q') is the code the division gives, ties included.  Adding 1.5 * 2^23 rounds to the nearest integer, ties
+// to even, and leaves it in the low mantissa bits; 0 <= a / s < 2^B - 1/2 holds for every member of the group, so
+// no clamp is needed.  A NaN reciprocal sets `doubt` and the caller recomputes the word with the division.
 // Returns code(x0) | code(x1) << 16.
 template <int BITS>
-__device__ __forceinline__ uint32_t code_pair(float x0, float x1, float z0, float inv0, float z1, float inv1, bool& doubt) {
-  const float a0 = __fsub_rn(x0, z0), a1 = __fsub_rn(x1, z1);
-  const float u0 = __fmaf_rn(a0, inv0, PACK_MAGIC), u1 = __fmaf_rn(a1, inv1, PACK_MAGIC);
-  const float d0 = __fmaf_rn(a0, inv0, -__fsub_rn(u0, PACK_MAGIC)), d1 = __fmaf_rn(a1, inv1, -__fsub_rn(u1, PACK_MAGIC));
-  doubt |= !(fabsf(d0) <= 0.49999f) | !(fabsf(d1) <= 0.49999f);
+__device__ __forceinline__ uint32_t code_pair(float x0, float x1, const float4& p0, const float4& p1, bool& doubt) {
+  const float a0 = __fsub_rn(x0, p0.x), a1 = __fsub_rn(x1, p1.x);
+  float q0 = __fmul_rn(a0, p0.y), q1 = __fmul_rn(a1, p1.y);
+  const float r0 = __fmaf_rn(-q0, p0.z, a0), r1 = __fmaf_rn(-q1, p1.z, a1);
+  q0 = __fmaf_rn(r0, p0.y, q0);
+  q1 = __fmaf_rn(r1, p1.y, q1);
+  const float u0 = __fadd_rn(q0, PACK_MAGIC), u1 = __fadd_rn(q1, PACK_MAGIC);
+  doubt |= (p0.y != p0.y) | (p1.y != p1.y);
   constexpr uint32_t QM = (1u << BITS) - 1u;
   return __byte_perm(__float_as_uint(u0), __float_as_uint(u1), 0x0400) & (QM | (QM << 16));
 }
@@ -74,8 +86,7 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
   constexpr int KP = PACK_THREADS / ((T / G) * (D / 2));               // token parts of a key group in the statistics
   static_assert(KP >= 1 && G % KP == 0, "key statistics: 128 threads over (group, channel pair, token part)");
   __shared__ __align__(16) uint8_t tile[T * ROWB];
-  __shared__ __align__(16) float2 par_zi[NPAR];  // (z, 1/s) of a group; keys: [group][channel], values: [channel group][token]
-  __shared__ float par_s[NPAR];
+  __shared__ __align__(16) float4 par[NPAR];  // (z, 1/s, s, -) of a group; keys: [group][channel], values: [channel group][token]
   // packed words (at most T * D * 2 / 32); before that, the key statistics' partial (min, max) pairs, two words per thread
   constexpr int NWBUF = (T * D * 2 / 32) > 2 * PACK_THREADS ? (T * D * 2 / 32) : 2 * PACK_THREADS;
   __shared__ __align__(16) uint32_t wbuf[NWBUF];
@@ -146,8 +157,7 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
         float z, sc;
         __half zh, sh;
         group_params(mn, mx, bits, eta, z, sc, zh, sh);
-        par_zi[item] = make_float2(z, rcp_or_zero(sc));
-        par_s[item] = sc;
+        par[item] = make_float4(z, safe_rcp(sc), sc, 0.f);
         const size_t grp = (size_t)bh * 2 * cap_g + (tq0 / G + gl);  // scale plane, then zero-point plane
         const int pos = k_meta_position(d, D);
         meta[grp * D + pos] = sh;
@@ -182,8 +192,7 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
         float z, sc;
         __half zh, sh;
         group_params(mn, mx, bits, eta, z, sc, zh, sh);
-        par_zi[gi * T + tl] = make_float2(z, rcp_or_zero(sc));
-        par_s[gi * T + tl] = sc;
+        par[gi * T + tl] = make_float4(z, safe_rcp(sc), sc, 0.f);
         const int tabs = tq0 + tl;
         const size_t t16 = (size_t)bh * (dm.nq_cap / 16) + tabs / 16;
         const int pos = v_meta_position(tabs % 16, gi, NG);
@@ -216,10 +225,10 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
 #pragma unroll
         for (int t = 0; t < NT; ++t) {
           const int tl = t * TPT + tt * 16 + row, gl = (t * TPT + tt * 16) / G;
-          const float4 zi = *reinterpret_cast<const float4*>(&par_zi[gl * D + d]);  // channels d, d + 1
+          const float4 p0 = par[gl * D + d], p1 = par[gl * D + d + 1];
           const uint32_t xx = *reinterpret_cast<const uint32_t*>(tile + tl * ROWB + d * 2);
-          word[t] |= code_pair<BITS>(__uint_as_float(xx << 16), __uint_as_float(xx & 0xffff0000u), zi.x, zi.y, zi.z, zi.w,
-                                     doubt[t]) << (BITS * slot);
+          word[t] |= code_pair<BITS>(__uint_as_float(xx << 16), __uint_as_float(xx & 0xffff0000u), p0, p1, doubt[t])
+                     << (BITS * slot);
         }
       }
     } else {
@@ -229,11 +238,11 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
 #pragma unroll
         for (int t = 0; t < NT; ++t) {
           const int tl = t * TPT + tt * 16 + col;  // tokens tl, tl + 1
-          const float4 zi = *reinterpret_cast<const float4*>(&par_zi[gi * T + tl]);
+          const float4 p0 = par[gi * T + tl], p1 = par[gi * T + tl + 1];
           const uint8_t* src = tile + tl * ROWB + d * 2;
           const float x0 = bf16_bits(*reinterpret_cast<const uint16_t*>(src));
           const float x1 = bf16_bits(*reinterpret_cast<const uint16_t*>(src + ROWB));
-          word[t] |= code_pair<BITS>(x0, x1, zi.x, zi.y, zi.z, zi.w, doubt[t]) << (BITS * slot);
+          word[t] |= code_pair<BITS>(x0, x1, p0, p1, doubt[t]) << (BITS * slot);
         }
       }
     }
@@ -248,13 +257,13 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
           if (kind == 0) {
             const int tl = t * TPT + tt * 16 + row, d = cb * 16 + col, g0 = ((t * TPT + tt * 16) / G) * D + d;
             const uint32_t xx = *reinterpret_cast<const uint32_t*>(tile + tl * ROWB + d * 2);
-            c0 = code_of(__uint_as_float(xx << 16), par_zi[g0].x, par_s[g0], QMAX);
-            c1 = code_of(__uint_as_float(xx & 0xffff0000u), par_zi[g0 + 1].x, par_s[g0 + 1], QMAX);
+            c0 = code_of(__uint_as_float(xx << 16), par[g0].x, par[g0].z, QMAX);
+            c1 = code_of(__uint_as_float(xx & 0xffff0000u), par[g0 + 1].x, par[g0 + 1].z, QMAX);
           } else {
             const int tl = t * TPT + tt * 16 + col, d = cb * 16 + row, g0 = ((cb * 16) / G) * T + tl;
             const uint8_t* src = tile + tl * ROWB + d * 2;
-            c0 = code_of(bf16_bits(*reinterpret_cast<const uint16_t*>(src)), par_zi[g0].x, par_s[g0], QMAX);
-            c1 = code_of(bf16_bits(*reinterpret_cast<const uint16_t*>(src + ROWB)), par_zi[g0 + 1].x, par_s[g0 + 1], QMAX);
+            c0 = code_of(bf16_bits(*reinterpret_cast<const uint16_t*>(src)), par[g0].x, par[g0].z, QMAX);
+            c1 = code_of(bf16_bits(*reinterpret_cast<const uint16_t*>(src + ROWB)), par[g0 + 1].x, par[g0 + 1].z, QMAX);
           }
           w |= (c0 | (c1 << 16)) << (BITS * slot);
         }

@@ -235,6 +235,44 @@ def test_decode_step_appends_inside_the_decode_kernel(kernel, oracle_tol):
                         util.check_attention(cache, oc, l, q[l], b, hk, o32[l], None, tol=short_context_tol)
 
 
+@pytest.mark.parametrize("bits", [(2, 2), (0, 0), (2, 0)])
+@pytest.mark.parametrize("D,g", [(128, 32), (128, 64), (64, 32)])
+def test_pack_on_lattice_data_with_exact_ties(bits, D, g):
+    """Inputs on a coarse lattice (small integers and halves, some groups constant, some spanning a power of two):
+    (x - z) / s falls exactly on rounding ties in a large share of the elements, where round-half-even decides
+    the code.  Codes, scales and zero-points against the oracle, bit for bit."""
+    L, B, Hkv, R = 2, 2, 2, 64
+    kq, vq = bits
+    S = 3 * R + 7
+    w = dict(n_layers=L, batch=B, n_q_heads=2 * Hkv, n_kv_heads=Hkv, head_dim=D, seq=S, residual_len=R,
+             group_size=g, kq=kq, vq=vq, km=0, vm=2, n_outliers=0, outlier_scale=1.0, seed=1, n_splits=0)
+    # (the wide channel makes logits of tens: the attention check uses the kernels that keep 2e-3 there)
+    cfg = W.make_xq_config(w, kernel=xq.XQ_KERNEL_GENERIC if D == 64 else xq.XQ_KERNEL_MMA_PRECISE)
+    cache = xq.Cache(cfg, DEV)
+    gen = torch.Generator().manual_seed(100 * D + g + kq)
+    kv = {}
+    for l in range(L):
+        K = torch.randint(-6, 7, (B, Hkv, S, D), generator=gen).float() * 0.5
+        V = torch.randint(-3, 4, (B, Hkv, S, D), generator=gen).float()
+        K[:, :, :, 5] = 2.0                      # constant key channel: scale 0, codes 0
+        V[:, :, 11, :] = -1.5                    # constant value token
+        K[:, :, :, 9] *= 64.0                    # a wide channel
+        V[:, :, 17, : D // 2] *= 0.03125         # a narrow group
+        kv[l] = (K.to(torch.bfloat16).to(DEV), V.to(torch.bfloat16).to(DEV))
+        for lo in range(0, S, 50):
+            cache.append_kv(l, kv[l][0][:, :, lo:lo + 50].contiguous(), kv[l][1][:, :, lo:lo + 50].contiguous())
+    torch.cuda.synchronize()
+    for l in range(L):
+        q = W.queries(w, l, 0, DEV)
+        o32 = cache.decode_attention(l, q, f32=True)
+        for b in range(B):
+            for hk in range(Hkv):
+                oc = util.oracle_for_stream(cfg, list(range(L)), b, hk, kv)
+                util.compare_regions(cache, oc, l, b, hk)
+                util.check_attention(cache, oc, l, q, b, hk, o32, None)
+    cache.close()
+
+
 @pytest.mark.parametrize("G,kernel", [(1, xq.XQ_KERNEL_AUTO), (1, xq.XQ_KERNEL_MMA_PRECISE), (2, xq.XQ_KERNEL_AUTO),
                                       (3, xq.XQ_KERNEL_MMA_PRECISE), (4, xq.XQ_KERNEL_MMA_PRECISE),
                                       (5, xq.XQ_KERNEL_AUTO), (8, xq.XQ_KERNEL_MMA)])
