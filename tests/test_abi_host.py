@@ -47,6 +47,10 @@ def test_config_check():
         assert xq.xq_equiv_bits(c) < 0
     # an odd kq is fine when the pair it cuts does not share codes
     assert xq.xq_config_check(_cfg(kq=31, km=32)) == xq.XQ_OK
+    # the precise tensor-core kernel: head_dim 128 and groups of at most four query heads only
+    assert xq.xq_config_check(_cfg(kernel=xq.XQ_KERNEL_MMA_PRECISE)) == xq.XQ_OK
+    assert xq.xq_config_check(_cfg(kernel=xq.XQ_KERNEL_MMA_PRECISE, n_kv_heads=4)) == xq.XQ_ERR_CONFIG
+    assert xq.xq_config_check(_cfg(kernel=xq.XQ_KERNEL_MMA_PRECISE, head_dim=64, residual_len=64)) == xq.XQ_ERR_CONFIG
 
 
 @pytest.mark.parametrize("kq,vq,km,vm", [(30, 2, 32, 16), (32, 0, 32, 16), (28, 0, 32, 28), (32, 0, 32, 20),
