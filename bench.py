@@ -30,7 +30,8 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "decode-attention GB/s at 32k ctx"
-APPEND_BLOCKS = 6  # window blocks quantized per layer in the append pass
+APPEND_BLOCKS = 6  # window blocks quantized per layer in the append pass, one block per call
+BULK_BLOCKS = 16   # then two calls per layer of this many blocks each (a prefill-sized append)
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the decode kernel (ncu, same launch shape as the
 # timed one; see profiles/).  Valid only for the kernel version the counters were taken on.
 NCU_TRAFFIC_BYTES = {"c2": 84.03e6 + 2.69e6}
@@ -211,7 +212,7 @@ def main():
     L, B, Hq, Hkv, D, S = w["n_layers"], w["batch"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"], w["seq"]
     K, Wm = args.steps, args.warmup
     R = w["residual_len"]
-    n_total = Wm + 3 * K + 8 + (APPEND_BLOCKS + 1) * R  # warm-up, three timed passes, then the append pass
+    n_total = Wm + 3 * K + 8 + (APPEND_BLOCKS + 1 + 2 * BULK_BLOCKS) * R  # warm-up, three timed passes, then the append pass
     cfg = W.make_xq_config(w, max_seq=S + n_total + 1, eta1=args.eta1, eta2=args.eta2, kernel=args.kernel,
                            n_splits=args.splits)
     cache = xq.Cache(cfg, dev)
@@ -344,12 +345,28 @@ def main():
     _, n_wapp, ms_wapp = xq.xq_timing_read(cache.handle, 3)
     xq.xq_timing_enable(cache.handle, 0)
     block_in_bytes = 2 * B * Hkv * R * D * 2  # 16-bit K and V of one block
+    # the same path at prefill size: BULK_BLOCKS window blocks per call (one pack launch each)
+    bulk = [torch.randn(B, Hkv, BULK_BLOCKS * R, D, generator=gk, device=dev).to(torch.bfloat16) for _ in range(3)]
+    xq.xq_timing_enable(cache.handle, 1)
+    barrier()
+    for i in range(2):
+        for l in range(L):
+            cache.append_kv(l, bulk[(i + l) % 3], bulk[(i + l + 1) % 3])
+    barrier()
+    _, n_bulk, ms_bulk = xq.xq_timing_read(cache.handle, 2)
+    xq.xq_timing_enable(cache.handle, 0)
+    del bulk
     append = {"block_tokens": R, "blocks_per_layer": APPEND_BLOCKS, "pack_launches": n_pack,
               "pack_avg_us": ms_pack / n_pack * 1e3 if n_pack else None,
               "pack_input_gbs": block_in_bytes / (ms_pack / n_pack * 1e-3) / 1e9 if n_pack else None,
               "pack_frac_of_measured_hbm": (block_in_bytes / (ms_pack / n_pack * 1e-3) / 1e9 / peak) if n_pack else None,
               "window_append_avg_us": ms_wapp / n_wapp * 1e3 if n_wapp else None,
-              "input_bytes_per_block": block_in_bytes}
+              "input_bytes_per_block": block_in_bytes,
+              "bulk": {"blocks_per_call": BULK_BLOCKS, "pack_launches": n_bulk,
+                       "pack_avg_us": ms_bulk / n_bulk * 1e3 if n_bulk else None,
+                       "pack_input_gbs": BULK_BLOCKS * block_in_bytes / (ms_bulk / n_bulk * 1e-3) / 1e9 if n_bulk else None,
+                       "pack_frac_of_measured_hbm": (BULK_BLOCKS * block_in_bytes / (ms_bulk / n_bulk * 1e-3) / 1e9 / peak)
+                       if n_bulk else None}}
 
     if rank == 0:
         nsq = nsw = None
