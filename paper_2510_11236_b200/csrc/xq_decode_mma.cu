@@ -482,15 +482,17 @@ __device__ __forceinline__ void ticket_merge(const DecodeParams& p, int ns, int 
   const Dims& dm = p.dm;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int bh = b * dm.Hkv + hk;
-  __threadfence();
+  // The CTA's barrier orders every thread's partial stores before thread 0's ticket; the ticket is a release
+  // (cumulative over what the barrier ordered) and an acquire at device scope, so the CTA that draws the last
+  // ticket sees all partials after its second barrier.  The partials are then read from L2 (ld.global.cg).
   __syncthreads();
   if (threadIdx.x == 0) {
-    unsigned t = atomicAdd(p.tickets + bh, 1u);
+    unsigned t;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;\n" : "=r"(t) : "l"(p.tickets + bh) : "memory");
     *s_flag = (t == (unsigned)(ns - 1));
   }
   __syncthreads();
   if (!*s_flag) return;
-  __threadfence();
   for (int a = warp; a < dm.G; a += MMA_WARPS) {
     const size_t hq = (size_t)b * dm.Hq + hk * dm.G + a;
     const float* ml = p.part_ml + hq * ns * 2;
