@@ -327,6 +327,8 @@ def main():
     ms3_max = sharding.max_over_ranks(ms3, dev)
     e2e_val = sharding.aggregate_rate(step_bytes(seq_before3 + 1, K), ms3_max, world) / 1e9
 
+    rc, nsq, nsw = xq.xq_split_plan(cache.handle, 0)  # the decode launches' split plan (before the appends below)
+
     # ---- pass 4: the quantize-and-pack path: every layer receives whole window blocks (R tokens per call), so each
     # ---- call quantizes and packs the block that filled the window (code-owning layers: codes + scale / zero-point;
     # ---- borrowing layers: scale / zero-point only)
@@ -369,8 +371,6 @@ def main():
                        if n_bulk else None}}
 
     if rank == 0:
-        nsq = nsw = None
-        rc, nsq, nsw = xq.xq_split_plan(cache.handle, 0)
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

@@ -199,7 +199,9 @@ double xq_equiv_bits(const xq_config* cfg);
 int xq_seq_len(const xq_cache* c, int layer);
 /* Of those, tokens in the quantized region (a multiple of residual_len). */
 int xq_quantized_len(const xq_cache* c, int layer);
-/* Splits (quantized-region, window) the next decode call on `layer` would use. */
+/* Splits per (sequence, kv head) stream (quantized-region, window) the next decode
+ * call on `layer` would use; where the library's own choice gives some streams one
+ * split more than others to fill the GPU, the larger number. */
 int xq_split_plan(const xq_cache* c, int layer, int* n_splits_quantized, int* n_splits_window);
 
 /* Where a layer's data lives inside the workspace, for tests and snapshots.

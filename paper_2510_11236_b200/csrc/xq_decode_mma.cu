@@ -430,7 +430,7 @@ __device__ __forceinline__ void window_tile(uint32_t wbuf, int n_valid, const ui
 // Combines warp states (rows of MS floats: mb has 8 rows per warp, ws has G rows
 // per warp; either may be absent) and writes the CTA's partial for each head.
 __device__ __forceinline__ void write_partial(const DecodeParams& p, const float* mb, const float* ws, int split,
-                                              int ns, int hk, int b) {
+                                              int stride, int hk, int b) {
   const Dims& dm = p.dm;
   const int d = threadIdx.x;  // MMA_THREADS == HD
   const int G = dm.G;
@@ -458,8 +458,8 @@ __device__ __forceinline__ void write_partial(const DecodeParams& p, const float
       }
     }
     size_t hq = (size_t)b * dm.Hq + hk * G + a;
-    p.part_acc[(hq * ns + split) * HD + d] = A;
-    if (d == 0) *reinterpret_cast<float2*>(p.part_ml + (hq * ns + split) * 2) = make_float2(M, Lsum);
+    p.part_acc[(hq * stride + split) * HD + d] = A;
+    if (d == 0) *reinterpret_cast<float2*>(p.part_ml + (hq * stride + split) * 2) = make_float2(M, Lsum);
   }
 }
 
@@ -478,7 +478,7 @@ __device__ __forceinline__ float4 ld_cg4(const float* p) {
 // its partials are visible device-wide; the CTA that draws the last ticket reads
 // all partials from L2 and writes out = sum_s acc_s 2^(m_s-M) / sum_s l_s 2^(m_s-M).
 // No CTA ever waits for another.
-__device__ __forceinline__ void ticket_merge(const DecodeParams& p, int ns, int hk, int b, int* s_flag) {
+__device__ __forceinline__ void ticket_merge(const DecodeParams& p, int ns, int stride, int hk, int b, int* s_flag) {
   const Dims& dm = p.dm;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int bh = b * dm.Hkv + hk;
@@ -495,8 +495,8 @@ __device__ __forceinline__ void ticket_merge(const DecodeParams& p, int ns, int 
   if (!*s_flag) return;
   for (int a = warp; a < dm.G; a += MMA_WARPS) {
     const size_t hq = (size_t)b * dm.Hq + hk * dm.G + a;
-    const float* ml = p.part_ml + hq * ns * 2;
-    const float* pa = p.part_acc + hq * ns * HD + lane * 4;
+    const float* ml = p.part_ml + hq * stride * 2;
+    const float* pa = p.part_acc + hq * stride * HD + lane * 4;
     // every load of a round is issued before anything waits for one: the merge costs one L2 round trip per 16
     // partials instead of one per partial
     float4 v[16];
@@ -670,14 +670,14 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
   float* ws = reinterpret_cast<float*>(smem);                  // window states of the window-only path
 
   const Dims& dm = p.dm;
-  const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gid = lane >> 2, tig = lane & 3;
   const int G = dm.G;
 
-  if (p.ns_q == 0) {  // nothing is quantized yet: window-only splits
+  if (p.ns_q == 0) {  // nothing is quantized yet: window-only splits, grid (splits, kv heads, sequences)
     grid_dependents_go();
     grid_dependency_wait();
+    const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int ns = p.ns_w;
     const int tiles = (p.r + 15) / 16;
     int t0, t1;
@@ -689,11 +689,32 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     window_tokens(p, t0, t1, hk, b, ws, wr);
     __syncthreads();
     write_partial(p, nullptr, ws, split, ns, hk, b);
-    ticket_merge(p, ns, hk, b, &s_flag);
+    ticket_merge(p, ns, ns, hk, b, &s_flag);
     return;
   }
 
-  const int ns = p.ns_q;
+  // Packed path: a one-dimensional grid of p.n_ctas CTAs dealt to the streams in order; the first
+  // n_ctas % streams streams get one split more than the others (the host only chooses such a count when the
+  // splits are many, so the CTAs' sizes differ by a few percent), which lets the grid fill every resident slot.
+  int split, ns, hk, b;
+  {
+    const unsigned n_streams = (unsigned)(dm.B * dm.Hkv), c = blockIdx.x;
+    const unsigned base = (unsigned)p.n_ctas / n_streams, rem = (unsigned)p.n_ctas - base * n_streams;
+    const unsigned big = rem * (base + 1u);
+    unsigned stream;
+    if (c < big) {
+      stream = c / (base + 1u);
+      split = (int)(c - stream * (base + 1u));
+      ns = (int)base + 1;
+    } else {
+      const unsigned c2 = c - big;
+      stream = rem + c2 / base;
+      split = (int)(c2 - (c2 / base) * base);
+      ns = (int)base;
+    }
+    hk = (int)(stream % (unsigned)dm.Hkv);
+    b = (int)(stream / (unsigned)dm.Hkv);
+  }
   const int units = p.n_q / 32;
   int u0, u1;
   share_of(units, ns, split, u0, u1);
@@ -983,8 +1004,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 3) decode_mma_kernel(DecodeParams
     }
   }
   __syncthreads();
-  write_partial(p, mb, nullptr, split, ns, hk, b);
-  ticket_merge(p, ns, hk, b, &s_flag);
+  write_partial(p, mb, nullptr, split, p.ns_q, hk, b);
+  ticket_merge(p, ns, p.ns_q, hk, b, &s_flag);
 }
 
 template <int BK, int BV, int GS>
@@ -1002,8 +1023,7 @@ cudaError_t launch_sp(const DecodeParams& p, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     configured = smem;
   }
-  const int ns = p.ns_q > 0 ? p.ns_q : p.ns_w;
-  dim3 grid(ns, p.dm.Hkv, p.dm.B);
+  const dim3 grid = p.ns_q > 0 ? dim3(p.n_ctas) : dim3(p.ns_w, p.dm.Hkv, p.dm.B);
   return launch_dependent(decode_mma_kernel<BK, BV, GS, SP, HP>, grid, dim3(MMA_THREADS), (size_t)smem, st, p);
 }
 

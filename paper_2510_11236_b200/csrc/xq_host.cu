@@ -197,7 +197,7 @@ int mma_ctas_per_sm(const xq_cache* c, int l) {
 // packed units and a share of the window (ns_w = 0 unless nothing is packed yet),
 // sized towards whole waves of resident CTAs.  Generic kernel: separate splits for
 // the packed region and for the window, in proportion to their bytes.
-void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w) {
+void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w, int* n_ctas_out = nullptr) {
   const Dims& dm = c->plan.dm;
   int S = c->seq[l];
   int r = residual_count(S, dm.R), nq = S - r;
@@ -214,6 +214,7 @@ void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w) {
     ns_w = 0;
     if (c->cfg.n_splits > 0) {
       ns_q = c->cfg.n_splits < units ? c->cfg.n_splits : units;
+      if (n_ctas_out) *n_ctas_out = ns_q * streams;
       return;
     }
     const double slots = (double)c->sm_count * mma_ctas_per_sm(c, l);
@@ -228,6 +229,15 @@ void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w) {
       if (score > best_score) { best_score = score; best = ns; }
     }
     ns_q = best;
+    if (n_ctas_out) *n_ctas_out = best * streams;
+    // One wave that does not fill every resident slot: give some streams one split more, if the splits are many
+    // enough for the CTAs' sizes to stay within a few percent of each other.
+    const long long slot_count = (long long)c->sm_count * mma_ctas_per_sm(c, l);
+    if ((long long)best * streams < slot_count && slot_count < (long long)(best + 1) * streams && best >= 8 &&
+        best + 1 <= units && best + 1 <= XQ_MAX_SPLITS) {
+      ns_q = best + 1;
+      if (n_ctas_out) *n_ctas_out = (int)slot_count;
+    }
     return;
   }
   double qb, wb;
@@ -308,7 +318,7 @@ int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, c
   p.q = (const uint16_t*)q;
   p.n_q = nq;
   p.r = r;
-  plan_splits(c, layer, p.ns_q, p.ns_w);
+  plan_splits(c, layer, p.ns_q, p.ns_w, &p.n_ctas);
   p.scale = c->scale;
   p.part_acc = (float*)(c->ws + c->plan.part_acc);
   p.part_ml = (float*)(c->ws + c->plan.part_ml);
@@ -507,7 +517,7 @@ int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out,
   p.q = (const uint16_t*)q;
   p.n_q = nq;
   p.r = r;
-  plan_splits(c, layer, p.ns_q, p.ns_w);
+  plan_splits(c, layer, p.ns_q, p.ns_w, &p.n_ctas);
   p.scale = c->scale;
   p.out = out;
   p.out_f32 = 0;

@@ -53,7 +53,8 @@ struct DecodeParams {
   const uint16_t* q;  // [B,Hq,D] bf16
   int n_q;            // quantized tokens
   int r;              // window tokens
-  int ns_q, ns_w;     // splits over the quantized region / over the window
+  int ns_q, ns_w;     // splits over the quantized region (most of any stream) / over the window
+  int n_ctas;         // tensor-core kernel, packed path: CTAs over all streams (n_ctas / streams or one more each)
   float scale;
   float* part_acc;    // [B,Hq,ns,D]
   float* part_ml;     // [B,Hq,ns,2]  (running max in log2 units, sum)
