@@ -53,20 +53,18 @@ extern "C" {
 #define XQ_ERR_ORDER (-4)    /* a code-borrowing layer is ahead of the layer owning codes */
 #define XQ_ERR_CUDA (-5)     /* a CUDA call failed; xq_last_cuda_error gives the code     */
 #define XQ_ERR_NOMEM (-6)    /* host allocation failed                                    */
+#define XQ_ERR_DEVICE (-7)   /* a kernel gave up a bounded wait (xq_check_device)         */
 
 #define XQ_BF16 0
 
 #define XQ_KERNEL_AUTO 0    /* tensor-core kernel when the shape allows it, else generic   */
 #define XQ_KERNEL_GENERIC 1 /* scalar kernel: any supported shape, slow, used as cross-check */
-#define XQ_KERNEL_MMA 2     /* tensor-core kernel: head_dim 128, group of <= 8 query heads  */
-/* The tensor-core kernel rounds the products q_d * s_d (query times key scale) to
- * fp16 before its matrix product: relative 2^-12 of every term of a logit.  Over
- * contexts with spread-out attention that stays far below 2e-3 in the result; a
- * query with very large logits on a few tokens (|logit| of tens) can see several
- * 1e-3.  This variant (head_dim 128, groups of <= 4 query heads) carries each
- * product as an fp16 pair (rounded value + what the rounding lost) and is about
- * 5 % slower. */
-#define XQ_KERNEL_MMA_PRECISE 3
+/* Tensor-core kernel (tcgen05, integer operands): head_dim 128, group of <= 8 query
+ * heads, layers that hold quantized tokens.  The products q_d * s_d (query times
+ * key scale) and p_t * s_t (softmax numerator times value scale) enter the matrix
+ * products as 21- and 23-bit fixed point relative to their largest member, the
+ * accumulation is exact (32-bit integers), everything else is fp32. */
+#define XQ_KERNEL_MMA 2
 
 #define XQ_MEM_DEVICE 0
 #define XQ_MEM_HOST 1
@@ -99,8 +97,8 @@ typedef struct xq_config {
 
 typedef struct xq_cache xq_cache; /* opaque; owns host memory only */
 
-/* Validates a configuration (rules above; head_dim % group_size == 0; with
- * head_dim 64 and a 1-bit layer, residual_len % 64 == 0).  XQ_OK or XQ_ERR_CONFIG. */
+/* Validates a configuration (rules above; head_dim % group_size == 0).
+ * XQ_OK or XQ_ERR_CONFIG. */
 int xq_config_check(const xq_config* cfg);
 
 /* Device bytes xq_create needs for `cfg`: windows, scale / zero-point, codes of
@@ -154,20 +152,24 @@ int xq_decode_attention_f32(xq_cache* c, int layer, const void* q, float* out, v
  * 16-byte aligned) but the split-K partials and merge tickets, which
  * xq_decode_attention keeps in the caller's workspace, live here in a
  * XQ_STATIC_SCRATCH_BYTES array that is part of the library image: every GPU
- * that loads the library holds that much device memory until the process exits.
- * The call allocates and frees nothing, on the host side of CUDA or through any
- * library.  Result: identical to xq_decode_attention.
+ * that the library's image is loaded on holds that much device memory until the
+ * process exits.  The call allocates and frees nothing, on the host side of CUDA
+ * or through any library.  Result: identical to xq_decode_attention.
  * Limits: the partials of the call (batch * n_q_heads * splits * (head_dim + 2)
- * floats, plus one ticket per (sequence, kv head)) must fit the array, else
+ * floats, plus one ticket per (sequence, kv head) and a status word) must fit the array, else
  * XQ_ERR_CAPACITY and nothing is launched; a smaller n_splits in xq_config
  * shrinks them.  The array is shared by every handle and every call on a device
  * and keeps the previous call's contents; the call clears the part that must
  * start at zero (the tickets) on `stream` before its kernel.  Two such calls
  * whose kernels may overlap on the GPU (different streams without an ordering
  * between them) race on the array: keep them on one stream or order them.
- * The first call on each device looks up the array's device address (a short
- * synchronous CUDA runtime query, no allocation); make that first call outside
- * any stream capture.  Other errors as xq_decode_attention. */
+ * xq_create looks up the array's device address (a short synchronous CUDA
+ * runtime query that also makes the driver place the library's image, the array
+ * included, on the device: create the handle at start-up, before the host fills
+ * its pools and outside any stream capture); the call itself only checks that
+ * the current device is the handle's (else XQ_ERR_ARG).  Unlike
+ * xq_decode_attention this call never fetches packed data ahead of the kernel
+ * that precedes it in the stream.  Other errors as xq_decode_attention. */
 #define XQ_STATIC_SCRATCH_BYTES (8u << 20)
 int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out, void* stream);
 
@@ -190,6 +192,13 @@ int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out,
 int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void* q, void* out,
                    const int32_t* layer_order, int mem, void* stream);
 
+/* Waits for `stream` and reports whether a kernel launched through this handle
+ * gave up one of its bounded waits (XQ_ERR_DEVICE; the outputs of that call are
+ * then invalid and the handle should be reset) -- every wait inside the kernels
+ * has an iteration limit instead of the ability to hang the GPU.  XQ_OK otherwise.
+ * Synchronizes; not for the hot path. */
+int xq_check_device(xq_cache* c, void* stream);
+
 /* Equivalent bit-width of Appendix C: stored code bits per cached element,
  * averaged over layers and over keys and values; scale / zero-point excluded,
  * a code-borrowing layer counts zero.  Negative if cfg is invalid. */
@@ -209,12 +218,16 @@ int xq_split_plan(const xq_cache* c, int layer, int* n_splits_quantized, int* n_
  * scale/zero, 3 value scale/zero, 4 key window, 5 value window.  Returns byte
  * offset from the workspace start and the byte stride between consecutive
  * (sequence, kv head) streams.
- * Layouts (all little-endian, one stream per (sequence, kv head)):
- *   codes: tiles of 128 uint32 (bit map: csrc/xq_layout.cuh);
- *   key scale/zero: [2][group capacity][head_dim] fp16 (all scale blocks, then all
- *     zero-point blocks; group capacity = stream_stride / (4 * head_dim)), permuted
- *     within a block; value scale/zero: per 16 tokens
- *     [2][16*head_dim/group_size] fp16; windows: [R][head_dim] bfloat16. */
+ * Layouts (all little-endian, one stream per (sequence, kv head); bit map and
+ * index functions: csrc/xq_layout.cuh):
+ *   key codes: per 32 tokens [chunk][token][<= 16 bytes] of the tokens' rows;
+ *   value codes: per 128 tokens [chunk][channel][16 bytes] of the channels' rows
+ *     (the words of a last, partly filled batch that no token has reached yet are
+ *     undefined);
+ *   key scale/zero: per token group [2][head_dim] fp16 (scales, then zero-points),
+ *     channel d at index (d % 32) * (head_dim / 32) + d / 32;
+ *   value scale/zero: per token [2][head_dim/group_size] fp16;
+ *   windows: [R][head_dim] bfloat16. */
 int xq_region(const xq_cache* c, int layer, int which, size_t* offset, size_t* stream_stride);
 
 /* Kernel launches issued through this handle since creation (all kinds). */

@@ -204,95 +204,107 @@ def merge_codes_weighted(e0: np.ndarray, e1: np.ndarray, gamma0: float) -> np.nd
 # --------------------------------------------------------------------------
 # Packed layouts (this build's choice; the paper does not discuss packing)
 # --------------------------------------------------------------------------
-# A code tile is 128 little-endian 32-bit words.  Each 16-bit half of a word is
-# cut into 16/bits slots of `bits` bits, slot 0 in the least significant bits.
-# D/16 channel blocks share the slots of a word; if slots remain, consecutive
-# 16-token sub-tiles fill them, so one tile spans 16 * (16/bits) / (D/16) tokens.
+# Words are little-endian 32-bit.  A byte of a word holds the codes of 8/bits
+# row elements, the four bytes of a word hold four consecutive row elements at
+# the same bit offset.  Keys: a row is one token (its D channels), rows are kept
+# in units of 32 tokens, each unit as chunks of at most 16 bytes per token.
+# Values: a row is one channel over a batch of 128 tokens, a batch is kept as
+# chunks of 16 bytes per channel.
 
-
-def tokens_per_code_tile(bits: int, D: int) -> int:
-    return 16 * ((16 // bits) // (D // 16))
+BATCH = 128  # tokens per value-code batch
 
 
 def k_code_position(t: int, d: int, bits: int, D: int):
     """(word index, bit offset) of key code (token t, channel d) in one (batch,
-    kv head) stream.  Within a 16x16 sub-block the token is the row and the
-    channel the column."""
-    cb_n = D // 16
-    tpt = tokens_per_code_tile(bits, D)
-    tile, tl = divmod(t, tpt)
-    tt, row = divmod(tl, 16)
-    cb, kk = divmod(d, 16)
-    lane = (row % 8) * 4 + (kk % 8) // 2
-    i = (row // 8) + 2 * (kk // 8)
-    slot = tt * cb_n + cb
-    return tile * 128 + lane * 4 + i, 16 * (kk % 2) + bits * slot
+    kv head) stream."""
+    n = 32 // bits                     # codes per word
+    word_in_row, e = divmod(d, n)      # e: element index inside the word
+    byte, step = e % 4, e // 4         # four consecutive channels share a bit offset
+    row_bytes = D * bits // 8
+    chunk_bytes = min(16, row_bytes)
+    chunk, off = divmod(4 * word_in_row, chunk_bytes)
+    unit, lane = divmod(t, 32)
+    addr = unit * 32 * row_bytes + chunk * 32 * chunk_bytes + lane * chunk_bytes + off
+    return addr // 4, 8 * byte + bits * step
 
 
 def v_code_position(t: int, d: int, bits: int, D: int):
-    """(word index, bit offset) of value code (token t, channel d): as for keys
-    with the roles swapped, the channel is the row and the token the column."""
-    cb_n = D // 16
-    tpt = tokens_per_code_tile(bits, D)
-    tile, tl = divmod(t, tpt)
-    tt, tk = divmod(tl, 16)
-    cb, cc = divmod(d, 16)
-    lane = (cc % 8) * 4 + (tk % 8) // 2
-    i = (cc // 8) + 2 * (tk // 8)
-    slot = tt * cb_n + cb
-    return tile * 128 + lane * 4 + i, 16 * (tk % 2) + bits * slot
+    """(word index, bit offset) of value code (token t, channel d): the channel
+    owns a row over the 128 tokens of a batch."""
+    n = 32 // bits
+    batch, tl = divmod(t, BATCH)
+    word_in_row, e = divmod(tl, n)
+    byte, step = e % 4, e // 4
+    chunk, w = divmod(word_in_row, 4)
+    addr = batch * D * 16 * bits + chunk * D * 16 + d * 16 + 4 * w
+    return addr // 4, 8 * byte + bits * step
 
 
-def _pack(codes: np.ndarray, bits: int, pos_fn) -> np.ndarray:
+def k_stream_words(T: int, bits: int, D: int) -> int:
+    """Words the key codes of T tokens occupy (T a multiple of 32)."""
+    return T * D * bits // 32
+
+
+def v_stream_words(T: int, bits: int, D: int) -> int:
+    """Words of the value-code batches that T tokens touch (whole batches)."""
+    return -(-T // BATCH) * D * 16 * bits // 4
+
+
+def _pack(codes: np.ndarray, bits: int, pos_fn, n_words: int):
+    """Returns (words, written): `written` marks the words that hold a code."""
     T, D = codes.shape
-    tpt = tokens_per_code_tile(bits, D)
-    assert T % tpt == 0
-    words = np.zeros((T // tpt) * 128, dtype=np.uint32)
+    words = np.zeros(n_words, dtype=np.uint32)
+    written = np.zeros(n_words, dtype=bool)
     for t in range(T):
         for d in range(D):
             w, b = pos_fn(t, d, bits, D)
             words[w] |= np.uint32(int(codes[t, d]) << b)
-    return words
-
-
-def _position_tables(T: int, D: int, bits: int, pos_fn):
-    w = np.empty((T, D), dtype=np.int64)
-    b = np.empty((T, D), dtype=np.int64)
-    for t in range(T):
-        for d in range(D):
-            w[t, d], b[t, d] = pos_fn(t, d, bits, D)
-    return w, b
+            written[w] = True
+    return words, written
 
 
 _TABLE_CACHE: dict = {}
 
 
-def _pack_fast(codes: np.ndarray, bits: int, pos_fn) -> np.ndarray:
-    """Same result as _pack; the (word, bit) table of one tile is built by calling
-    the position function for every element of that tile and then reused for
-    every tile (the position function is periodic in the tile by construction;
-    tests check _pack_fast == _pack)."""
+def _pack_fast(codes: np.ndarray, bits: int, pos_fn, n_words: int, period: int):
+    """Same result as _pack.  The position function repeats with `period` tokens
+    (32 for keys, 128 for values) up to a constant word offset per period; the
+    (word, bit) table of one period is built by calling it for every element of
+    the first period and the offset by calling it once more (tests check
+    _pack_fast == _pack)."""
     T, D = codes.shape
-    tpt = tokens_per_code_tile(bits, D)
-    assert T % tpt == 0
     key = (pos_fn.__name__, bits, D)
     if key not in _TABLE_CACHE:
-        _TABLE_CACHE[key] = _position_tables(tpt, D, bits, pos_fn)
-    w, b = _TABLE_CACHE[key]
-    n_tiles = T // tpt
-    c = codes.reshape(n_tiles, tpt, D).astype(np.uint32) << b.astype(np.uint32)[None]
-    words = np.zeros((n_tiles, 128), dtype=np.uint32)
-    for tile in range(n_tiles):
-        np.bitwise_or.at(words[tile], w.reshape(-1), c[tile].reshape(-1))
-    return words.reshape(-1)
+        w = np.empty((period, D), dtype=np.int64)
+        b = np.empty((period, D), dtype=np.int64)
+        for t in range(period):
+            for d in range(D):
+                w[t, d], b[t, d] = pos_fn(t, d, bits, D)
+        stride = pos_fn(period, 0, bits, D)[0] - pos_fn(0, 0, bits, D)[0]
+        _TABLE_CACHE[key] = (w, b, stride)
+    w, b, stride = _TABLE_CACHE[key]
+    words = np.zeros(n_words, dtype=np.uint32)
+    written = np.zeros(n_words, dtype=bool)
+    for p0 in range(0, T, period):
+        n = min(period, T - p0)
+        c = codes[p0:p0 + n].astype(np.uint32) << b[:n].astype(np.uint32)
+        idx = (w[:n] + (p0 // period) * stride).reshape(-1)
+        np.bitwise_or.at(words, idx, c.reshape(-1))
+        written[idx] = True
+    return words, written
 
 
-def pack_k_codes(codes: np.ndarray, bits: int, fast: bool = True) -> np.ndarray:
-    return (_pack_fast if fast else _pack)(codes, bits, k_code_position)
+def pack_k_codes(codes: np.ndarray, bits: int, fast: bool = True):
+    T, D = codes.shape
+    assert T % 32 == 0
+    n = k_stream_words(T, bits, D)
+    return _pack_fast(codes, bits, k_code_position, n, 32) if fast else _pack(codes, bits, k_code_position, n)
 
 
-def pack_v_codes(codes: np.ndarray, bits: int, fast: bool = True) -> np.ndarray:
-    return (_pack_fast if fast else _pack)(codes, bits, v_code_position)
+def pack_v_codes(codes: np.ndarray, bits: int, fast: bool = True):
+    T, D = codes.shape
+    n = v_stream_words(T, bits, D)
+    return _pack_fast(codes, bits, v_code_position, n, BATCH) if fast else _pack(codes, bits, v_code_position, n)
 
 
 def _unpack(words: np.ndarray, T: int, D: int, bits: int, pos_fn) -> np.ndarray:
@@ -314,46 +326,32 @@ def unpack_v_codes(words, T, D, bits):
 
 
 def k_meta_position(d: int, D: int) -> int:
-    """Index of channel d inside the D-entry scale (or zero-point) block of one
-    key token-group: 8-entry chunks, chunk 4*(d//32) + ((d%16)%8)//2, and inside
-    the chunk the entry ((d//16)%2)*4 + ((d%16)//8)*2 + d%2."""
-    cb, kk = divmod(d, 16)
-    chunk = (cb // 2) * 4 + (kk % 8) // 2
-    return chunk * 8 + (cb % 2) * 4 + (kk // 8) * 2 + (kk % 2)
+    """Index of channel d among the D scales (or the D zero-points) of one key
+    token group: channels d, d+32, d+64, ... are neighbours."""
+    return (d % 32) * (D // 32) + d // 32
 
 
 def pack_k_meta(s_hat: np.ndarray, z_hat: np.ndarray) -> np.ndarray:
-    """[n_groups, D] fp16 scale and zero -> uint16 [2, n_groups, D]: the plane of
-    permuted scale blocks, then the plane of permuted zero-point blocks."""
+    """[n_groups, D] fp16 scale and zero -> uint16 [n_groups, 2, D]: per token
+    group the permuted scales, then the permuted zero-points."""
     n, D = s_hat.shape
-    out = np.zeros((2, n, D), dtype=np.uint16)
+    out = np.zeros((n, 2, D), dtype=np.uint16)
     su = s_hat.astype(np.float16).view(np.uint16)
     zu = z_hat.astype(np.float16).view(np.uint16)
     for d in range(D):
         p = k_meta_position(d, D)
-        out[0, :, p] = su[:, d]
-        out[1, :, p] = zu[:, d]
+        out[:, 0, p] = su[:, d]
+        out[:, 1, p] = zu[:, d]
     return out
 
 
-def v_meta_position(tk: int, gi: int, n_g: int) -> int:
-    """Index of (token tk of a 16-token tile, channel group gi) inside the
-    16*n_g-entry scale (or zero-point) block of that tile."""
-    return ((tk % 8) // 2) * (n_g * 4) + gi * 4 + (tk // 8) * 2 + (tk % 2)
-
-
 def pack_v_meta(s_hat: np.ndarray, z_hat: np.ndarray) -> np.ndarray:
-    """[T, n_g] fp16 scale and zero -> uint16 [T/16, 2, 16*n_g]."""
+    """[T, n_g] fp16 scale and zero -> uint16 [T, 2, n_g]: per token its n_g
+    scales, then its n_g zero-points."""
     T, n_g = s_hat.shape
-    assert T % 16 == 0
-    out = np.zeros((T // 16, 2, 16 * n_g), dtype=np.uint16)
-    su = s_hat.astype(np.float16).view(np.uint16).reshape(T // 16, 16, n_g)
-    zu = z_hat.astype(np.float16).view(np.uint16).reshape(T // 16, 16, n_g)
-    for tk in range(16):
-        for gi in range(n_g):
-            p = v_meta_position(tk, gi, n_g)
-            out[:, 0, p] = su[:, tk, gi]
-            out[:, 1, p] = zu[:, tk, gi]
+    out = np.zeros((T, 2, n_g), dtype=np.uint16)
+    out[:, 0, :] = s_hat.astype(np.float16).view(np.uint16)
+    out[:, 1, :] = z_hat.astype(np.float16).view(np.uint16)
     return out
 
 

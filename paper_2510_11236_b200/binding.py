@@ -14,9 +14,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libxq.so")
 
 XQ_OK = 0
-XQ_ERR_CONFIG, XQ_ERR_ARG, XQ_ERR_CAPACITY, XQ_ERR_ORDER, XQ_ERR_CUDA, XQ_ERR_NOMEM = -1, -2, -3, -4, -5, -6
+XQ_ERR_CONFIG, XQ_ERR_ARG, XQ_ERR_CAPACITY, XQ_ERR_ORDER, XQ_ERR_CUDA, XQ_ERR_NOMEM, XQ_ERR_DEVICE = -1, -2, -3, -4, -5, -6, -7
 XQ_BF16 = 0
-XQ_KERNEL_AUTO, XQ_KERNEL_GENERIC, XQ_KERNEL_MMA, XQ_KERNEL_MMA_PRECISE = 0, 1, 2, 3
+XQ_KERNEL_AUTO, XQ_KERNEL_GENERIC, XQ_KERNEL_MMA = 0, 1, 2
 XQ_MEM_DEVICE, XQ_MEM_HOST = 0, 1
 XQ_MAX_SPLITS = 256
 XQ_STATIC_SCRATCH_BYTES = 8 << 20
@@ -51,6 +51,7 @@ _SIGNATURES = {
     "xq_decode_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                       ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.c_int,
                                       ctypes.c_void_p]),
+    "xq_check_device": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "xq_equiv_bits": (ctypes.c_double, [ctypes.POINTER(xq_config)]),
     "xq_seq_len": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
     "xq_quantized_len": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
@@ -148,6 +149,10 @@ def xq_decode_step(handle, K_new, V_new, q, out, layer_order=None, mem: int = XQ
     if layer_order is not None:
         order = (ctypes.c_int32 * len(layer_order))(*layer_order)
     return lib().xq_decode_step(handle, _ptr(K_new), _ptr(V_new), _ptr(q), _ptr(out), order, mem, stream)
+
+
+def xq_check_device(handle, stream: int = 0) -> int:
+    return lib().xq_check_device(handle, stream)
 
 
 def xq_equiv_bits(cfg: xq_config) -> float:
@@ -264,6 +269,11 @@ class Cache:
         if rc:
             raise XQError(rc, "xq_decode_step")
         return out
+
+    def check_device(self):
+        rc = xq_check_device(self.handle, self._stream())
+        if rc:
+            raise XQError(rc, "xq_check_device")
 
     def seq_len(self, layer):
         return xq_seq_len(self.handle, layer)

@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(GEN_WARPS * 32) decode_generic_kernel(DecodePa
   const uint32_t* kc = p.L.k_codes + (size_t)bh * ((size_t)dm.nq_cap * D * bk / 32);
   const uint32_t* vc = p.L.v_codes + (size_t)bh * ((size_t)dm.nq_cap * D * bv / 32);
   const uint16_t* km = p.L.k_meta + (size_t)bh * (dm.nq_cap / g) * 2 * D;
-  const uint16_t* vm = p.L.v_meta + (size_t)bh * (dm.nq_cap / 16) * 2 * 16 * NG;
+  const uint16_t* vm = p.L.v_meta + (size_t)bh * dm.nq_cap * 2 * NG;
   const uint16_t* wk = p.L.win_k + (size_t)bh * dm.R * D;
   const uint16_t* wv = p.L.win_v + (size_t)bh * dm.R * D;
   const float scale2 = p.scale * 1.4426950408889634f;
@@ -81,14 +81,12 @@ __global__ void __launch_bounds__(GEN_WARPS * 32) decode_generic_kernel(DecodePa
         if (quant) {
           CodePos pk = k_code_position(t, d, bk, D);
           float c = (float)((kc[pk.word] >> pk.bit) & ((1u << bk) - 1));
-          const uint16_t* mk = km + (size_t)(t / g) * D;  // scale plane; the zero-point plane follows it
+          const uint16_t* mk = km + (size_t)(t / g) * 2 * D;  // the group's D scales, then its D zero-points
           int pos = k_meta_position(d, D);
-          kx[j] = fmaf(c, f16_bits_f(mk[pos]), f16_bits_f(mk[(size_t)(dm.nq_cap / g) * D + pos]));
+          kx[j] = fmaf(c, f16_bits_f(mk[pos]), f16_bits_f(mk[D + pos]));
           CodePos pv = v_code_position(t, d, bv, D);
           float cv = (float)((vc[pv.word] >> pv.bit) & ((1u << bv) - 1));
-          const uint16_t* mv = vm + (size_t)(t / 16) * 2 * 16 * NG;
-          int vpos = v_meta_position(t % 16, d / g, NG);
-          vx[j] = fmaf(cv, f16_bits_f(mv[vpos]), f16_bits_f(mv[16 * NG + vpos]));
+          vx[j] = fmaf(cv, f16_bits_f(vm[v_scale_index(t, d / g, NG)]), f16_bits_f(vm[v_zero_index(t, d / g, NG)]));
         } else {
           kx[j] = bf16_bits_f(wk[(size_t)t * D + d]);
           vx[j] = bf16_bits_f(wv[(size_t)t * D + d]);

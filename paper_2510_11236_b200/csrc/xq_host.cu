@@ -5,7 +5,6 @@
 #include <stdlib.h>
 #include <string.h>
 
-#include <mutex>
 #include <new>
 #include <vector>
 
@@ -30,7 +29,7 @@ struct LayerRegions {
 struct Plan {
   Dims dm;
   std::vector<LayerRegions> layers;
-  size_t part_acc, part_ml, tickets, staging, total;
+  size_t part_acc, part_ml, tickets, status, staging, total;
   size_t staging_kv_bytes, staging_q_bytes;
 };
 
@@ -50,10 +49,7 @@ bool check(const xq_config* c) {
   if (!(c->sm_scale >= 0.f) || isinf(c->sm_scale)) return false;
   if (c->n_splits < 0 || c->n_splits > XQ_MAX_SPLITS) return false;
   if (c->io_dtype != XQ_BF16) return false;
-  if (c->kernel < XQ_KERNEL_AUTO || c->kernel > XQ_KERNEL_MMA_PRECISE) return false;
-  if (c->kernel == XQ_KERNEL_MMA_PRECISE && (c->head_dim != 128 || c->n_q_heads / c->n_kv_heads > 4)) return false;
-  bool any_1bit = c->kq < c->n_layers || c->vq < c->n_layers;
-  if (c->head_dim == 64 && any_1bit && c->residual_len % 64) return false;
+  if (c->kernel < XQ_KERNEL_AUTO || c->kernel > XQ_KERNEL_MMA) return false;
   // both layers of a sharing pair must have the same bit-width
   for (int l = 1; l < c->n_layers; l += 2) {
     if (!owns_codes(l, c->km) && layer_bits(l, c->kq) != layer_bits(l - 1, c->kq)) return false;
@@ -66,7 +62,8 @@ void make_plan(const xq_config* c, Plan& pl) {
   Dims& dm = pl.dm;
   dm.B = c->batch; dm.Hq = c->n_q_heads; dm.Hkv = c->n_kv_heads; dm.G = dm.Hq / dm.Hkv;
   dm.D = c->head_dim; dm.g = c->group_size; dm.R = c->residual_len; dm.NG = dm.D / dm.g;
-  dm.nq_cap = c->max_seq > 1 ? ((c->max_seq - 1) / dm.R) * dm.R : 0;
+  // quantized tokens never exceed ((max_seq - 1) / R) * R; the regions hold whole 128-token batches
+  dm.nq_cap = padded_capacity(c->max_seq > 1 ? ((c->max_seq - 1) / dm.R) * dm.R : 0);
   const size_t BH = (size_t)dm.B * dm.Hkv;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
@@ -78,7 +75,7 @@ void make_plan(const xq_config* c, Plan& pl) {
     r.win_k = take(BH * r.stride[4]);
     r.win_v = take(BH * r.stride[5]);
     r.stride[2] = (size_t)(dm.nq_cap / dm.g) * 2 * dm.D * 2;
-    r.stride[3] = (size_t)(dm.nq_cap / 16) * 2 * 16 * dm.NG * 2;
+    r.stride[3] = (size_t)dm.nq_cap * 2 * dm.NG * 2;
     r.k_meta = take(BH * r.stride[2]);
     r.v_meta = take(BH * r.stride[3]);
     r.stride[0] = (size_t)dm.nq_cap * dm.D * bk / 8;
@@ -89,6 +86,7 @@ void make_plan(const xq_config* c, Plan& pl) {
   pl.part_acc = take((size_t)dm.B * dm.Hq * XQ_MAX_SPLITS * dm.D * 4);
   pl.part_ml = take((size_t)dm.B * dm.Hq * XQ_MAX_SPLITS * 2 * 4);
   pl.tickets = take(BH * 4);
+  pl.status = take(4);
   pl.staging_kv_bytes = (size_t)c->n_layers * BH * dm.D * 2;
   pl.staging_q_bytes = (size_t)c->n_layers * dm.B * dm.Hq * dm.D * 2;
   pl.staging = take(2 * align_up(pl.staging_kv_bytes, 256) + 2 * align_up(pl.staging_q_bytes, 256));
@@ -110,25 +108,14 @@ static __device__ __align__(256) unsigned char g_static_scratch[XQ_STATIC_SCRATC
 
 namespace {
 
-constexpr int STATIC_MAX_DEVICES = 64;
-std::mutex g_static_mutex;
-uint8_t* g_static_address[STATIC_MAX_DEVICES] = {};
-
-// Device address of g_static_scratch on the current device; looked up once per device.
+// Device address of g_static_scratch on the current device (a synchronous runtime query that also makes the
+// driver load this module's image, array included, on that device).
 cudaError_t static_scratch_address(uint8_t** out) {
-  int dev = -1;
-  cudaError_t e = cudaGetDevice(&dev);
+  void* p = nullptr;
+  cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
   if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= STATIC_MAX_DEVICES) return cudaErrorInvalidDevice;
-  std::lock_guard<std::mutex> lock(g_static_mutex);
-  if (!g_static_address[dev]) {
-    void* p = nullptr;
-    e = cudaGetSymbolAddress(&p, g_static_scratch);
-    if (e != cudaSuccess) return e;
-    if (!p || ((uintptr_t)p & 255)) return cudaErrorInvalidSymbol;
-    g_static_address[dev] = (uint8_t*)p;
-  }
-  *out = g_static_address[dev];
+  if (!p || ((uintptr_t)p & 255)) return cudaErrorInvalidSymbol;
+  *out = (uint8_t*)p;
   return cudaSuccess;
 }
 
@@ -143,6 +130,8 @@ struct xq_cache {
   int last_cuda;
   float scale;
   int sm_count;
+  int device;            // CUDA device the handle was created on (-1: none)
+  uint8_t* static_base;  // device address of the library's static scratch array on that device (null: not resolved)
   bool tickets_clean;  // the ticket counters have been zeroed on a stream
   std::vector<uint8_t> repacked;  // per layer: codes or parameters it reads were written since its last decode
   int mma_ctas[2][2];  // resident CTAs per SM of the tensor-core kernel by (key bits - 1, value bits - 1); 0 = not asked yet
@@ -188,53 +177,47 @@ int mma_ctas_per_sm(const xq_cache* c, int l) {
   int& slot = const_cast<xq_cache*>(c)->mma_ctas[bk - 1][bv - 1];
   if (slot == 0) {
     slot = decode_mma_ctas_per_sm(c->plan.dm, bk, bv);
-    if (slot <= 0) slot = 3;  // no device to ask
+    if (slot <= 0) slot = 2;  // no device to ask
   }
   return slot;
 }
 
-// Splits per (sequence, kv head) stream.  Tensor-core kernel: every split takes
-// packed units and a share of the window (ns_w = 0 unless nothing is packed yet),
-// sized towards whole waves of resident CTAs.  Generic kernel: separate splits for
-// the packed region and for the window, in proportion to their bytes.
+// Splits per (sequence, kv head) stream.  Tensor-core kernel (layers with quantized
+// tokens): every split takes whole batches of the packed region and a share of the
+// window (ns_w = 0), sized towards whole waves of resident CTAs.  Generic kernel:
+// separate splits for the packed region and for the window, in proportion to their bytes.
 void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w, int* n_ctas_out = nullptr) {
   const Dims& dm = c->plan.dm;
   int S = c->seq[l];
   int r = residual_count(S, dm.R), nq = S - r;
   int units = nq / 32, tiles = (r + 15) / 16;
   const int streams = dm.B * dm.Hkv;
-  if (layer_uses_mma(c, l)) {
-    if (units == 0) {
-      ns_q = 0;
-      ns_w = c->cfg.n_splits > 0 ? c->cfg.n_splits : 4;
-      if (ns_w > tiles) ns_w = tiles;
-      if (ns_w < 1) ns_w = 1;
-      return;
-    }
+  if (layer_uses_mma(c, l) && nq > 0) {
+    // the tensor-core kernel: whole 128-token batches per CTA, every CTA also takes a share of the window
+    const int batches = (nq + XQ_BATCH - 1) / XQ_BATCH;
     ns_w = 0;
     if (c->cfg.n_splits > 0) {
-      ns_q = c->cfg.n_splits < units ? c->cfg.n_splits : units;
+      ns_q = c->cfg.n_splits < batches ? c->cfg.n_splits : batches;
       if (n_ctas_out) *n_ctas_out = ns_q * streams;
       return;
     }
-    const double slots = (double)c->sm_count * mma_ctas_per_sm(c, l);
+    const long long slot_count = (long long)c->sm_count * mma_ctas_per_sm(c, l);
     int best = 1;
     double best_score = -1.0;
-    for (int ns = 1; ns <= 64 && ns <= units; ++ns) {
+    for (int ns = 1; ns <= XQ_MAX_SPLITS && ns <= batches; ++ns) {
       double ctas = (double)ns * streams;
-      double waves = ceil(ctas / slots);
-      double fill = ctas / (waves * slots);
-      double upc = (double)units / ns;          // units per CTA
-      double score = fill * upc / (upc + 12.0);  // ~12 units' worth of fixed cost per CTA
+      double waves = ceil(ctas / (double)slot_count);
+      double fill = ctas / (waves * (double)slot_count);
+      double bpc = (double)batches / ns;         // batches per CTA
+      double score = fill * bpc / (bpc + 5.0);   // ~5 batches' worth of fixed cost per CTA
       if (score > best_score) { best_score = score; best = ns; }
     }
     ns_q = best;
     if (n_ctas_out) *n_ctas_out = best * streams;
     // One wave that does not fill every resident slot: give some streams one split more, if the splits are many
     // enough for the CTAs' sizes to stay within a few percent of each other.
-    const long long slot_count = (long long)c->sm_count * mma_ctas_per_sm(c, l);
     if ((long long)best * streams < slot_count && slot_count < (long long)(best + 1) * streams && best >= 8 &&
-        best + 1 <= units && best + 1 <= XQ_MAX_SPLITS) {
+        best + 1 <= batches && best + 1 <= XQ_MAX_SPLITS) {
       ns_q = best + 1;
       if (n_ctas_out) *n_ctas_out = (int)slot_count;
     }
@@ -291,84 +274,130 @@ struct Timer {
 
 int fail_cuda(xq_cache* c, cudaError_t e) { c->last_cuda = (int)e; return XQ_ERR_CUDA; }
 
-// K_new / V_new: one new token per stream that the tensor-core kernel appends itself (see append_fuses); the
-// layer's length already counts it.
-int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, cudaStream_t st,
-                const void* K_new = nullptr, const void* V_new = nullptr) {
+// Where the split-K partials, the merge tickets and the kernel status word of a decode call live.
+struct Scratch {
+  float* part_acc;
+  float* part_ml;
+  unsigned int* tickets;
+  int* status;
+};
+
+// Checks a decode call and fills the kernel parameters (everything but the scratch).  Touches no state.
+// K_new / V_new: one new token per stream that the tensor-core kernel appends itself; S_eff is the layer's
+// length with that token counted.
+int prepare_decode(const xq_cache* c, int layer, const void* q, void* out, int out_f32, const void* K_new,
+                   const void* V_new, int S_eff, DecodeParams& p, bool& use_mma) {
   if (!c || !q || !out) return XQ_ERR_ARG;
   if (layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
   if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return XQ_ERR_ARG;
+  if (((uintptr_t)K_new & 15) || ((uintptr_t)V_new & 15)) return XQ_ERR_ARG;
   const Dims& dm = c->plan.dm;
-  int S = c->seq[layer];
+  const int S = S_eff;
   if (S < 1) return XQ_ERR_ARG;
-  int r = residual_count(S, dm.R), nq = S - r;
+  const int r = residual_count(S, dm.R), nq = S - r;
   // a code-borrowing layer needs the owning layer's codes for all of its quantized tokens
-  bool bor_k = !owns_codes(layer, c->cfg.km), bor_v = !owns_codes(layer, c->cfg.vm);
-  if (bor_k || bor_v) {
-    int So = c->seq[layer - 1];
-    int nqo = So - residual_count(So, dm.R);
-    if (nqo < nq) return XQ_ERR_ORDER;
+  if (!owns_codes(layer, c->cfg.km) || !owns_codes(layer, c->cfg.vm)) {
+    const int So = c->seq[layer - 1];
+    if (So - residual_count(So, dm.R) < nq) return XQ_ERR_ORDER;
   }
-  DecodeParams p;
-  p.early_fetch = 0;
-  p.K_new = p.V_new = nullptr;
-  p.precise = 0;
+  use_mma = layer_uses_mma(c, layer) && nq > 0;
+  if (c->cfg.kernel >= XQ_KERNEL_MMA && !layer_uses_mma(c, layer)) return XQ_ERR_CONFIG;
+  if (K_new && !use_mma) return XQ_ERR_ARG;
   p.dm = dm;
   p.L = layer_ptrs(c, layer);
   p.q = (const uint16_t*)q;
   p.n_q = nq;
   p.r = r;
-  plan_splits(c, layer, p.ns_q, p.ns_w, &p.n_ctas);
+  p.n_ctas = 0;
+  {
+    // plan_splits reads the layer's length from the handle: give it the effective one
+    xq_cache* cc = const_cast<xq_cache*>(c);
+    const int keep = cc->seq[layer];
+    cc->seq[layer] = S;
+    plan_splits(c, layer, p.ns_q, p.ns_w, &p.n_ctas);
+    cc->seq[layer] = keep;
+  }
   p.scale = c->scale;
-  p.part_acc = (float*)(c->ws + c->plan.part_acc);
-  p.part_ml = (float*)(c->ws + c->plan.part_ml);
-  bool use_mma = layer_uses_mma(c, layer);
-  if (c->cfg.kernel >= XQ_KERNEL_MMA && !use_mma) return XQ_ERR_CONFIG;
   p.out = out;
   p.out_f32 = out_f32;
-  p.tickets = (unsigned int*)(c->ws + c->plan.tickets);
+  p.early_fetch = 0;
   p.K_new = (const uint16_t*)K_new;
   p.V_new = (const uint16_t*)V_new;
-  p.precise = c->cfg.kernel == XQ_KERNEL_MMA_PRECISE;
-  if (K_new && !(use_mma && nq > 0)) return XQ_ERR_ARG;
+  return XQ_OK;
+}
+
+// Launches a prepared decode call.  The tensor-core kernel merges its partials itself.
+int launch_decode(xq_cache* c, DecodeParams& p, bool use_mma, const Scratch& s, cudaStream_t st) {
+  p.part_acc = s.part_acc;
+  p.part_ml = s.part_ml;
+  p.tickets = s.tickets;
+  p.status = s.status;
   cudaError_t e;
-  if (use_mma) {
-    if (!c->tickets_clean) {
-      e = cudaMemsetAsync(p.tickets, 0, (size_t)dm.B * dm.Hkv * 4, st);
-      if (e != cudaSuccess) return fail_cuda(c, e);
-      c->tickets_clean = true;
-    }
-    // the packed streams may be fetched ahead of the preceding kernel unless a pack kernel wrote them since
-    // this layer's last decode (then that kernel may be the writer, or only just behind it)
-    p.early_fetch = c->repacked[layer] ? 0 : 1;
-    c->repacked[layer] = 0;
-    {
-      Timer t(c, st, 0);
-      e = launch_decode_mma(p, st);  // merges the partials itself
-    }
-    c->launches++;
-    if (e != cudaSuccess) { c->tickets_clean = false; return fail_cuda(c, e); }
-    return XQ_OK;
-  }
   {
     Timer t(c, st, 0);
-    e = launch_decode_generic(p, st);
+    e = use_mma ? launch_decode_mma(p, st) : launch_decode_generic(p, st);
   }
   c->launches++;
   if (e != cudaSuccess) return fail_cuda(c, e);
+  if (use_mma) return XQ_OK;
   MergeParams m;
-  m.dm = dm;
+  m.dm = p.dm;
   m.ns = p.ns_q + p.ns_w;
   m.part_acc = p.part_acc;
   m.part_ml = p.part_ml;
-  m.out = out;
-  m.out_f32 = out_f32;
+  m.out = p.out;
+  m.out_f32 = p.out_f32;
   {
     Timer t(c, st, 1);
     e = launch_merge(m, st);
   }
   c->launches++;
   if (e != cudaSuccess) return fail_cuda(c, e);
+  return XQ_OK;
+}
+
+Scratch workspace_scratch(const xq_cache* c) {
+  Scratch s;
+  s.part_acc = (float*)(c->ws + c->plan.part_acc);
+  s.part_ml = (float*)(c->ws + c->plan.part_ml);
+  s.tickets = (unsigned int*)(c->ws + c->plan.tickets);
+  s.status = (int*)(c->ws + c->plan.status);
+  return s;
+}
+
+// The ticket counters and the status word start at zero: cleared once per handle on the first stream used.
+int ensure_clean_scratch(xq_cache* c, cudaStream_t st) {
+  if (c->tickets_clean) return XQ_OK;
+  const Dims& dm = c->plan.dm;
+  cudaError_t e = cudaMemsetAsync(c->ws + c->plan.tickets, 0, (size_t)dm.B * dm.Hkv * 4, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + c->plan.status, 0, 4, st);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->tickets_clean = true;
+  return XQ_OK;
+}
+
+int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, cudaStream_t st,
+                const void* K_new = nullptr, const void* V_new = nullptr) {
+  if (!c) return XQ_ERR_ARG;
+  if (layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
+  DecodeParams p;
+  bool use_mma = false;
+  int rc = prepare_decode(c, layer, q, out, out_f32, K_new, V_new, c->seq[layer] + (K_new ? 1 : 0), p, use_mma);
+  if (rc != XQ_OK) return rc;
+  if (use_mma) {
+    rc = ensure_clean_scratch(c, st);
+    if (rc != XQ_OK) return rc;
+    // the packed streams may be fetched ahead of the preceding kernel unless a pack kernel wrote them since
+    // this layer's last decode (then that kernel may be the writer, or only just behind it)
+    p.early_fetch = c->repacked[layer] ? 0 : 1;
+  }
+  rc = launch_decode(c, p, use_mma, workspace_scratch(c), st);
+  if (rc != XQ_OK) {
+    if (use_mma) c->tickets_clean = false;
+    return rc;
+  }
+  if (use_mma) c->repacked[layer] = 0;
+  if (K_new) c->seq[layer] += 1;
   return XQ_OK;
 }
 
@@ -405,13 +434,23 @@ int xq_create(const xq_config* cfg, void* dev_workspace, size_t bytes, xq_cache*
   c->used = 0;
   c->sm_count = 148;
   c->tickets_clean = false;
+  c->device = -1;
+  c->static_base = nullptr;
   memset(c->mma_ctas, 0, sizeof(c->mma_ctas));
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) == cudaSuccess &&
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
     c->sm_count = sms;
-  else
-    cudaGetLastError();  // no device (host-only use of the handle): keep the default
+    c->device = dev;
+    // Set-up, not the hot path: the address of the static scratch array of xq_decode_attention_static.  The query
+    // makes the driver place the library's image (the array included) on this device now.
+    if (static_scratch_address(&c->static_base) != cudaSuccess) {
+      cudaGetLastError();
+      c->static_base = nullptr;
+    }
+  } else {
+    cudaGetLastError();  // no device (host-only use of the handle): keep the defaults
+  }
   *out = c;
   return XQ_OK;
 }
@@ -426,6 +465,8 @@ int xq_destroy(xq_cache* c) {
 int xq_reset(xq_cache* c) {
   if (!c) return XQ_ERR_ARG;
   for (auto& s : c->seq) s = 0;
+  for (auto& r : c->repacked) r = 1;  // as after xq_create: the first decode of a layer waits for its predecessor
+  c->tickets_clean = false;           // tickets and status are cleared again before their next use
   return XQ_OK;
 }
 
@@ -450,11 +491,7 @@ int xq_append_kv(xq_cache* c, int layer, const void* K, const void* V, int n_tok
     p.own_k = owns_codes(layer, c->cfg.km); p.own_v = owns_codes(layer, c->cfg.vm);
     p.eta_k = L.bk == 1 ? c->cfg.eta1 : c->cfg.eta2;
     p.eta_v = L.bv == 1 ? c->cfg.eta1 : c->cfg.eta2;
-    // tokens per CTA: whole key groups and whole code tiles of both kinds; the
-    // configuration check makes the window a multiple of 64 whenever this is 64
-    p.tb = dm.g > 32 ? dm.g : 32;
-    if (tokens_per_code_tile(L.bk, dm.D) > p.tb) p.tb = tokens_per_code_tile(L.bk, dm.D);
-    if (tokens_per_code_tile(L.bv, dm.D) > p.tb) p.tb = tokens_per_code_tile(L.bv, dm.D);
+    p.tb = dm.g > 32 ? dm.g : 32;  // tokens per CTA: whole key groups, whole words of either kind
     cudaError_t e;
     {
       Timer t(c, st, 2);
@@ -494,98 +531,67 @@ int xq_decode_attention_f32(xq_cache* c, int layer, const void* q, float* out, v
 }
 
 int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out, void* stream) {
-  if (!c || !q || !out) return XQ_ERR_ARG;
+  if (!c) return XQ_ERR_ARG;
   if (layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
-  if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return XQ_ERR_ARG;
   cudaStream_t st = (cudaStream_t)stream;
-  const Dims& dm = c->plan.dm;
-  const int S = c->seq[layer];
-  if (S < 1) return XQ_ERR_ARG;
-  const int r = residual_count(S, dm.R), nq = S - r;
-  if (!owns_codes(layer, c->cfg.km) || !owns_codes(layer, c->cfg.vm)) {
-    const int So = c->seq[layer - 1];
-    if (So - residual_count(So, dm.R) < nq) return XQ_ERR_ORDER;
-  }
-  const bool use_mma = layer_uses_mma(c, layer);
-  if (c->cfg.kernel >= XQ_KERNEL_MMA && !use_mma) return XQ_ERR_CONFIG;
   DecodeParams p;
-  p.early_fetch = 0;
-  p.K_new = p.V_new = nullptr;
-  p.precise = c->cfg.kernel == XQ_KERNEL_MMA_PRECISE;
-  p.dm = dm;
-  p.L = layer_ptrs(c, layer);
-  p.q = (const uint16_t*)q;
-  p.n_q = nq;
-  p.r = r;
-  plan_splits(c, layer, p.ns_q, p.ns_w, &p.n_ctas);
-  p.scale = c->scale;
-  p.out = out;
-  p.out_f32 = 0;
-  // carve the static array: [partial accumulators | partial (max, sum) | tickets]
+  bool use_mma = false;
+  int rc = prepare_decode(c, layer, q, out, 0, nullptr, nullptr, c->seq[layer], p, use_mma);
+  if (rc != XQ_OK) return rc;
+  // the array belongs to the device the handle was created on
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return fail_cuda(c, cudaGetLastError());
+  if (dev != c->device) return XQ_ERR_ARG;
+  if (!c->static_base) return fail_cuda(c, cudaErrorInvalidSymbol);
+  // carve the static array: [partial accumulators | partial (max, sum) | tickets | status]
+  const Dims& dm = c->plan.dm;
   const size_t ns = (size_t)p.ns_q + (size_t)p.ns_w;
   const size_t acc_bytes = align_up((size_t)dm.B * dm.Hq * ns * dm.D * 4, 256);
   const size_t ml_bytes = align_up((size_t)dm.B * dm.Hq * ns * 2 * 4, 256);
-  const size_t ticket_bytes = (size_t)dm.B * dm.Hkv * 4;
-  if (acc_bytes + ml_bytes + ticket_bytes > (size_t)XQ_STATIC_SCRATCH_BYTES) return XQ_ERR_CAPACITY;
-  uint8_t* base = nullptr;
-  cudaError_t e = static_scratch_address(&base);
-  if (e != cudaSuccess) return fail_cuda(c, e);
-  p.part_acc = (float*)base;
-  p.part_ml = (float*)(base + acc_bytes);
-  p.tickets = (unsigned int*)(base + acc_bytes + ml_bytes);
+  const size_t ticket_bytes = align_up((size_t)dm.B * dm.Hkv * 4, 256);
+  if (acc_bytes + ml_bytes + ticket_bytes + 256 > (size_t)XQ_STATIC_SCRATCH_BYTES) return XQ_ERR_CAPACITY;
+  Scratch s;
+  s.part_acc = (float*)c->static_base;
+  s.part_ml = (float*)(c->static_base + acc_bytes);
+  s.tickets = (unsigned int*)(c->static_base + acc_bytes + ml_bytes);
+  s.status = (int*)(c->static_base + acc_bytes + ml_bytes + ticket_bytes);
   if (use_mma) {
-    // the array keeps whatever the previous call (of any handle) left: tickets must start at zero
-    e = cudaMemsetAsync(p.tickets, 0, ticket_bytes, st);
+    // the array keeps whatever the previous call (of any handle) left: tickets and status must start at zero
+    cudaError_t e = cudaMemsetAsync(s.tickets, 0, ticket_bytes + 256, st);
     if (e != cudaSuccess) return fail_cuda(c, e);
-    {
-      Timer t(c, st, 0);
-      e = launch_decode_mma(p, st);
-    }
-    c->launches++;
-    if (e != cudaSuccess) return fail_cuda(c, e);
-    return XQ_OK;
   }
-  {
-    Timer t(c, st, 0);
-    e = launch_decode_generic(p, st);
-  }
-  c->launches++;
-  if (e != cudaSuccess) return fail_cuda(c, e);
-  MergeParams m;
-  m.dm = dm;
-  m.ns = (int)ns;
-  m.part_acc = p.part_acc;
-  m.part_ml = p.part_ml;
-  m.out = out;
-  m.out_f32 = 0;
-  {
-    Timer t(c, st, 1);
-    e = launch_merge(m, st);
-  }
-  c->launches++;
-  if (e != cudaSuccess) return fail_cuda(c, e);
-  return XQ_OK;
+  return launch_decode(c, p, use_mma, s, st);  // early_fetch stays 0: this call never fetches ahead of its predecessor
 }
 
 int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void* q, void* out,
                    const int32_t* layer_order, int mem, void* stream) {
   if (!c || !K_new || !V_new || !q || !out) return XQ_ERR_ARG;
   if (mem != XQ_MEM_DEVICE && mem != XQ_MEM_HOST) return XQ_ERR_ARG;
-  if (layer_order) {
-    std::vector<char> seen(c->cfg.n_layers, 0);
-    for (int i = 0; i < c->cfg.n_layers; ++i) {
-      int l = layer_order[i];
-      if (l < 0 || l >= c->cfg.n_layers || seen[l]) return XQ_ERR_ARG;
-      bool borrows = !owns_codes(l, c->cfg.km) || !owns_codes(l, c->cfg.vm);
-      if (borrows && !seen[l - 1]) return XQ_ERR_ORDER;
+  if (mem == XQ_MEM_DEVICE &&
+      (((uintptr_t)K_new & 15) || ((uintptr_t)V_new & 15) || ((uintptr_t)q & 15) || ((uintptr_t)out & 15)))
+    return XQ_ERR_ARG;
+  const Dims& dm = c->plan.dm;
+  const int L = c->cfg.n_layers;
+  // Everything that can be refused is checked before the first copy or launch, on a copy of the layer lengths
+  // advanced in processing order, so that a refused call leaves the cache as it was.
+  {
+    std::vector<char> seen(L, 0);
+    std::vector<int> len(c->seq);
+    for (int i = 0; i < L; ++i) {
+      const int l = layer_order ? layer_order[i] : i;
+      if (l < 0 || l >= L || seen[l]) return XQ_ERR_ARG;
       seen[l] = 1;
+      if (len[l] + 1 > c->cfg.max_seq) return XQ_ERR_CAPACITY;
+      len[l] += 1;
+      if (!owns_codes(l, c->cfg.km) || !owns_codes(l, c->cfg.vm)) {
+        if (!seen[l - 1]) return XQ_ERR_ORDER;
+        const int nq = len[l] - residual_count(len[l], dm.R), nqo = len[l - 1] - residual_count(len[l - 1], dm.R);
+        if (nqo < nq) return XQ_ERR_ORDER;
+      }
+      if (c->cfg.kernel >= XQ_KERNEL_MMA && !layer_uses_mma(c, l)) return XQ_ERR_CONFIG;
     }
   }
   cudaStream_t st = (cudaStream_t)stream;
-  const Dims& dm = c->plan.dm;
-  const int L = c->cfg.n_layers;
-  for (int l = 0; l < L; ++l)
-    if (c->seq[l] + 1 > c->cfg.max_seq) return XQ_ERR_CAPACITY;
   const size_t kv_layer = (size_t)dm.B * dm.Hkv * dm.D * 2;
   const size_t q_layer = (size_t)dm.B * dm.Hq * dm.D * 2;
   const uint8_t *dk = (const uint8_t*)K_new, *dv = (const uint8_t*)V_new, *dq = (const uint8_t*)q;
@@ -600,6 +606,7 @@ int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void
     if (e != cudaSuccess) return fail_cuda(c, e);
     dk = sk; dv = sv; dq = sq; dout = so;
   }
+  // Only a CUDA error can stop the loop below (the cache is then in an undefined state, as after any XQ_ERR_CUDA).
   for (int i = 0; i < L; ++i) {
     const int l = layer_order ? layer_order[i] : i;
     // One token that neither fills a window block nor is the layer's first quantized step goes into the window
@@ -608,9 +615,7 @@ int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void
     const int nq_old = s_old - residual_count(s_old, dm.R), nq_new = s_old + 1 - residual_count(s_old + 1, dm.R);
     int rc;
     if (nq_new == nq_old && nq_old > 0 && layer_uses_mma(c, l)) {
-      c->seq[l] = s_old + 1;
       rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st, dk + l * kv_layer, dv + l * kv_layer);
-      if (rc != XQ_OK) c->seq[l] = s_old;
     } else {
       rc = xq_append_kv(c, l, dk + l * kv_layer, dv + l * kv_layer, 1, stream);
       if (rc != XQ_OK) return rc;
@@ -623,6 +628,17 @@ int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void
     if (e != cudaSuccess) return fail_cuda(c, e);
   }
   return XQ_OK;
+}
+
+int xq_check_device(xq_cache* c, void* stream) {
+  if (!c) return XQ_ERR_ARG;
+  cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (!c->tickets_clean) return XQ_OK;  // the status word has not been used yet
+  int status = 0;
+  e = cudaMemcpy(&status, c->ws + c->plan.status, 4, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  return status ? XQ_ERR_DEVICE : XQ_OK;
 }
 
 double xq_equiv_bits(const xq_config* cfg) {
@@ -712,6 +728,7 @@ const char* xq_strerror(int code) {
     case XQ_ERR_ORDER: return "code-owning layer is behind the layer that borrows its codes";
     case XQ_ERR_CUDA: return "CUDA error (see xq_last_cuda_error)";
     case XQ_ERR_NOMEM: return "out of host memory";
+    case XQ_ERR_DEVICE: return "a kernel gave up a bounded wait (results of that call are invalid)";
     default: return "unknown error";
   }
 }

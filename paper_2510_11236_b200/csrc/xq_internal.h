@@ -7,15 +7,15 @@ namespace xq {
 
 struct Dims {
   int B, Hq, Hkv, G, D, g, R, NG;
-  int nq_cap;  // capacity of the quantized region in tokens (multiple of R)
+  int nq_cap;  // capacity of the quantized region in tokens, padded to whole 128-token batches
 };
 
 // Device addresses of one layer's regions (codes: of the layer that owns them).
 struct LayerPtrs {
   uint16_t* win_k;   // [B,Hkv,R,D] bf16
   uint16_t* win_v;
-  uint16_t* k_meta;  // [B,Hkv,2,nq_cap/g,D] fp16 (scale plane, zero-point plane)
-  uint16_t* v_meta;  // [B,Hkv,nq_cap/16,2,16*NG] fp16
+  uint16_t* k_meta;  // [B,Hkv,nq_cap/g,2,D] fp16 (per token group: scales, then zero-points)
+  uint16_t* v_meta;  // [B,Hkv,nq_cap,2,NG] fp16 (per token: scales, then zero-points)
   uint32_t* k_codes; // [B,Hkv,nq_cap*D*bk/32]
   uint32_t* v_codes;
   int bk, bv;
@@ -54,7 +54,7 @@ struct DecodeParams {
   int n_q;            // quantized tokens
   int r;              // window tokens
   int ns_q, ns_w;     // splits over the quantized region (most of any stream) / over the window
-  int n_ctas;         // tensor-core kernel, packed path: CTAs over all streams (n_ctas / streams or one more each)
+  int n_ctas;         // tensor-core kernel: CTAs over all streams (n_ctas / streams splits per stream, or one more)
   float scale;
   float* part_acc;    // [B,Hq,ns,D]
   float* part_ml;     // [B,Hq,ns,2]  (running max in log2 units, sum)
@@ -70,7 +70,7 @@ struct DecodeParams {
   // window holds that row reads it from here and stores it into the window.
   const uint16_t* K_new;
   const uint16_t* V_new;
-  int precise;  // tensor-core kernel, groups of <= 4 query heads: carry q_d s_d as an fp16 pair (XQ_KERNEL_MMA_PRECISE)
+  int* status;  // device word the tensor-core kernel sets when one of its bounded waits gave up
 };
 
 struct MergeParams {

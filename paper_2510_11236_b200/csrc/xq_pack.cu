@@ -59,7 +59,7 @@ __device__ __forceinline__ float safe_rcp(float s) {
 // rint(q') is the code the division gives, ties included.  Adding 1.5 * 2^23 rounds to the nearest integer, ties
 // to even, and leaves it in the low mantissa bits; 0 <= a / s < 2^B - 1/2 holds for every member of the group, so
 // no clamp is needed.  A NaN reciprocal sets `doubt` and the caller recomputes the word with the division.
-// Returns code(x0) | code(x1) << 16.
+// Returns code(x0) | code(x1) << 8: two neighbouring bytes of a packed word.
 template <int BITS>
 __device__ __forceinline__ uint32_t code_pair(float x0, float x1, const float4& p0, const float4& p1, bool& doubt) {
   const float a0 = __fsub_rn(x0, p0.x), a1 = __fsub_rn(x1, p1.x);
@@ -70,13 +70,14 @@ __device__ __forceinline__ uint32_t code_pair(float x0, float x1, const float4& 
   const float u0 = __fadd_rn(q0, PACK_MAGIC), u1 = __fadd_rn(q1, PACK_MAGIC);
   doubt |= (p0.y != p0.y) | (p1.y != p1.y);
   constexpr uint32_t QM = (1u << BITS) - 1u;
-  return __byte_perm(__float_as_uint(u0), __float_as_uint(u1), 0x0400) & (QM | (QM << 16));
+  return __byte_perm(__float_as_uint(u0), __float_as_uint(u1), 0x0040) & (QM | (QM << 8));
 }
 
 // One CTA: T tokens x D channels of one (sequence, kv head), keys (blockIdx.x even) or values (odd).  Staged
-// rows are padded; the statistics and the codes read them without bank conflicts; thread (lane, i) builds word
-// 4 * lane + i of every code tile of the CTA, the words are collected in shared memory and leave in 16-byte
-// vectors.  G: group size; T = p.tb: a multiple of G and of both kinds' tokens per code tile.
+// rows are padded.  Keys: a thread builds whole words of a token's row (four consecutive channels per bit
+// offset), the words are collected in shared memory in stream order and leave in 16-byte vectors.  Values: a
+// thread builds whole words of a channel's row over the tile's tokens and stores them itself.
+// G: group size; T = p.tb: a multiple of G and of 32.
 template <int D, int G, int T>
 __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
   constexpr int ROWB = D * 2 + PACK_ROW_PAD;
@@ -158,10 +159,10 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
         __half zh, sh;
         group_params(mn, mx, bits, eta, z, sc, zh, sh);
         par[item] = make_float4(z, safe_rcp(sc), sc, 0.f);
-        const size_t grp = (size_t)bh * 2 * cap_g + (tq0 / G + gl);  // scale plane, then zero-point plane
+        const size_t grp = (size_t)bh * cap_g + (tq0 / G + gl);  // per group: D scales, then D zero-points
         const int pos = k_meta_position(d, D);
-        meta[grp * D + pos] = sh;
-        meta[(grp + cap_g) * D + pos] = zh;
+        meta[grp * 2 * D + pos] = sh;
+        meta[grp * 2 * D + D + pos] = zh;
       }
     }
   } else {
@@ -194,92 +195,96 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
         group_params(mn, mx, bits, eta, z, sc, zh, sh);
         par[gi * T + tl] = make_float4(z, safe_rcp(sc), sc, 0.f);
         const int tabs = tq0 + tl;
-        const size_t t16 = (size_t)bh * (dm.nq_cap / 16) + tabs / 16;
-        const int pos = v_meta_position(tabs % 16, gi, NG);
-        meta[(t16 * 2 + 0) * (16 * NG) + pos] = sh;
-        meta[(t16 * 2 + 1) * (16 * NG) + pos] = zh;
+        __half* mine = meta + (size_t)bh * dm.nq_cap * 2 * NG;
+        mine[v_scale_index(tabs, gi, NG)] = sh;
+        mine[v_zero_index(tabs, gi, NG)] = zh;
       }
     }
   }
   if (!own) return;  // PseudoQuantize: parameters only
   __syncthreads();
 
-  // codes: thread (lane, i) = word 4 * lane + i of every tile: rows (lane / 4) + 8 (i % 2), columns 2 (lane % 4) +
-  // 8 (i / 2) and the next one of each 16 x 16 block (keys: row = token, column = channel; values: the reverse)
-  const int lane = tid & 31, i = tid >> 5;
-  const int row = (lane >> 2) + 8 * (i & 1), col = 2 * (lane & 3) + 8 * (i >> 1);
-  auto build = [&](auto bits_c) {
-    constexpr int BITS = decltype(bits_c)::value;
-    constexpr int NSLOT = 16 / BITS;
-    constexpr int TPT = 16 * (NSLOT / CB);
-    constexpr int NT = T >= TPT ? T / TPT : 1;  // code tiles of the CTA (the host never launches a T below TPT)
-    constexpr float QMAX = (float)((1 << BITS) - 1);
-    uint32_t word[NT];
-    bool doubt[NT];
-#pragma unroll
-    for (int t = 0; t < NT; ++t) { word[t] = 0u; doubt[t] = false; }
-    if (kind == 0) {
-#pragma unroll
-      for (int slot = 0; slot < NSLOT; ++slot) {
-        const int tt = slot / CB, cb = slot % CB, d = cb * 16 + col;
-#pragma unroll
-        for (int t = 0; t < NT; ++t) {
-          const int tl = t * TPT + tt * 16 + row, gl = (t * TPT + tt * 16) / G;
-          const float4 p0 = par[gl * D + d], p1 = par[gl * D + d + 1];
-          const uint32_t xx = *reinterpret_cast<const uint32_t*>(tile + tl * ROWB + d * 2);
-          word[t] |= code_pair<BITS>(__uint_as_float(xx << 16), __uint_as_float(xx & 0xffff0000u), p0, p1, doubt[t])
-                     << (BITS * slot);
-        }
-      }
-    } else {
-#pragma unroll
-      for (int slot = 0; slot < NSLOT; ++slot) {
-        const int tt = slot / CB, cb = slot % CB, d = cb * 16 + row, gi = (cb * 16) / G;
-#pragma unroll
-        for (int t = 0; t < NT; ++t) {
-          const int tl = t * TPT + tt * 16 + col;  // tokens tl, tl + 1
-          const float4 p0 = par[gi * T + tl], p1 = par[gi * T + tl + 1];
-          const uint8_t* src = tile + tl * ROWB + d * 2;
-          const float x0 = bf16_bits(*reinterpret_cast<const uint16_t*>(src));
-          const float x1 = bf16_bits(*reinterpret_cast<const uint16_t*>(src + ROWB));
-          word[t] |= code_pair<BITS>(x0, x1, p0, p1, doubt[t]) << (BITS * slot);
-        }
-      }
-    }
-#pragma unroll
-    for (int t = 0; t < NT; ++t) {
-      if (doubt[t]) {  // rare: the word again, with the division
-        uint32_t w = 0u;
-#pragma unroll 1
-        for (int slot = 0; slot < NSLOT; ++slot) {
-          const int tt = slot / CB, cb = slot % CB;
-          uint32_t c0, c1;
-          if (kind == 0) {
-            const int tl = t * TPT + tt * 16 + row, d = cb * 16 + col, g0 = ((t * TPT + tt * 16) / G) * D + d;
-            const uint32_t xx = *reinterpret_cast<const uint32_t*>(tile + tl * ROWB + d * 2);
-            c0 = code_of(__uint_as_float(xx << 16), par[g0].x, par[g0].z, QMAX);
-            c1 = code_of(__uint_as_float(xx & 0xffff0000u), par[g0 + 1].x, par[g0 + 1].z, QMAX);
-          } else {
-            const int tl = t * TPT + tt * 16 + col, d = cb * 16 + row, g0 = ((cb * 16) / G) * T + tl;
-            const uint8_t* src = tile + tl * ROWB + d * 2;
-            c0 = code_of(bf16_bits(*reinterpret_cast<const uint16_t*>(src)), par[g0].x, par[g0].z, QMAX);
-            c1 = code_of(bf16_bits(*reinterpret_cast<const uint16_t*>(src + ROWB)), par[g0 + 1].x, par[g0 + 1].z, QMAX);
-          }
-          w |= (c0 | (c1 << 16)) << (BITS * slot);
-        }
-        word[t] = w;
-      }
-      wbuf[t * 128 + lane * 4 + i] = word[t];
-    }
-    return NT * 128;
-  };
-  const int n_words = (bits == 2) ? build(std::integral_constant<int, 2>{}) : build(std::integral_constant<int, 1>{});
-  __syncthreads();
-
+  // codes
   uint32_t* codes = kind ? p.L.v_codes : p.L.k_codes;
   const size_t stream_words = (size_t)dm.nq_cap * D * bits / 32;
-  uint4* dst = reinterpret_cast<uint4*>(codes + (size_t)bh * stream_words + (size_t)(tq0 / 32) * (D * bits));
-  for (int v = tid; v < n_words / 4; v += PACK_THREADS) dst[v] = reinterpret_cast<const uint4*>(wbuf)[v];
+  auto build = [&](auto bits_c) {
+    constexpr int BITS = decltype(bits_c)::value;
+    constexpr int N = 32 / BITS;        // codes per word
+    constexpr float QMAX = (float)((1 << BITS) - 1);
+    if (kind == 0) {
+      constexpr int NW = D * BITS / 32;  // words per token row
+      const size_t w0 = k_code_position(tq0, 0, BITS, D).word;  // the tile's words are one contiguous run
+#pragma unroll
+      for (int k = 0; k < (T * NW + PACK_THREADS - 1) / PACK_THREADS; ++k) {
+        const int item = tid + k * PACK_THREADS;
+        if (item < T * NW) {
+          const int tl = item % T, i = item / T, gl = tl / G;
+          const uint8_t* row = tile + tl * ROWB;
+          uint32_t word = 0u;
+          bool doubt = false;
+#pragma unroll
+          for (int s4 = 0; s4 < N / 4; ++s4) {
+            const int d = i * N + 4 * s4;
+            const uint2 xx = *reinterpret_cast<const uint2*>(row + d * 2);
+            const float4 p0 = par[gl * D + d], p1 = par[gl * D + d + 1], p2 = par[gl * D + d + 2], p3 = par[gl * D + d + 3];
+            const uint32_t lo = code_pair<BITS>(__uint_as_float(xx.x << 16), __uint_as_float(xx.x & 0xffff0000u), p0, p1, doubt);
+            const uint32_t hi = code_pair<BITS>(__uint_as_float(xx.y << 16), __uint_as_float(xx.y & 0xffff0000u), p2, p3, doubt);
+            word |= (lo | (hi << 16)) << (BITS * s4);
+          }
+          if (doubt) {  // rare: the word again, with the division
+            word = 0u;
+#pragma unroll 1
+            for (int e = 0; e < N; ++e) {
+              const int d = i * N + (e / 4) * 4 + (e % 4);
+              const float4 pp = par[gl * D + d];
+              const uint32_t c = code_of(bf16_bits(*reinterpret_cast<const uint16_t*>(row + d * 2)), pp.x, pp.z, QMAX);
+              word |= c << (8 * (e % 4) + BITS * (e / 4));
+            }
+          }
+          wbuf[k_code_position(tq0 + tl, i * N, BITS, D).word - w0] = word;
+        }
+      }
+      __syncthreads();
+      uint4* dst = reinterpret_cast<uint4*>(codes + (size_t)bh * stream_words + w0);
+      for (int v = tid; v < T * NW / 4; v += PACK_THREADS) dst[v] = reinterpret_cast<const uint4*>(wbuf)[v];
+    } else {
+      constexpr int WPC = T / N;  // words per channel over the tile's tokens
+#pragma unroll
+      for (int k = 0; k < (D * WPC + PACK_THREADS - 1) / PACK_THREADS; ++k) {
+        const int item = tid + k * PACK_THREADS;
+        if (item < D * WPC) {
+          const int d = item % D, wi = item / D, gi = d / G;
+          uint32_t word = 0u;
+          bool doubt = false;
+#pragma unroll
+          for (int s4 = 0; s4 < N / 4; ++s4) {
+            const int tl = wi * N + 4 * s4;
+            const uint8_t* src = tile + tl * ROWB + d * 2;
+            const float4 p0 = par[gi * T + tl], p1 = par[gi * T + tl + 1], p2 = par[gi * T + tl + 2], p3 = par[gi * T + tl + 3];
+            const float x0 = bf16_bits(*reinterpret_cast<const uint16_t*>(src));
+            const float x1 = bf16_bits(*reinterpret_cast<const uint16_t*>(src + ROWB));
+            const float x2 = bf16_bits(*reinterpret_cast<const uint16_t*>(src + 2 * ROWB));
+            const float x3 = bf16_bits(*reinterpret_cast<const uint16_t*>(src + 3 * ROWB));
+            const uint32_t lo = code_pair<BITS>(x0, x1, p0, p1, doubt);
+            const uint32_t hi = code_pair<BITS>(x2, x3, p2, p3, doubt);
+            word |= (lo | (hi << 16)) << (BITS * s4);
+          }
+          if (doubt) {
+            word = 0u;
+#pragma unroll 1
+            for (int e = 0; e < N; ++e) {
+              const int tl = wi * N + (e / 4) * 4 + (e % 4);
+              const float4 pp = par[gi * T + tl];
+              const uint32_t c = code_of(bf16_bits(*reinterpret_cast<const uint16_t*>(tile + tl * ROWB + d * 2)), pp.x, pp.z, QMAX);
+              word |= c << (8 * (e % 4) + BITS * (e / 4));
+            }
+          }
+          codes[(size_t)bh * stream_words + v_code_position(tq0 + wi * N, d, BITS, D).word] = word;
+        }
+      }
+    }
+  };
+  if (bits == 2) build(std::integral_constant<int, 2>{}); else build(std::integral_constant<int, 1>{});
 }
 
 cudaError_t launch_pack(const PackParams& p, cudaStream_t st) {
@@ -288,10 +293,8 @@ cudaError_t launch_pack(const PackParams& p, cudaStream_t st) {
   const int key = p.dm.D * 10000 + p.dm.g * 100 + p.tb;
   switch (key) {
     case 1283232: pack_kernel<128, 32, 32><<<grid, PACK_THREADS, 0, st>>>(p); break;
-    case 1283264: pack_kernel<128, 32, 64><<<grid, PACK_THREADS, 0, st>>>(p); break;
     case 1286464: pack_kernel<128, 64, 64><<<grid, PACK_THREADS, 0, st>>>(p); break;
     case 643232: pack_kernel<64, 32, 32><<<grid, PACK_THREADS, 0, st>>>(p); break;
-    case 643264: pack_kernel<64, 32, 64><<<grid, PACK_THREADS, 0, st>>>(p); break;
     case 646464: pack_kernel<64, 64, 64><<<grid, PACK_THREADS, 0, st>>>(p); break;
     default: return cudaErrorInvalidValue;
   }

@@ -38,8 +38,7 @@ def test_config_check():
     bad = [dict(head_dim=96), dict(group_size=48), dict(residual_len=48), dict(n_q_heads=30),
            dict(eta1=0.6), dict(eta2=-0.1), dict(kq=33), dict(km=-1), dict(n_splits=1000),
            dict(residual_len=32, group_size=64), dict(max_seq=0), dict(kernel=9),
-           dict(kq=31, km=0),  # pair (30, 31) would mix 2-bit and 1-bit keys on shared codes
-           dict(head_dim=64, residual_len=32, vq=0)]
+           dict(kq=31, km=0)]  # pair (30, 31) would mix 2-bit and 1-bit keys on shared codes
     for kw in bad:
         c = _cfg(**kw)
         assert xq.xq_config_check(c) == xq.XQ_ERR_CONFIG, kw
@@ -47,10 +46,8 @@ def test_config_check():
         assert xq.xq_equiv_bits(c) < 0
     # an odd kq is fine when the pair it cuts does not share codes
     assert xq.xq_config_check(_cfg(kq=31, km=32)) == xq.XQ_OK
-    # the precise tensor-core kernel: head_dim 128 and groups of at most four query heads only
-    assert xq.xq_config_check(_cfg(kernel=xq.XQ_KERNEL_MMA_PRECISE)) == xq.XQ_OK
-    assert xq.xq_config_check(_cfg(kernel=xq.XQ_KERNEL_MMA_PRECISE, n_kv_heads=4)) == xq.XQ_ERR_CONFIG
-    assert xq.xq_config_check(_cfg(kernel=xq.XQ_KERNEL_MMA_PRECISE, head_dim=64, residual_len=64)) == xq.XQ_ERR_CONFIG
+    assert xq.xq_config_check(_cfg(kernel=xq.XQ_KERNEL_MMA)) == xq.XQ_OK
+    assert xq.xq_config_check(_cfg(head_dim=64, residual_len=32, vq=0)) == xq.XQ_OK
 
 
 @pytest.mark.parametrize("kq,vq,km,vm", [(30, 2, 32, 16), (32, 0, 32, 16), (28, 0, 32, 28), (32, 0, 32, 20),
