@@ -56,14 +56,12 @@ namespace {
 
 constexpr int HD = 128;
 constexpr int BT = 128;          // tokens per batch
-constexpr int CT = 128;          // compute threads = tensor-memory lanes
-constexpr int W_MMA = 4, W_TMA = 5, W_WIN = 6;
-constexpr int UTHREADS = 224;
 constexpr int NSTG = 4;          // staged batches
 constexpr int TAU = 3;           // log2 units a logit may exceed the softmax reference before it is raised
 constexpr int MREF = 2;          // a raised reference sits this far below the (rounded-up) largest logit
 constexpr int FRAC_V = 23 - TAU; // fraction bits of the value-side fixed point
-constexpr int WAIT_LIMIT = 1 << 20;
+constexpr int WAIT_LIMIT = 1 << 20;     // polls of a wait before it gives up
+constexpr uint32_t WAIT_HINT_NS = 10000;  // longest suspension of one poll (it ends at once when the phase completes)
 constexpr float MAGIC_V = 8388608.0f;              // 2^23: x + MAGIC_V holds rint(x) in its mantissa, 0 <= x < 2^23
 constexpr float MAGIC_K = 8388608.0f + 1228800.0f;  // offset 75 * 2^14: signed x, |x| <= 2^20
 constexpr int MS = HD + 4;       // state row: acc[HD], m, l, padding
@@ -144,7 +142,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* dead) {
   for (int i = 0; i < WAIT_LIMIT; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 31) == 31 && *dead) return false;
+    if (*dead) return false;
   }
   *dead = 1;
   return false;
@@ -161,14 +159,23 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
-// barriers of the 128 compute threads (hardware barrier 1; barrier 0 is __syncthreads of the whole CTA)
-__device__ __forceinline__ void bar_sync_compute() { asm volatile("bar.sync 1, 128;\n" ::: "memory"); }
-__device__ __forceinline__ bool bar_or_compute(bool v) {
+// barriers of a team of 128 compute threads (hardware barrier `id` >= 1; barrier 0 is __syncthreads of the whole CTA)
+__device__ __forceinline__ void bar_sync_team(uint32_t id) { asm volatile("bar.sync %0, 128;\n" ::"r"(id) : "memory"); }
+__device__ __forceinline__ void bar_sync_compute() { bar_sync_team(1); }
+__device__ __forceinline__ bool bar_or_team(uint32_t id, bool v) {
   uint32_t r;
   asm volatile(
-      "{\n.reg .pred p, q;\nsetp.ne.b32 p, %1, 0;\nbar.red.or.pred q, 1, 128, p;\nselp.u32 %0, 1, 0, q;\n}\n"
-      : "=r"(r) : "r"((int)v) : "memory");
+      "{\n.reg .pred p, q;\nsetp.ne.b32 p, %2, 0;\nbar.red.or.pred q, %1, 128, p;\nselp.u32 %0, 1, 0, q;\n}\n"
+      : "=r"(r) : "r"(id), "r"((int)v) : "memory");
   return r != 0;
+}
+// running count in shared memory; release of what this thread (and, through __syncwarp, its warp) wrote before,
+// acquire of what the earlier arrivals released
+__device__ __forceinline__ unsigned atom_add_acq_rel(unsigned int* counter) {
+  unsigned old;
+  asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;\n"
+               : "=r"(old) : "r"((uint32_t)__cvta_generic_to_shared(counter)) : "memory");
+  return old;
 }
 __device__ __forceinline__ uint32_t elect_one() {
   uint32_t pred;
@@ -191,6 +198,19 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
       "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
       "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+// NC (16 or 32) consecutive columns of this thread's lane
+template <int NC>
+__device__ __forceinline__ void tmem_st_cols(uint32_t taddr, const uint32_t (&r)[NC]) {
+  if constexpr (NC == 32) tmem_st32(taddr, r);
+  else tmem_st16(taddr, r);
 }
 __device__ __forceinline__ void tmem_ld4(uint32_t taddr, uint32_t* r) {
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];\n"
@@ -285,11 +305,13 @@ struct Plan {
   static constexpr int OFF_BK = NSTG * St::BYTES;
   static constexpr int OFF_BV = OFF_BK + B_BYTES;
   static constexpr int OFF_WIN = OFF_BV + B_BYTES;
-  static constexpr int OFF_RED = OFF_WIN + WIN_BYTES;                    // reductions: [4 warps][64] words
-  static constexpr int OFF_WST = OFF_RED + 4 * 64 * 4;                   // window state rows [GP][MS]
+  static constexpr int OFF_RED = OFF_WIN + WIN_BYTES;                    // reductions: [2 teams][4 warps][64] words
+  static constexpr int META_SLOT = NGB * GP * 4;                         // logit biases of a batch: [group][head] fp32
+  static constexpr int OFF_META = OFF_RED + 2 * 4 * 64 * 4;              // one slot per stage
+  static constexpr int OFF_WST = OFF_META + NSTG * META_SLOT;            // window state rows [GP][MS]
   static constexpr int OFF_MST = OFF_WST + GP * MS * 4;                  // main state rows [GP][MS]
   static constexpr int TOTAL = OFF_MST + GP * MS * 4;
-  // tensor memory columns
+  // tensor memory columns: A_K, A_V, S of even and odd batches, O
   static constexpr uint32_t COL_AK = 0, COL_AV = 32, COL_S = 64, COL_O = 64 + 2 * N;
   static constexpr uint32_t COLS_USED = 64 + 3 * N;
   static constexpr uint32_t TM_COLS = COLS_USED <= 128 ? 128 : (COLS_USED <= 256 ? 256 : 512);
@@ -302,66 +324,6 @@ __device__ __forceinline__ int k_weight_log2(int d) { return BK == 2 ? 2 * (((d 
 // value codes: same for token t of a batch
 template <int BV>
 __device__ __forceinline__ int v_weight_log2(int t) { return BV == 2 ? 0 : ((t % 32) / 4) & 1; }
-
-// Expands this thread's token (lane `lane` of unit `unit` of the staged batch) into its A_K row: 32 columns.
-template <int BK>
-__device__ __forceinline__ void expand_keys(uint32_t kc_smem, int unit, int lane, uint32_t row_taddr) {
-  uint32_t r[32];
-  if (BK == 2) {
-    const uint4 c0 = lds128(kc_smem + unit * 1024 + lane * 16), c1 = lds128(kc_smem + unit * 1024 + 512 + lane * 16);
-    const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const uint32_t hi = w[i] >> 4;
-      r[4 * i + 0] = w[i] & 0x03030303u;
-      r[4 * i + 1] = w[i] & 0x0C0C0C0Cu;
-      r[4 * i + 2] = hi & 0x03030303u;
-      r[4 * i + 3] = hi & 0x0C0C0C0Cu;
-    }
-  } else {
-    const uint4 c0 = lds128(kc_smem + unit * 512 + lane * 16);
-    const uint32_t w[4] = {c0.x, c0.y, c0.z, c0.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint32_t hi = w[i] >> 4;
-#pragma unroll
-      for (int m = 0; m < 4; ++m) {
-        r[8 * i + m] = w[i] & (0x01010101u << m);
-        r[8 * i + 4 + m] = hi & (0x01010101u << m);
-      }
-    }
-  }
-  tmem_st32(row_taddr, r);
-}
-
-// Expands this thread's channel d into its A_V row: 32 columns over the batch's 128 tokens.  The values keep
-// small weights (1-bit: 1 or 2; 2-bit: 1): every rounding of the other operand is multiplied by them.
-template <int BV>
-__device__ __forceinline__ void expand_values(uint32_t vc_smem, int d, uint32_t row_taddr) {
-  uint32_t r[32];
-  if (BV == 1) {
-    const uint4 c0 = lds128(vc_smem + d * 16);
-    const uint32_t w[4] = {c0.x, c0.y, c0.z, c0.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const uint32_t s = w[i] >> (2 * k);
-        r[8 * i + 2 * k] = s & 0x01010101u;
-        r[8 * i + 2 * k + 1] = s & 0x02020202u;
-      }
-    }
-  } else {
-    const uint4 c0 = lds128(vc_smem + d * 16), c1 = lds128(vc_smem + 2048 + d * 16);
-    const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) r[4 * i + k] = (w[i] >> (2 * k)) & 0x03030303u;
-    }
-  }
-  tmem_st32(row_taddr, r);
-}
 
 // ---------------------------------------------------------------------------
 // window tiles on the legacy tensor-core path: 16 tokens of the 16-bit window are staged row by row and folded
@@ -610,7 +572,8 @@ __device__ __forceinline__ void ticket_merge(const DecodeParams& p, int ns, int 
   if (threadIdx.x == 0) p.tickets[bh] = 0u;  // ready for the next launch on this stream
 }
 
-// stores the NCOL operand bytes of one (row, group) slice; words[h] holds the four bytes of head h
+// stores NCOL consecutive operand bytes of a row (inside one 16-byte block, or two whole blocks); words[h] holds
+// the four bytes of head h
 template <int NCOL>
 __device__ __forceinline__ void store_slice(uint32_t addr, const uint32_t* words) {
   if constexpr (NCOL == 4) sts32(addr, words[0]);
@@ -621,27 +584,113 @@ __device__ __forceinline__ void store_slice(uint32_t addr, const uint32_t* words
     sts128(addr + 128, words[4], words[5], words[6], words[7]);
   }
 }
-// byte offset, within a row of the B operand, of the first column of group `grp`
-template <int NCOL>
-__device__ __forceinline__ uint32_t slice_offset(int grp) {
-  const int n0 = grp * NCOL;
-  return (uint32_t)((n0 >> 4) * 128 + (n0 & 15));
+// Expands this thread's share of its token's packed key row into A_K columns: team t of NT takes the columns
+// [t * 32 / NT, (t + 1) * 32 / NT).  `unit` is the token's 32-token unit of the staged batch.
+template <int BK, int NT>
+__device__ __forceinline__ void expand_keys(uint32_t kc_smem, int unit, int lane, int team, uint32_t row_taddr) {
+  constexpr int NW = (BK == 2 ? 8 : 4) / NT;  // packed words this thread expands
+  uint32_t w[NW];
+  if constexpr (BK == 2) {
+    // [chunk][token][16 bytes]: chunk c holds words 4c .. 4c + 3
+    if constexpr (NT == 1) {
+      const uint4 c0 = lds128(kc_smem + unit * 1024 + lane * 16), c1 = lds128(kc_smem + unit * 1024 + 512 + lane * 16);
+      w[0] = c0.x; w[1] = c0.y; w[2] = c0.z; w[3] = c0.w; w[4] = c1.x; w[5] = c1.y; w[6] = c1.z; w[7] = c1.w;
+    } else {
+      const uint4 c0 = lds128(kc_smem + unit * 1024 + team * 512 + lane * 16);
+      w[0] = c0.x; w[1] = c0.y; w[2] = c0.z; w[3] = c0.w;
+    }
+  } else {
+    if constexpr (NT == 1) {
+      const uint4 c0 = lds128(kc_smem + unit * 512 + lane * 16);
+      w[0] = c0.x; w[1] = c0.y; w[2] = c0.z; w[3] = c0.w;
+    } else {
+      const uint2 c0 = lds64(kc_smem + unit * 512 + lane * 16 + team * 8);
+      w[0] = c0.x; w[1] = c0.y;
+    }
+  }
+  uint32_t r[32 / NT];
+#pragma unroll
+  for (int i = 0; i < NW; ++i) {
+    const uint32_t hi = w[i] >> 4;
+    if constexpr (BK == 2) {
+      r[4 * i + 0] = w[i] & 0x03030303u;
+      r[4 * i + 1] = w[i] & 0x0C0C0C0Cu;
+      r[4 * i + 2] = hi & 0x03030303u;
+      r[4 * i + 3] = hi & 0x0C0C0C0Cu;
+    } else {
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        r[8 * i + m] = w[i] & (0x01010101u << m);
+        r[8 * i + 4 + m] = hi & (0x01010101u << m);
+      }
+    }
+  }
+  tmem_st_cols<32 / NT>(row_taddr + team * (32 / NT), r);
 }
+
+// Expands this thread's share of channel d's packed row into A_V columns (32 columns over the batch's 128 tokens).
+// The values keep small weights (1-bit: 1 or 2; 2-bit: 1): every rounding of the other operand is multiplied by them.
+template <int BV, int NT>
+__device__ __forceinline__ void expand_values(uint32_t vc_smem, int d, int team, uint32_t row_taddr) {
+  constexpr int NW = (BV == 2 ? 8 : 4) / NT;
+  uint32_t w[NW];
+  if constexpr (BV == 2) {
+    if constexpr (NT == 1) {
+      const uint4 c0 = lds128(vc_smem + d * 16), c1 = lds128(vc_smem + 2048 + d * 16);
+      w[0] = c0.x; w[1] = c0.y; w[2] = c0.z; w[3] = c0.w; w[4] = c1.x; w[5] = c1.y; w[6] = c1.z; w[7] = c1.w;
+    } else {
+      const uint4 c0 = lds128(vc_smem + team * 2048 + d * 16);
+      w[0] = c0.x; w[1] = c0.y; w[2] = c0.z; w[3] = c0.w;
+    }
+  } else {
+    if constexpr (NT == 1) {
+      const uint4 c0 = lds128(vc_smem + d * 16);
+      w[0] = c0.x; w[1] = c0.y; w[2] = c0.z; w[3] = c0.w;
+    } else {
+      const uint2 c0 = lds64(vc_smem + d * 16 + team * 8);
+      w[0] = c0.x; w[1] = c0.y;
+    }
+  }
+  uint32_t r[32 / NT];
+#pragma unroll
+  for (int i = 0; i < NW; ++i) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t s = w[i] >> (2 * k);
+      if constexpr (BV == 1) {
+        r[8 * i + 2 * k] = s & 0x01010101u;
+        r[8 * i + 2 * k + 1] = s & 0x02020202u;
+      } else {
+        r[4 * i + k] = s & 0x03030303u;
+      }
+    }
+  }
+  tmem_st_cols<32 / NT>(row_taddr + team * (32 / NT), r);
+}
+
+// byte offset, within a row of a B operand, of column n
+__device__ __forceinline__ uint32_t column_offset(int n) { return (uint32_t)((n >> 4) * 128 + (n & 15)); }
 
 // ---------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------
-// GP: heads per kv head padded to a power of two; SP: window tiles with the heads in the even columns (G <= 4).
-template <int BK, int BV, int GS, int GP, bool SP>
-__global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p) {
+// GP: heads per kv head padded to a power of two; SP: window tiles with the heads in the even columns (G <= 4);
+// NT: teams of four compute warps (a team takes GP / NT heads and 32 / NT columns of every expansion).
+template <int BK, int BV, int GS, int GP, bool SP, int NT>
+__global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umma_kernel(DecodeParams p) {
   using St = Stage<BK, BV, GS>;
   using Pl = Plan<BK, BV, GS, GP>;
   constexpr int NGB = St::NGB, N = Pl::N, NCOL = Pl::NCOL;
-  constexpr int WPG = GS / 32;  // warps whose rows share a group
+  constexpr int WPG = GS / 32;        // warps of a team whose rows share a group
+  constexpr int NCW = 4 * NT;         // compute warps
+  constexpr int W_WIN = NCW, W_BIAS = NCW + 1, W_MMA = NCW + 2;
+  constexpr int HT = GP / NT;         // heads of a team
+  constexpr int TCOL = 4 * HT;        // operand columns (bytes) of a team within a (row, group) slice
   constexpr uint32_t LBO = Pl::LBO;
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ __align__(8) unsigned long long bar_mem[2 * NSTG + 5];
   __shared__ uint32_t tmem_base_sm;
+  __shared__ int tma_issued;              // batches whose copies have been issued
   __shared__ int s_flag;
   __shared__ volatile int dead_sm;
 
@@ -682,8 +731,12 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
 
   const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(smem);
   const uint32_t bars = (uint32_t)__cvta_generic_to_shared(&bar_mem[0]);
-  const uint32_t bar_full = bars, bar_empty = bars + 8 * NSTG, bar_kready = bars + 8 * (2 * NSTG),
-                 bar_vready = bar_kready + 8, bar_sready = bar_kready + 16, bar_odone = bar_kready + 32;
+  const uint32_t bar_full = bars;                     // [NSTG] the bulk copies of a batch have landed
+  const uint32_t bar_bias = bar_full + 8 * NSTG;      // [NSTG] the logit biases of a batch are written
+  const uint32_t bar_sready = bar_bias + 8 * NSTG;    // [2] the key products of a batch are complete
+  const uint32_t bar_odone = bar_sready + 16;         // the value products of a batch are complete
+  const uint32_t bar_kready = bar_odone + 8;          // every compute warp has written its part of A_K and B_K
+  const uint32_t bar_vready = bar_kready + 8;         // the same for A_V and B_V (and the batch's stage is free)
   float* wst = reinterpret_cast<float*>(smem + Pl::OFF_WST);
   float* mst = reinterpret_cast<float*>(smem + Pl::OFF_MST);
 
@@ -691,13 +744,14 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
 #pragma unroll
     for (int s = 0; s < NSTG; ++s) {
       mbar_init(bar_full + 8 * s, 1);
-      mbar_init(bar_empty + 8 * s, 4);
+      mbar_init(bar_bias + 8 * s, 1);
     }
-    mbar_init(bar_kready, 4);
-    mbar_init(bar_vready, 4);
     mbar_init(bar_sready, 1);
     mbar_init(bar_sready + 8, 1);
     mbar_init(bar_odone, 1);
+    mbar_init(bar_kready, NCW);
+    mbar_init(bar_vready, NCW);
+    tma_issued = 0;
     dead_sm = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
@@ -711,38 +765,32 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
   tc_fence_after();
   const uint32_t tbase = tmem_base_sm;
 
-  if (warp == W_TMA) {
-    // ================= producer: one lane keeps the stage ring full =================
+  // Copies of batch j of this CTA's range into its stage (one thread; the stage is free)
+  auto issue_batch = [&](int j) {
+    const int s = j % NSTG;
+    const size_t bj = (size_t)(b0 + j);
+    const uint8_t* gk = reinterpret_cast<const uint8_t*>(p.L.k_codes) + (size_t)bh * ((size_t)dm.nq_cap * (HD * BK / 8)) + bj * St::KC;
+    const uint8_t* gkm = reinterpret_cast<const uint8_t*>(p.L.k_meta) + (size_t)bh * ((size_t)(dm.nq_cap / GS) * 512) + bj * St::KM;
+    const uint8_t* gv = reinterpret_cast<const uint8_t*>(p.L.v_codes) + (size_t)bh * ((size_t)dm.nq_cap * (HD * BV / 8)) + bj * St::VC;
+    const uint8_t* gvm = reinterpret_cast<const uint8_t*>(p.L.v_meta) + (size_t)bh * ((size_t)dm.nq_cap * 4 * NGB) + bj * St::VM;
+    const uint32_t dst = sm_base + s * St::BYTES, fb = bar_full + 8 * s;
+    mbar_expect_tx(fb, St::BYTES);
+    bulk_load(dst, gk, St::KC, fb);
+    bulk_load(dst + St::OFF_KM, gkm, St::KM, fb);
+    bulk_load(dst + St::OFF_VC, gv, St::VC, fb);
+    bulk_load(dst + St::OFF_VM, gvm, St::VM, fb);
+    tma_issued = j + 1;
+  };
+
+  if (warp == W_MMA) {
+    // ================= MMA warp: copies and products (the loop is warp-uniform, one elected lane issues) ============
     // Packed data that earlier calls completed may be fetched while the preceding kernel still runs; when a pack
-    // kernel may have written it since this layer's last decode, the producer waits for that kernel first.
+    // kernel may have written it since this layer's last decode, the first copies wait for that kernel.
     if (!p.early_fetch) grid_dependency_wait();
     if (lane == 0) {
-      const uint8_t* gk = reinterpret_cast<const uint8_t*>(p.L.k_codes) + (size_t)bh * ((size_t)dm.nq_cap * (HD * BK / 8)) + (size_t)b0 * St::KC;
-      const uint8_t* gkm = reinterpret_cast<const uint8_t*>(p.L.k_meta) + (size_t)bh * ((size_t)(dm.nq_cap / GS) * 512) + (size_t)b0 * St::KM;
-      const uint8_t* gv = reinterpret_cast<const uint8_t*>(p.L.v_codes) + (size_t)bh * ((size_t)dm.nq_cap * (HD * BV / 8)) + (size_t)b0 * St::VC;
-      const uint8_t* gvm = reinterpret_cast<const uint8_t*>(p.L.v_meta) + (size_t)bh * ((size_t)dm.nq_cap * 4 * NGB) + (size_t)b0 * St::VM;
-      int issued = 0;
-      for (int j = 0; j < nb; ++j) {
-        const int s = j % NSTG;
-        if (j >= NSTG && !mbar_wait(bar_empty + 8 * s, ((j / NSTG) - 1) & 1, &dead_sm)) break;
-        const uint32_t dst = sm_base + s * St::BYTES, fb = bar_full + 8 * s;
-        mbar_expect_tx(fb, St::BYTES);
-        bulk_load(dst, gk + (size_t)j * St::KC, St::KC, fb);
-        bulk_load(dst + St::OFF_KM, gkm + (size_t)j * St::KM, St::KM, fb);
-        bulk_load(dst + St::OFF_VC, gv + (size_t)j * St::VC, St::VC, fb);
-        bulk_load(dst + St::OFF_VM, gvm + (size_t)j * St::VM, St::VM, fb);
-        issued = j + 1;
-      }
-      if (dead_sm) {  // leaving early: no copy of this CTA may still be in flight when its shared memory is released
-        for (int j = max(0, issued - NSTG); j < issued; ++j) {
-          bool done = false;
-          for (int it = 0; it < WAIT_LIMIT && !done; ++it) done = mbar_try_wait(bar_full + 8 * (j % NSTG), (j / NSTG) & 1);
-        }
-      }
+      for (int j = 0; j < nb && j < NSTG; ++j) issue_batch(j);
     }
     __syncwarp();
-  } else if (warp == W_MMA) {
-    // ================= MMA warp: the loop is warp-uniform, one elected lane issues =================
     const uint64_t dK = smem_desc(sm_base + Pl::OFF_BK, LBO, 128), dV = smem_desc(sm_base + Pl::OFF_BV, LBO, 128);
     constexpr uint32_t KSTEP = (4 * LBO) >> 4;  // descriptor units per 32 rows of K
     constexpr uint32_t IDESC = idesc_i8(N);
@@ -751,26 +799,28 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
         const bool ok = mbar_wait(bar_kready, i & 1, &dead_sm);
         tc_fence_after();
         if (ok && elect_one()) {
-          const uint32_t dS = tbase + Pl::COL_S + (uint32_t)(i & 1) * N;
-          umma_i8<false>(dS, tbase + Pl::COL_AK, dK, IDESC);
-          umma_i8<true>(dS, tbase + Pl::COL_AK + 8, dK + KSTEP, IDESC);
-          umma_i8<true>(dS, tbase + Pl::COL_AK + 16, dK + 2 * KSTEP, IDESC);
-          umma_i8<true>(dS, tbase + Pl::COL_AK + 24, dK + 3 * KSTEP, IDESC);
+          const uint32_t dS = tbase + Pl::COL_S + (uint32_t)(i & 1) * N, aK = tbase + Pl::COL_AK;
+          umma_i8<false>(dS, aK, dK, IDESC);
+          umma_i8<true>(dS, aK + 8, dK + KSTEP, IDESC);
+          umma_i8<true>(dS, aK + 16, dK + 2 * KSTEP, IDESC);
+          umma_i8<true>(dS, aK + 24, dK + 3 * KSTEP, IDESC);
           umma_commit(bar_sready + 8 * (i & 1));
         }
         __syncwarp();
       }
-      if (i > 0) {  // values of batch i - 1
-        const bool ok = mbar_wait(bar_vready, (i - 1) & 1, &dead_sm);
+      if (i > 0) {  // values of batch i - 1; its stage is free
+        const int k = i - 1;
+        const bool ok = mbar_wait(bar_vready, k & 1, &dead_sm);
         tc_fence_after();
-        if (ok && elect_one()) {
-          const uint32_t dO = tbase + Pl::COL_O;
-          if (i == 1) umma_i8<false>(dO, tbase + Pl::COL_AV, dV, IDESC);
-          else umma_i8<true>(dO, tbase + Pl::COL_AV, dV, IDESC);
-          umma_i8<true>(dO, tbase + Pl::COL_AV + 8, dV + KSTEP, IDESC);
-          umma_i8<true>(dO, tbase + Pl::COL_AV + 16, dV + 2 * KSTEP, IDESC);
-          umma_i8<true>(dO, tbase + Pl::COL_AV + 24, dV + 3 * KSTEP, IDESC);
+        if (ok && lane == 0) {
+          const uint32_t dO = tbase + Pl::COL_O, aV = tbase + Pl::COL_AV;
+          if (k == 0) umma_i8<false>(dO, aV, dV, IDESC);
+          else umma_i8<true>(dO, aV, dV, IDESC);
+          umma_i8<true>(dO, aV + 8, dV + KSTEP, IDESC);
+          umma_i8<true>(dO, aV + 16, dV + 2 * KSTEP, IDESC);
+          umma_i8<true>(dO, aV + 24, dV + 3 * KSTEP, IDESC);
           umma_commit(bar_odone);
+          if (k + NSTG < nb) issue_batch(k + NSTG);
         }
         __syncwarp();
       }
@@ -788,26 +838,71 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
         if (lane == 0) { wst[h * MS + HD] = -CUDART_INF_F; wst[h * MS + HD + 1] = 0.f; }
       }
     }
+  } else if (warp == W_BIAS) {
+    // ================= bias warp: sigma * sum_d q_d z_d per (token group, head) of a batch =================
+    grid_dependency_wait();  // q comes from the preceding kernel
+    // One row of legacy tensor-core products per batch: rows = the batch's token groups (zero-points read as they
+    // are staged, fp16), columns = heads (q as fp16: exact for bf16 inputs of ordinary magnitude), fp32 accumulate.
+    const int gid = lane >> 2, tig = lane & 3;
+    const float scale2 = p.scale * 1.4426950408889634f;
+    uint32_t qf[16];  // B fragments: head gid, staged positions 16 ks + 2 tig (+1) and + 8
+    {
+      const bool real = gid < G;
+      const uint16_t* qp = p.q + ((size_t)b * dm.Hq + hk * G + (real ? gid : 0)) * HD;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int pos = 16 * (i >> 1) + 8 * (i & 1) + 2 * tig;  // staged position -> channel (pos % 4) * 32 + pos / 4
+        const float q0 = real ? bf16_to_f(qp[(pos & 3) * 32 + (pos >> 2)]) : 0.f;
+        const float q1 = real ? bf16_to_f(qp[((pos + 1) & 3) * 32 + ((pos + 1) >> 2)]) : 0.f;
+        const __half2 h2 = __floats2half2_rn(q0, q1);
+        qf[i] = *reinterpret_cast<const uint32_t*>(&h2);
+      }
+    }
+    for (int i = 0; i < nb; ++i) {
+      const int s = i % NSTG;
+      mbar_wait(bar_full + 8 * s, (i / NSTG) & 1, &dead_sm);
+      const uint32_t zrow = sm_base + s * St::BYTES + St::OFF_KM + (gid < NGB ? gid : 0) * 512 + 256 + 4 * tig;
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const uint32_t a0 = gid < NGB ? lds32(zrow + 32 * ks) : 0u, a2 = gid < NGB ? lds32(zrow + 32 * ks + 16) : 0u;
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+            : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(qf[2 * ks]), "r"(qf[2 * ks + 1]));
+      }
+      if (gid < NGB) {
+        float* slot = reinterpret_cast<float*>(smem + Pl::OFF_META + s * Pl::META_SLOT) + gid * GP;
+        if (2 * tig < GP) slot[2 * tig] = c[0] * scale2;
+        if (2 * tig + 1 < GP) slot[2 * tig + 1] = c[1] * scale2;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_bias + 8 * s);
+    }
   } else {
     // ================= compute warps: thread = tensor-memory lane =================
+    const int team = NT == 1 ? 0 : warp >> 2, qw = warp & 3;  // qw: lane quarter
+    const int ctid = qw * 32 + lane;                          // row: token of the batch / channel
+    const int h0 = team * HT;                                 // first head of the team
     grid_dependency_wait();  // q comes from the preceding kernel
     if (!p.early_fetch) grid_dependents_go();
-    const int gam = warp / WPG;  // this warp's rows: key token group of the batch / channel group of O
-    const uint32_t row_t = tbase + ((uint32_t)(warp * 32) << 16);
+    const int gam = qw / WPG;  // this warp's rows: key token group of the batch / channel group of O
+    const uint32_t row_t = tbase + ((uint32_t)(qw * 32) << 16);
     const float scale2 = p.scale * 1.4426950408889634f;
+    const uint32_t bar_team = 1 + team;  // hardware barrier of the team's 128 threads
 
-    // ---- q: this lane's channels lane + 32 j of every head, pre-scaled for the B_K operand ----
+    // ---- q: this lane's channels lane + 32 j of the team's heads, pre-scaled for the B_K operand ----
     // B_K holds rint(q_d s_d 2^(Eq + Es) / w_d): w_d is the weight the code of channel d carries in its A byte,
     // Eq puts the head's largest |q| and Es the group's largest scale just below 2^10 (|product| < 2^20).
-    float qp[GP][4], cq[GP], kz[GP];
+    float qp[HT][4], cq[HT];
     {
       const int wl = k_weight_log2<BK>(lane);  // the same for lane + 32 j
 #pragma unroll
-      for (int h = 0; h < GP; ++h) {
+      for (int h = 0; h < HT; ++h) {
         float qv[4], am = 0.f;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          qv[j] = h < G ? bf16_to_f(p.q[((size_t)b * dm.Hq + hk * G + h) * HD + lane + 32 * j]) : 0.f;
+          qv[j] = h0 + h < G ? bf16_to_f(p.q[((size_t)b * dm.Hq + hk * G + h0 + h) * HD + lane + 32 * j]) : 0.f;
           am = fmaxf(am, fabsf(qv[j]));
         }
         const float qmax = __uint_as_float(redux_max_u32(__float_as_uint(am)));
@@ -816,17 +911,16 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
 #pragma unroll
         for (int j = 0; j < 4; ++j) qp[h][j] = qv[j] * e2;
         cq[h] = scale2 * pow2i(-Eq);
-        kz[h] = cq[h] * pow2i(wl) * 262144.0f;  // bias partial sums leave the lane as fixed point, 18 fraction bits
       }
     }
 
-    // softmax state of the CTA (the same in every compute thread) and this thread's partial sums
-    float m[GP], l[GP], zacc[NGB][GP];
+    // softmax state of the team (the same in each of its threads) and this thread's partial sums
+    float m[HT], l[HT], zacc[NGB][HT];
     int Ev[NGB];        // value scales of channel group gi are taken relative to 2^Ev[gi]
     float vsc[NGB];     // 2^(FRAC_V - Ev[gi]) / (weight of this thread's token in its A_V byte)
-    const float wv_inv = pow2i(-v_weight_log2<BV>(tid));
+    const float wv_inv = pow2i(-v_weight_log2<BV>(ctid));
 #pragma unroll
-    for (int h = 0; h < GP; ++h) {
+    for (int h = 0; h < HT; ++h) {
       m[h] = -CUDART_INF_F;
       l[h] = 0.f;
 #pragma unroll
@@ -835,40 +929,32 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
 #pragma unroll
     for (int gi = 0; gi < NGB; ++gi) { Ev[gi] = -24; vsc[gi] = pow2i(FRAC_V + 24) * wv_inv; }
 
-    // B_K, logit scale and q . z bias of the batch staged at `st` for this warp's token group
-    auto prep_keys = [&](uint32_t st, float (&ck)[GP], float (&bias)[GP]) {
+    // A_K row and B_K slice of the batch staged at `st` for this warp's token group; returns the logit scales
+    auto prep_keys = [&](uint32_t st, float (&ck)[HT]) {
+      expand_keys<BK, NT>(st, qw, lane, team, row_t + Pl::COL_AK);
       const uint32_t km = st + St::OFF_KM + gam * 512 + lane * 8;
-      const uint2 sraw = lds64(km), zraw = lds64(km + 256);
+      const uint2 sraw = lds64(km);
       const float2 s01 = __half22float2(*reinterpret_cast<const __half2*>(&sraw.x));
       const float2 s23 = __half22float2(*reinterpret_cast<const __half2*>(&sraw.y));
-      const float2 z01 = __half22float2(*reinterpret_cast<const __half2*>(&zraw.x));
-      const float2 z23 = __half22float2(*reinterpret_cast<const __half2*>(&zraw.y));
-      const float sf[4] = {s01.x, s01.y, s23.x, s23.y}, zf[4] = {z01.x, z01.y, z23.x, z23.y};
+      const float sf[4] = {s01.x, s01.y, s23.x, s23.y};
       const float smx = fmaxf(fmaxf(sf[0], sf[1]), fmaxf(sf[2], sf[3]));
       const float smax = __uint_as_float(redux_max_u32(__float_as_uint(smx)));
       const int Es = smax > 0.f ? 9 - exponent_of(smax) : 0;
       const float e2 = pow2i(Es), e2i = pow2i(-Es);
-      const uint32_t bk = sm_base + Pl::OFF_BK + (lane >> 3) * LBO + (lane & 7) * 16 + slice_offset<NCOL>(gam);
+      const uint32_t bk = sm_base + Pl::OFF_BK + (lane >> 3) * LBO + (lane & 7) * 16 + column_offset(gam * NCOL + team * TCOL);
 #pragma unroll
       for (int jj = 0; jj < 4 / WPG; ++jj) {
-        const int j = WPG == 1 ? jj : 2 * (warp % WPG) + jj;  // with two warps per group each takes half the channels
+        const int j = WPG == 1 ? jj : 2 * (qw % WPG) + jj;  // with two warps per group each takes half the channels
         const float sp = sf[j] * e2;
-        uint32_t words[GP];
+        uint32_t words[HT];
 #pragma unroll
-        for (int h = 0; h < GP; ++h) words[h] = __float_as_uint(fmaf(qp[h][j], sp, MAGIC_K));
-        store_slice<NCOL>(bk + 4 * j * LBO, words);
+        for (int h = 0; h < HT; ++h) words[h] = __float_as_uint(fmaf(qp[h][j], sp, MAGIC_K));
+        store_slice<TCOL>(bk + 4 * j * LBO, words);
       }
 #pragma unroll
-      for (int h = 0; h < GP; ++h) {
-        ck[h] = cq[h] * e2i;
-        float t = qp[h][0] * zf[0];
-        t = fmaf(qp[h][1], zf[1], t);
-        t = fmaf(qp[h][2], zf[2], t);
-        t = fmaf(qp[h][3], zf[3], t);
-        bias[h] = (float)redux_add_s32(__float2int_rn(t * kz[h])) * (1.0f / 262144.0f);
-      }
+      for (int h = 0; h < HT; ++h) ck[h] = cq[h] * e2i;
     };
-    // this warp's A rows and B slices are written: hand them to the MMA warp
+    // this warp's part of the key (value) operands is written: hand it to the MMA warp
     auto publish = [&](uint32_t bar) {
       tc_wait_st();
       proxy_fence();
@@ -877,25 +963,25 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
       if (lane == 0) mbar_arrive(bar);
     };
 
-    // Raises the softmax references and / or the value-scale exponents so that every numerator of this batch is
-    // at most 2^TAU and every normalised value scale below 1, and rescales what has been accumulated.
-    auto raise = [&](int i, const float (&x)[GP], const float (&sv)[NGB]) {
-      int* red = reinterpret_cast<int*>(smem + Pl::OFF_RED);  // [4 warps][64]
+    // Raises the team's softmax references and / or value-scale exponents so that every numerator of this batch
+    // is at most 2^TAU and every normalised value scale below 1, and rescales what has been accumulated.
+    auto raise = [&](int i, const float (&x)[HT], const float (&sv)[NGB]) {
+      int* red = reinterpret_cast<int*>(smem + Pl::OFF_RED) + team * 256;  // [4 warps][64]
 #pragma unroll
-      for (int h = 0; h < GP; ++h) {
+      for (int h = 0; h < HT; ++h) {
         const int k = redux_max_s32(float_key(x[h]));
-        if (lane == 0) red[warp * 64 + h] = k;
+        if (lane == 0) red[qw * 64 + h] = k;
       }
 #pragma unroll
       for (int gi = 0; gi < NGB; ++gi) {
         const uint32_t u = redux_max_u32(__float_as_uint(sv[gi]));
-        if (lane == 0) red[warp * 64 + 8 + gi] = (int)u;
+        if (lane == 0) red[qw * 64 + 8 + gi] = (int)u;
       }
-      bar_sync_compute();
-      float dmh[GP];
+      bar_sync_team(bar_team);
+      float dmh[HT];
       int dE_row = 0;
 #pragma unroll
-      for (int h = 0; h < GP; ++h) {
+      for (int h = 0; h < HT; ++h) {
         const int k = max(max(red[h], red[64 + h]), max(red[128 + h], red[192 + h]));
         const float xm = key_float(k);
         float mn = m[h];
@@ -916,14 +1002,14 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
         Ev[gi] = En;
         vsc[gi] = pow2i(FRAC_V - En) * wv_inv;
       }
-      if (i > 0) {  // O of this thread's channel: its group's columns, three byte planes per head
+      if (i > 0) {  // O of this thread's channel: its group's columns of the team's heads, three byte planes per head
         mbar_wait(bar_odone, (i - 1) & 1, &dead_sm);
         tc_fence_after();
-        uint32_t o[NCOL];
-        tmem_ld_row<NCOL>(row_t + Pl::COL_O + gam * NCOL, o);
+        uint32_t o[TCOL];
+        tmem_ld_row<TCOL>(row_t + Pl::COL_O + gam * NCOL + team * TCOL, o);
         tc_wait_ld();
 #pragma unroll
-        for (int h = 0; h < GP; ++h) {
+        for (int h = 0; h < HT; ++h) {
           const int k = (int)fminf(dmh[h], 64.f) + dE_row;
           unsigned long long T = (unsigned long long)o[4 * h] + ((unsigned long long)o[4 * h + 1] << 8) +
                                  ((unsigned long long)o[4 * h + 2] << 16);
@@ -932,43 +1018,41 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
           o[4 * h + 1] = 0u;
           o[4 * h + 2] = (uint32_t)(T >> 16);
         }
-        tmem_st_row<NCOL>(row_t + Pl::COL_O + gam * NCOL, o);
+        tmem_st_row<TCOL>(row_t + Pl::COL_O + gam * NCOL + team * TCOL, o);
         tc_wait_st();
       }
-      bar_sync_compute();  // the reduction scratch may be written again
+      bar_sync_team(bar_team);  // the reduction scratch may be written again
     };
 
     // ---- prologue: keys of the first batch ----
-    float ck[GP], bias[GP], ck_n[GP], bias_n[GP];
+    float ck[HT], ck_n[HT];
     mbar_wait(bar_full, 0, &dead_sm);
-    expand_keys<BK>(sm_base, warp, lane, row_t + Pl::COL_AK);
-    prep_keys(sm_base, ck, bias);
+    prep_keys(sm_base, ck);
     publish(bar_kready);
 #pragma unroll
-    for (int h = 0; h < GP; ++h) { ck_n[h] = ck[h]; bias_n[h] = bias[h]; }
+    for (int h = 0; h < HT; ++h) ck_n[h] = ck[h];
 
     // ---- main loop: keys of batch i + 1 go to the tensor core, then softmax and values of batch i ----
 #pragma unroll 1
     for (int i = 0; i < nb; ++i) {
-      const uint32_t st = sm_base + (i % NSTG) * St::BYTES;
+      const int s = i % NSTG;
+      const uint32_t st = sm_base + s * St::BYTES;
       mbar_wait(bar_sready + 8 * (i & 1), (i >> 1) & 1, &dead_sm);  // S of batch i is complete; A_K and B_K are free
       tc_fence_after();
       if (i + 1 < nb) {
         const int sn = (i + 1) % NSTG;
-        const uint32_t stn = sm_base + sn * St::BYTES;
         mbar_wait(bar_full + 8 * sn, ((i + 1) / NSTG) & 1, &dead_sm);
-        expand_keys<BK>(stn, warp, lane, row_t + Pl::COL_AK);
-        prep_keys(stn, ck_n, bias_n);
+        prep_keys(sm_base + sn * St::BYTES, ck_n);
         publish(bar_kready);
       }
 
-      // logits of this thread's token: its group's columns of S
-      uint32_t d[NCOL];
-      tmem_ld_row<NCOL>(row_t + Pl::COL_S + (uint32_t)(i & 1) * N + gam * NCOL, d);
+      // logits of this thread's token: its group's columns of S for the team's heads
+      uint32_t d[TCOL];
+      tmem_ld_row<TCOL>(row_t + Pl::COL_S + (uint32_t)(i & 1) * N + gam * NCOL + team * TCOL, d);
       // value scale / zero-point of this thread's token
       float sv[NGB], zv[NGB];
       if constexpr (NGB == 4) {
-        const uint4 raw = lds128(st + St::OFF_VM + tid * 16);
+        const uint4 raw = lds128(st + St::OFF_VM + ctid * 16);
         const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
         const float2 c = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
         const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&raw.z));
@@ -976,22 +1060,29 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
         sv[0] = a.x; sv[1] = a.y; sv[2] = c.x; sv[3] = c.y;
         zv[0] = e.x; zv[1] = e.y; zv[2] = f.x; zv[3] = f.y;
       } else {
-        const uint2 raw = lds64(st + St::OFF_VM + tid * 8);
+        const uint2 raw = lds64(st + St::OFF_VM + ctid * 8);
         const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
         const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
         sv[0] = a.x; sv[1] = a.y;
         zv[0] = e.x; zv[1] = e.y;
       }
-      const bool valid = (b0 + i) * BT + tid < p.n_q;  // only the stream's last batch can be ragged
+      mbar_wait(bar_bias + 8 * s, (i / NSTG) & 1, &dead_sm);
+      float bias[HT];
+      {
+        const float* slot = reinterpret_cast<const float*>(smem + Pl::OFF_META + s * Pl::META_SLOT) + gam * GP + h0;
+#pragma unroll
+        for (int h = 0; h < HT; ++h) bias[h] = slot[h];
+      }
+      const bool valid = (b0 + i) * BT + ctid < p.n_q;  // only the stream's last batch can be ragged
       if (!valid) {
 #pragma unroll
         for (int gi = 0; gi < NGB; ++gi) { sv[gi] = 0.f; zv[gi] = 0.f; }
       }
       tc_wait_ld();
-      float x[GP];
+      float x[HT];
       bool need = false;
 #pragma unroll
-      for (int h = 0; h < GP; ++h) {
+      for (int h = 0; h < HT; ++h) {
         // sum_d c_d w_d X_d = D0 + 2^8 D1 + 2^16 D2 - 2^14 D3 (D3 = 75 * row sum undoes the offset 75 * 2^14 of X_d)
         const int S = (int)(d[4 * h] + (d[4 * h + 1] << 8) + (d[4 * h + 2] << 16) - (d[4 * h + 3] << 14));
         x[h] = valid ? fmaf((float)S, ck[h], bias[h]) : -CUDART_INF_F;
@@ -999,72 +1090,71 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
       }
 #pragma unroll
       for (int gi = 0; gi < NGB; ++gi) need |= __float_as_int(sv[gi]) >= ((Ev[gi] + 127) << 23);
-      if (bar_or_compute(need)) raise(i, x, sv);
+      if (bar_or_team(bar_team, need)) raise(i, x, sv);
 
-      float pe[GP];
+      float pe[HT];
 #pragma unroll
-      for (int h = 0; h < GP; ++h) {
+      for (int h = 0; h < HT; ++h) {
         pe[h] = ex2(x[h] - m[h]);
         l[h] += pe[h];
 #pragma unroll
         for (int gi = 0; gi < NGB; ++gi) zacc[gi][h] = fmaf(pe[h], zv[gi], zacc[gi][h]);
       }
-      if (i > 0) mbar_wait(bar_odone, (i - 1) & 1, &dead_sm);  // the value MMAs of batch i - 1 are done with A_V and B_V
+      if (i > 0) mbar_wait(bar_odone, (i - 1) & 1, &dead_sm);  // the value products of batch i - 1 are done with A_V and B_V
       tc_fence_after();
       {
-        const uint32_t bv = sm_base + Pl::OFF_BV + (tid >> 3) * LBO + (tid & 7) * 16;
+        const uint32_t bv = sm_base + Pl::OFF_BV + (ctid >> 3) * LBO + (ctid & 7) * 16;
 #pragma unroll
         for (int gi = 0; gi < NGB; ++gi) {
           const float sp = sv[gi] * vsc[gi];
-          uint32_t words[GP];
+          uint32_t words[HT];
 #pragma unroll
-          for (int h = 0; h < GP; ++h) words[h] = __float_as_uint(fmaf(pe[h], sp, MAGIC_V));
-          store_slice<NCOL>(bv + slice_offset<NCOL>(gi), words);
+          for (int h = 0; h < HT; ++h) words[h] = __float_as_uint(fmaf(pe[h], sp, MAGIC_V));
+          store_slice<TCOL>(bv + column_offset(gi * NCOL + team * TCOL), words);
         }
       }
-      expand_values<BV>(st + St::OFF_VC, tid, row_t + Pl::COL_AV);
+      expand_values<BV, NT>(st + St::OFF_VC, ctid, team, row_t + Pl::COL_AV);
       publish(bar_vready);
-      if (lane == 0) mbar_arrive(bar_empty + 8 * (i % NSTG));  // every read of the stage is done (publish synchronised the warp)
 #pragma unroll
-      for (int h = 0; h < GP; ++h) { ck[h] = ck_n[h]; bias[h] = bias_n[h]; }
+      for (int h = 0; h < HT; ++h) ck[h] = ck_n[h];
     }
 
-    // ---- epilogue: O of this thread's channel, the CTA's sums, one state row per head ----
+    // ---- epilogue: O of this thread's channel, the team's sums, one state row per head ----
     mbar_wait(bar_odone, (nb - 1) & 1, &dead_sm);
     tc_fence_after();
-    uint32_t o[NCOL];
-    tmem_ld_row<NCOL>(row_t + Pl::COL_O + gam * NCOL, o);
-    float* redf = reinterpret_cast<float*>(smem + Pl::OFF_RED);  // [4 warps][64]: l[GP], then zacc[NGB][GP]
+    uint32_t o[TCOL];
+    tmem_ld_row<TCOL>(row_t + Pl::COL_O + gam * NCOL + team * TCOL, o);
+    float* redf = reinterpret_cast<float*>(smem + Pl::OFF_RED) + team * 256;  // [4 warps][64]: l[HT], then zacc[NGB][HT]
 #pragma unroll
-    for (int h = 0; h < GP; ++h) {
+    for (int h = 0; h < HT; ++h) {
       float v = l[h];
 #pragma unroll
       for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
-      if (lane == 0) redf[warp * 64 + h] = v;
+      if (lane == 0) redf[qw * 64 + h] = v;
 #pragma unroll
       for (int gi = 0; gi < NGB; ++gi) {
         float z = zacc[gi][h];
 #pragma unroll
         for (int s = 16; s > 0; s >>= 1) z += __shfl_xor_sync(0xffffffffu, z, s);
-        if (lane == 0) redf[warp * 64 + GP + gi * GP + h] = z;
+        if (lane == 0) redf[qw * 64 + HT + gi * HT + h] = z;
       }
     }
     tc_wait_ld();
-    bar_sync_compute();
+    bar_sync_team(bar_team);
     int Erow = Ev[0];
 #pragma unroll
     for (int gi = 1; gi < NGB; ++gi) Erow = gi == gam ? Ev[gi] : Erow;
     const float unit = pow2i(Erow - FRAC_V);
 #pragma unroll
-    for (int h = 0; h < GP; ++h) {
-      if (h < G) {
+    for (int h = 0; h < HT; ++h) {
+      if (h0 + h < G) {
         const float T = fmaf(__uint2float_rn(o[4 * h + 2]), 65536.f, fmaf(__uint2float_rn(o[4 * h + 1]), 256.f, __uint2float_rn(o[4 * h])));
-        const int zi = GP + gam * GP + h;
+        const int zi = HT + gam * HT + h;
         const float zs = (redf[zi] + redf[64 + zi]) + (redf[128 + zi] + redf[192 + zi]);
-        mst[h * MS + tid] = fmaf(T, unit, zs);
-        if (tid == 0) {
-          mst[h * MS + HD] = m[h];
-          mst[h * MS + HD + 1] = (redf[h] + redf[64 + h]) + (redf[128 + h] + redf[192 + h]);
+        mst[(h0 + h) * MS + ctid] = fmaf(T, unit, zs);
+        if (ctid == 0) {
+          mst[(h0 + h) * MS + HD] = m[h];
+          mst[(h0 + h) * MS + HD + 1] = (redf[h] + redf[64 + h]) + (redf[128 + h] + redf[192 + h]);
         }
       }
     }
@@ -1088,37 +1178,53 @@ __global__ void __launch_bounds__(UTHREADS, 2) decode_umma_kernel(DecodeParams p
     }
     ticket_merge(p, ns, stride, hk, b, &s_flag);
   }
-  if (dead && tid == 0) atomicExch(p.status, 1);
+  if (dead && tid == 0) {
+    // leaving early: no copy of this CTA may still be in flight when its shared memory is released
+    const int issued = tma_issued;
+    for (int j = max(0, issued - NSTG); j < issued; ++j) {
+      bool done = false;
+      for (int it = 0; it < WAIT_LIMIT && !done; ++it) done = mbar_try_wait(bar_full + 8 * (j % NSTG), (j / NSTG) & 1);
+    }
+    atomicExch(p.status, 1);
+  }
   __syncthreads();
   if (warp == W_MMA)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tbase), "r"(Pl::TM_COLS) : "memory");
 }
 
 template <int BK, int BV, int GS, int GP>
+struct Variant {
+  static constexpr bool SP = GP <= 4;
+  static constexpr int NT = 1;
+  static constexpr int THREADS = (4 * NT + 3) * 32;
+  static auto kernel() { return decode_umma_kernel<BK, BV, GS, GP, SP, NT>; }
+};
+
+template <int BK, int BV, int GS, int GP>
 cudaError_t launch_gp(const DecodeParams& p, cudaStream_t st) {
   using Pl = Plan<BK, BV, GS, GP>;
-  constexpr bool SP = GP <= 4;
-  auto kernel = decode_umma_kernel<BK, BV, GS, GP, SP>;
+  using Va = Variant<BK, BV, GS, GP>;
+  auto kernel = Va::kernel();
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Pl::TOTAL);
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  return launch_dependent(kernel, dim3(p.n_ctas), dim3(UTHREADS), (size_t)Pl::TOTAL, st, p);
+  return launch_dependent(kernel, dim3(p.n_ctas), dim3(Va::THREADS), (size_t)Pl::TOTAL, st, p);
 }
 
 template <int BK, int BV, int GS, int GP>
 int ctas_per_sm_gp() {
   using Pl = Plan<BK, BV, GS, GP>;
-  constexpr bool SP = GP <= 4;
-  auto kernel = decode_umma_kernel<BK, BV, GS, GP, SP>;
+  using Va = Variant<BK, BV, GS, GP>;
+  auto kernel = Va::kernel();
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Pl::TOTAL) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
   int n = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, UTHREADS, Pl::TOTAL) != cudaSuccess) {
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, Va::THREADS, Pl::TOTAL) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
