@@ -55,7 +55,8 @@ extern "C" {
 #define XQ_ERR_NOMEM (-6)    /* host allocation failed                                    */
 #define XQ_ERR_DEVICE (-7)   /* a kernel gave up a bounded wait (xq_check_device)         */
 
-#define XQ_BF16 0
+#define XQ_BF16 0 /* bfloat16 */
+#define XQ_F16 1  /* IEEE half precision */
 
 #define XQ_KERNEL_AUTO 0    /* tensor-core kernel when the shape allows it, else generic   */
 #define XQ_KERNEL_GENERIC 1 /* scalar kernel: any supported shape, slow, used as cross-check */
@@ -82,15 +83,36 @@ typedef struct xq_config {
   int32_t residual_len; /* R: window capacity; a multiple of g and of 32                  */
   int32_t kq, vq;       /* key / value layers [0,kq) / [0,vq) use 2 bits, the rest 1 bit
                            (Appendix E)                                                   */
-  int32_t km, vm;       /* from layer km / vm on, odd layer l reads the codes of l-1
-                           (Algorithm 1, dequantize loop); km = vm = n_layers: no sharing.
-                           The two layers of a sharing pair must have equal bit-width.    */
+  int32_t km, vm;       /* from layer km / vm on, layers share integer codes in groups
+                           (Algorithm 1, dequantize loop: odd layer l reads the codes of
+                           l-1); km = vm = n_layers: no sharing.  The layers of a sharing
+                           group must have equal bit-width.                               */
   float eta1, eta2;     /* calibration parameter eta_B for B = 1, 2, in [0, 0.5] (Eq. 5)  */
   float sm_scale;       /* softmax scale; 0 selects 1/sqrt(head_dim)                      */
   int32_t n_splits;     /* sequence splits per (sequence, KV head) in decode; 0 = library
                            chooses; at most XQ_MAX_SPLITS                                 */
-  int32_t io_dtype;     /* XQ_BF16                                                        */
+  int32_t io_dtype;     /* type of K, V, q, out and of the residual window: XQ_BF16 or
+                           XQ_F16                                                         */
   int32_t kernel;       /* XQ_KERNEL_*                                                    */
+  /* Cross-layer sharing pattern (Section 3.3.3, 3.3.4; ablations of Tables gamma and
+   * group).  All zero selects the accelerated scheme of the paper's main results:
+   * pairs, first layer dominant, its codes shared as they are. */
+  int32_t share_group;    /* G: layers per sharing group, 2, 3 or 4; 0 = 2.  G = 2 follows
+                             Algorithm 1 (layer l >= km pairs with its neighbour of the
+                             other parity); G = 3, 4: contiguous groups counted from km
+                             (vm), and (n_layers - km) % G == 0 is required (likewise vm) */
+  int32_t share_dominant; /* k in [0, G): the group's layer whose codes all its layers read
+                             (Section 3.3.4); the others keep scale and zero-point only.
+                             A layer ahead of its dominant layer can decode only once that
+                             layer has appended (xq_decode_step: pass a layer_order that
+                             names the dominant layer first)                              */
+  float gamma1;           /* weighted-average merging (Section 3.3.3, Appendix F), G = 2 and
+                             k = 0 only: weight of the pair's second layer, in [0, 1];
+                             gamma_0 = 1 - gamma1.  0: no merging.  Otherwise the second
+                             layer's append quantizes its own block too and replaces the
+                             pair's codes by round(gamma_0 e_0 + gamma1 e_1), ties to even
+                             (evaluated in double precision); until then the block holds
+                             the first layer's codes e_0                                  */
 } xq_config;
 
 #define XQ_MAX_SPLITS 256

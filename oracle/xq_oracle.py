@@ -57,6 +57,23 @@ def layer_bits(layer: int, q: int) -> int:
     return 2 if layer < q else 1
 
 
+def code_owner(layer: int, m: int, group: int = 2, dominant: int = 0) -> int:
+    """The layer whose integer codes `layer` reads (itself when it keeps its own).
+    Below the sharing start m every layer keeps its codes.  From m on, the layers
+    form groups of `group` layers and only the group's dominant layer (index
+    `dominant` within the group) stores codes (Section 3.3.4; ablation of Table
+    group: contiguous groups of size G, "store and share only in the k-th layer").
+    Groups of two follow Algorithm 1's dequantize loop, which tests the layer's
+    parity (an odd layer reuses layer - 1: dominant 0); groups of three and four
+    are counted from m, which is what gives Table group its common width (20 of
+    32 value layers stored for G = 2, 3, 4 with sharing from layer 8, 14, 16)."""
+    if layer < m:
+        return layer
+    if group == 2:
+        return layer - layer % 2 + dominant
+    return layer - (layer - m) % group + dominant
+
+
 def owns_codes(layer: int, m: int) -> bool:
     """Algorithm 1, dequantize loop: a layer keeps its own integer codes when it
     lies below the sharing start m or is the first (even) layer of its pair;
@@ -64,23 +81,23 @@ def owns_codes(layer: int, m: int) -> bool:
     group size G=2).  The quantize loop of Algorithm 1 prints vm / vq in this
     test for keys / values; the dequantize loop and Appendix C use km / vm, which
     is the reading taken here."""
-    return layer < m or layer % 2 == 0
+    return code_owner(layer, m) == layer
 
 
-def equiv_bits_one(q: int, m: int, n_layers: int) -> float:
+def equiv_bits_one(q: int, m: int, n_layers: int, group: int = 2, dominant: int = 0) -> float:
     """Average stored code bits per element of one cache kind, by direct count:
     every code-owning layer stores bits(l) per element, a subordinate layer stores
     none (Appendix C: codes only, scale / zero-point excluded)."""
     total = 0
     for l in range(n_layers):
-        if owns_codes(l, m):
+        if code_owner(l, m, group, dominant) == l:
             total += layer_bits(l, q)
     return total / n_layers
 
 
-def equiv_bits(kq: int, vq: int, km: int, vm: int, n_layers: int = 32) -> float:
+def equiv_bits(kq: int, vq: int, km: int, vm: int, n_layers: int = 32, group: int = 2, dominant: int = 0) -> float:
     """Equivalent bit-width of Appendix C: mean of the key and value figures."""
-    return 0.5 * (equiv_bits_one(kq, km, n_layers) + equiv_bits_one(vq, vm, n_layers))
+    return 0.5 * (equiv_bits_one(kq, km, n_layers, group, dominant) + equiv_bits_one(vq, vm, n_layers, group, dominant))
 
 
 def equiv_bits_closed_form(kq: int, vq: int, km: int, vm: int, n_layers: int = 32) -> float:
@@ -198,6 +215,16 @@ def merge_codes_weighted(e0: np.ndarray, e1: np.ndarray, gamma0: float) -> np.nd
     gamma0 in (5/6, 1] reproduces e0, i.e. the accelerated sharing used on the
     hot path."""
     v = gamma0 * e0.astype(np.float64) + (1.0 - gamma0) * e1.astype(np.float64)
+    return np.rint(v).astype(np.uint8)
+
+
+def merge_codes_gamma1(e0: np.ndarray, e1: np.ndarray, gamma1) -> np.ndarray:
+    """The same with the pair's weights stated as the library's configuration
+    states them: gamma1 (a float32) is the second layer's weight and
+    gamma0 = 1 - gamma1, both taken in double precision."""
+    g1 = float(np.float32(gamma1))
+    g0 = 1.0 - g1
+    v = g0 * e0.astype(np.float64) + g1 * e1.astype(np.float64)
     return np.rint(v).astype(np.uint8)
 
 
@@ -389,12 +416,18 @@ class OracleCache:
     """
 
     def __init__(self, n_layers, batch, n_q_heads, n_kv_heads, head_dim, group_size,
-                 residual_len, kq, vq, km, vm, eta1, eta2, sm_scale=None):
+                 residual_len, kq, vq, km, vm, eta1, eta2, sm_scale=None,
+                 share_group=2, share_dominant=0, gamma1=0.0, f16=False):
         self.L, self.B, self.Hq, self.Hkv, self.D = n_layers, batch, n_q_heads, n_kv_heads, head_dim
         self.g, self.R = group_size, residual_len
         self.kq, self.vq, self.km, self.vm = kq, vq, km, vm
         self.eta = {1: np.float32(eta1), 2: np.float32(eta2)}
         self.sm_scale = float(sm_scale) if sm_scale else 1.0 / np.sqrt(head_dim)
+        # sharing pattern: layers per group, dominant layer of a group, weight of a pair's second layer in the
+        # merged codes (0: the dominant layer's codes are shared as they are); f16: inputs are IEEE half precision
+        self.share_group, self.share_dominant, self.gamma1 = share_group or 2, share_dominant, gamma1
+        self.f16 = f16
+        assert self.gamma1 == 0.0 or (self.share_group == 2 and self.share_dominant == 0)
         assert n_q_heads % n_kv_heads == 0 and residual_len % group_size == 0
         assert head_dim % group_size == 0
         self.layers = [self._empty_layer() for _ in range(n_layers)]
@@ -415,10 +448,24 @@ class OracleCache:
     def v_bits(self, l):
         return layer_bits(l, self.vq)
 
+    def k_owner(self, l):
+        return code_owner(l, self.km, self.share_group, self.share_dominant)
+
+    def v_owner(self, l):
+        return code_owner(l, self.vm, self.share_group, self.share_dominant)
+
+    def _merges(self, l, m):
+        """Section 3.3.3 / Appendix F with G = 2: the pair's second layer quantizes its
+        own block as well and the pair's codes become the rounded weighted average.  In
+        an incremental cache that happens when the second layer's block fills; until
+        then the block holds the first layer's codes."""
+        return self.gamma1 > 0.0 and l >= m and l % 2 == 1
+
     def _flush(self, l):
         st = self.layers[l]
         B, H = self.B, self.Hkv
-        own_k, own_v = owns_codes(l, self.km), owns_codes(l, self.vm)
+        mrg_k, mrg_v = self._merges(l, self.km), self._merges(l, self.vm)
+        own_k, own_v = self.k_owner(l) == l or mrg_k, self.v_owner(l) == l or mrg_v
         bk, bv = self.k_bits(l), self.v_bits(l)
         kc, ks, kz, vc, vs, vz = [], [], [], [], [], []
         for b in range(B):
@@ -431,16 +478,28 @@ class OracleCache:
         def stack(xs):
             return None if xs[0] is None else np.stack(xs).reshape((B, H) + xs[0].shape)
 
-        st["k_codes"].append(stack(kc)); st["k_s"].append(stack(ks)); st["k_z"].append(stack(kz))
-        st["v_codes"].append(stack(vc)); st["v_s"].append(stack(vs)); st["v_z"].append(stack(vz))
+        blk = len(st["k_s"])  # index of the block being quantized
+        kcs, vcs = stack(kc), stack(vc)
+        if mrg_k:  # the pair's codes of this block: weighted average with the first layer's, rounded
+            first = self.layers[l - 1]["k_codes"]
+            assert len(first) > blk, "the pair's first layer must have quantized this block"
+            first[blk] = merge_codes_gamma1(first[blk], kcs, self.gamma1)
+            kcs = None
+        if mrg_v:
+            first = self.layers[l - 1]["v_codes"]
+            assert len(first) > blk, "the pair's first layer must have quantized this block"
+            first[blk] = merge_codes_gamma1(first[blk], vcs, self.gamma1)
+            vcs = None
+        st["k_codes"].append(kcs); st["k_s"].append(stack(ks)); st["k_z"].append(stack(kz))
+        st["v_codes"].append(vcs); st["v_s"].append(stack(vs)); st["v_z"].append(stack(vz))
         st["win_k"] = st["win_k"][:, :, :0]
         st["win_v"] = st["win_v"][:, :, :0]
 
     def append(self, l: int, k_bits16: np.ndarray, v_bits16: np.ndarray):
-        """k_bits16, v_bits16: [B, H_kv, n, D] bfloat16 bit patterns."""
+        """k_bits16, v_bits16: [B, H_kv, n, D] bit patterns of the 16-bit input type."""
         st = self.layers[l]
-        k = bf16_bits_to_f32(k_bits16)
-        v = bf16_bits_to_f32(v_bits16)
+        k = self._widen(k_bits16)
+        v = self._widen(v_bits16)
         n = k.shape[2]
         i = 0
         while i < n:
@@ -452,6 +511,12 @@ class OracleCache:
             st["seq"] += take
             i += take
 
+    def _widen(self, bits16):
+        """16-bit inputs to fp32, exactly."""
+        if self.f16:
+            return np.ascontiguousarray(bits16).view(np.float16).astype(np.float32)
+        return bf16_bits_to_f32(bits16)
+
     def n_quantized(self, l):
         return self.R * len(self.layers[l]["k_s"])
 
@@ -462,8 +527,7 @@ class OracleCache:
     def codes_and_meta(self, l):
         """Logical arrays of layer l's quantized region: codes come from the
         code-owning layer of the pair, scale / zero-point from layer l itself."""
-        lk = l if owns_codes(l, self.km) else l - 1
-        lv = l if owns_codes(l, self.vm) else l - 1
+        lk, lv = self.k_owner(l), self.v_owner(l)
         nq = self.n_quantized(l)
         assert self.n_quantized(lk) >= nq and self.n_quantized(lv) >= nq
         nb = nq // self.R
@@ -489,7 +553,7 @@ class OracleCache:
         """q_bits16: [B, H_q, D] bfloat16 bits.  Returns fp64 [B, H_q, D]; query head
         h reads kv head h // (H_q / H_kv).  `pairs` optionally restricts the work
         to a list of (batch, q head); other entries are NaN."""
-        q = bf16_bits_to_f32(q_bits16).astype(np.float64)
+        q = self._widen(q_bits16).astype(np.float64)
         G = self.Hq // self.Hkv
         out = np.full((self.B, self.Hq, self.D), np.nan, dtype=np.float64)
         todo = pairs if pairs is not None else [(b, h) for b in range(self.B) for h in range(self.Hq)]

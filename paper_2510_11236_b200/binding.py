@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libxq.so")
 
 XQ_OK = 0
 XQ_ERR_CONFIG, XQ_ERR_ARG, XQ_ERR_CAPACITY, XQ_ERR_ORDER, XQ_ERR_CUDA, XQ_ERR_NOMEM, XQ_ERR_DEVICE = -1, -2, -3, -4, -5, -6, -7
-XQ_BF16 = 0
+XQ_BF16, XQ_F16 = 0, 1
 XQ_KERNEL_AUTO, XQ_KERNEL_GENERIC, XQ_KERNEL_MMA = 0, 1, 2
 XQ_MEM_DEVICE, XQ_MEM_HOST = 0, 1
 XQ_MAX_SPLITS = 256
@@ -30,6 +30,7 @@ class xq_config(ctypes.Structure):
         ("kq", ctypes.c_int32), ("vq", ctypes.c_int32), ("km", ctypes.c_int32), ("vm", ctypes.c_int32),
         ("eta1", ctypes.c_float), ("eta2", ctypes.c_float), ("sm_scale", ctypes.c_float),
         ("n_splits", ctypes.c_int32), ("io_dtype", ctypes.c_int32), ("kernel", ctypes.c_int32),
+        ("share_group", ctypes.c_int32), ("share_dominant", ctypes.c_int32), ("gamma1", ctypes.c_float),
     ]
 
 
@@ -203,10 +204,10 @@ def xq_strerror(code: int) -> str:
 
 def make_config(*, n_layers, batch, n_q_heads, n_kv_heads, head_dim, max_seq, group_size=32, residual_len=128,
                 kq=None, vq=None, km=0, vm=0, eta1=0.0, eta2=0.0, sm_scale=0.0, n_splits=0,
-                kernel=XQ_KERNEL_AUTO) -> xq_config:
+                kernel=XQ_KERNEL_AUTO, io_dtype=XQ_BF16, share_group=0, share_dominant=0, gamma1=0.0) -> xq_config:
     return xq_config(n_layers, batch, n_q_heads, n_kv_heads, head_dim, max_seq, group_size, residual_len,
                      n_layers if kq is None else kq, n_layers if vq is None else vq, km, vm,
-                     eta1, eta2, sm_scale, n_splits, XQ_BF16, kernel)
+                     eta1, eta2, sm_scale, n_splits, io_dtype, kernel, share_group, share_dominant, gamma1)
 
 
 class Cache:
@@ -257,7 +258,7 @@ class Cache:
     def decode_attention(self, layer, q, out=None, f32=False):
         import torch
         if out is None:
-            out = torch.empty(q.shape, dtype=torch.float32 if f32 else torch.bfloat16, device=q.device)
+            out = torch.empty(q.shape, dtype=torch.float32 if f32 else q.dtype, device=q.device)
         fn = xq_decode_attention_f32 if f32 else xq_decode_attention
         rc = fn(self.handle, layer, q, out, self._stream())
         if rc:

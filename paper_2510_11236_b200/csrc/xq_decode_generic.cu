@@ -19,6 +19,8 @@ namespace xq {
 
 __device__ __forceinline__ float bf16_bits_f(uint16_t u) { return __uint_as_float(((uint32_t)u) << 16); }
 __device__ __forceinline__ float f16_bits_f(uint16_t u) { return __half2float(__ushort_as_half(u)); }
+// an element of q, K, V or the window: IEEE half precision or bfloat16
+__device__ __forceinline__ float io_bits_f(uint16_t u, int f16) { return f16 ? f16_bits_f(u) : bf16_bits_f(u); }
 
 constexpr int GEN_WARPS = 4;
 constexpr int GEN_HEADS = 8;  // query heads processed per pass
@@ -70,7 +72,7 @@ __global__ void __launch_bounds__(GEN_WARPS * 32) decode_generic_kernel(DecodePa
 #pragma unroll
       for (int j = 0; j < DPL; ++j) {
         acc[a][j] = 0.f;
-        q[a][j] = (a < nh) ? bf16_bits_f(p.q[((size_t)b * dm.Hq + hk * dm.G + g0 + a) * D + lane + 32 * j]) : 0.f;
+        q[a][j] = (a < nh) ? io_bits_f(p.q[((size_t)b * dm.Hq + hk * dm.G + g0 + a) * D + lane + 32 * j], p.f16) : 0.f;
       }
     }
     for (int t = t0 + warp; t < t1; t += GEN_WARPS) {
@@ -88,8 +90,8 @@ __global__ void __launch_bounds__(GEN_WARPS * 32) decode_generic_kernel(DecodePa
           float cv = (float)((vc[pv.word] >> pv.bit) & ((1u << bv) - 1));
           vx[j] = fmaf(cv, f16_bits_f(vm[v_scale_index(t, d / g, NG)]), f16_bits_f(vm[v_zero_index(t, d / g, NG)]));
         } else {
-          kx[j] = bf16_bits_f(wk[(size_t)t * D + d]);
-          vx[j] = bf16_bits_f(wv[(size_t)t * D + d]);
+          kx[j] = io_bits_f(wk[(size_t)t * D + d], p.f16);
+          vx[j] = io_bits_f(wv[(size_t)t * D + d], p.f16);
         }
       }
 #pragma unroll
@@ -173,6 +175,8 @@ __global__ void merge_kernel(MergeParams p) {
   size_t oi = ((size_t)b * dm.Hq + hq) * D + d;
   if (p.out_f32)
     reinterpret_cast<float*>(p.out)[oi] = o;
+  else if (p.f16)
+    reinterpret_cast<__half*>(p.out)[oi] = __float2half_rn(o);
   else
     reinterpret_cast<__nv_bfloat16*>(p.out)[oi] = __float2bfloat16_rn(o);
 }

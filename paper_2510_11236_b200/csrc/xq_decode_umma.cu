@@ -75,6 +75,9 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 __device__ __forceinline__ float bf16_to_f(uint32_t u16) { return __uint_as_float(u16 << 16); }
+__device__ __forceinline__ float f16_to_f(uint32_t u16) { return __half2float(__ushort_as_half((unsigned short)u16)); }
+// an element of q: IEEE half precision or bfloat16
+__device__ __forceinline__ float io_to_f(uint32_t u16, int f16) { return f16 ? f16_to_f(u16) : bf16_to_f(u16); }
 __device__ __forceinline__ uint4 lds128(uint32_t a) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
@@ -339,12 +342,21 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(d) : "r"(a));
   return d;
 }
-__device__ __forceinline__ void mma16816_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                              uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+// 16-bit operands of the window's type (F16: IEEE half precision, else bfloat16), fp32 accumulate
+template <bool F16>
+__device__ __forceinline__ void mma16816_io(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                            uint32_t b0, uint32_t b1) {
+  if constexpr (F16) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  } else {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  }
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
@@ -354,10 +366,20 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, u
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&h);
+template <bool F16>
+__device__ __forceinline__ uint32_t pack_io2(float lo, float hi) {
+  if constexpr (F16) {
+    __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+  } else {
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+  }
 }
+template <bool F16>
+__device__ __forceinline__ float io2_lo(uint32_t w) { return F16 ? f16_to_f(w & 0xffffu) : bf16_to_f(w & 0xffffu); }
+template <bool F16>
+__device__ __forceinline__ float io2_hi(uint32_t w) { return F16 ? f16_to_f(w >> 16) : bf16_to_f(w >> 16); }
 
 // One warp stages window tokens [tb, tb + 16) (rows at or beyond t1 are zero-filled); no commit.  With a fused
 // append the newest row (index r - 1) is not in the window yet: it comes from the step's input.
@@ -400,7 +422,7 @@ __device__ __forceinline__ void window_store_new(const DecodeParams& p, int tb, 
 // One warp folds the staged tile (n_valid of its 16 tokens exist) into its softmax state: S^T = K q^T with tokens
 // as rows and the heads in the eight columns (SP: head h in column 2h, odd columns padding), O^T += V^T P.
 // qb: q of the head of column lane/4 as bf16 pairs in B-operand order; accZ row 8 carries sum_t p_t.
-template <bool SP>
+template <bool SP, bool F16>
 __device__ __forceinline__ void window_tile(uint32_t wbuf, int n_valid, const uint32_t (&qb)[16], float scale2,
                                             float (&accO)[8][4], float (&accZ)[4], float& m0, float& m1, int lane) {
   const int gid = lane >> 2;
@@ -410,7 +432,7 @@ __device__ __forceinline__ void window_tile(uint32_t wbuf, int n_valid, const ui
   for (int ks = 0; ks < 8; ++ks) {
     uint32_t a0, a1, a2, a3;
     ldmatrix_x4(ka + ks * 32, a0, a1, a2, a3);
-    mma16816_bf16(s, a0, a1, a2, a3, qb[2 * ks], qb[2 * ks + 1]);
+    mma16816_io<F16>(s, a0, a1, a2, a3, qb[2 * ks], qb[2 * ks + 1]);
   }
   const bool va = gid < n_valid, vb = gid + 8 < n_valid;
   const float x00 = va ? s[0] * scale2 : -CUDART_INF_F, x01 = SP ? 0.f : (va ? s[1] * scale2 : -CUDART_INF_F);
@@ -433,28 +455,28 @@ __device__ __forceinline__ void window_tile(uint32_t wbuf, int n_valid, const ui
   m0 = mn0; m1 = mn1;
   const float p00 = ex2(x00 - m0), p10 = ex2(x10 - m0);
   const float p01 = SP ? 0.f : ex2(x01 - m1), p11 = SP ? 0.f : ex2(x11 - m1);
-  // numerators as bf16 hi + lo (16 bits of precision), transposed into B-operand order
-  const uint32_t h0 = pack_bf16x2(p00, p01), h1 = pack_bf16x2(p10, p11);
-  const uint32_t l0 = pack_bf16x2(p00 - bf16_to_f(h0 & 0xffff), p01 - bf16_to_f(h0 >> 16));
-  const uint32_t l1 = pack_bf16x2(p10 - bf16_to_f(h1 & 0xffff), p11 - bf16_to_f(h1 >> 16));
+  // numerators as a 16-bit pair hi + lo (at least 16 bits of precision), transposed into B-operand order
+  const uint32_t h0 = pack_io2<F16>(p00, p01), h1 = pack_io2<F16>(p10, p11);
+  const uint32_t l0 = pack_io2<F16>(p00 - io2_lo<F16>(h0), p01 - io2_hi<F16>(h0));
+  const uint32_t l1 = pack_io2<F16>(p10 - io2_lo<F16>(h1), p11 - io2_hi<F16>(h1));
   const uint32_t bh0 = movmatrix_trans(h0), bh1 = movmatrix_trans(h1), bl0 = movmatrix_trans(l0), bl1 = movmatrix_trans(l1);
-  const uint32_t ones = (gid == 0) ? 0x3F803F80u : 0u;  // row 8 of the sums tile: sum_t p_t
-  mma16816_bf16(accZ, 0u, ones, 0u, ones, bh0, bh1);
-  mma16816_bf16(accZ, 0u, ones, 0u, ones, bl0, bl1);
+  const uint32_t ones = (gid == 0) ? (F16 ? 0x3C003C00u : 0x3F803F80u) : 0u;  // row 8 of the sums tile: sum_t p_t
+  mma16816_io<F16>(accZ, 0u, ones, 0u, ones, bh0, bh1);
+  mma16816_io<F16>(accZ, 0u, ones, 0u, ones, bl0, bl1);
   const int mi = lane >> 3;
   const uint32_t va_addr = wbuf + 16 * WROW + ((lane & 7) + 8 * (mi >> 1)) * WROW + (mi & 1) * 16;
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
     uint32_t a0, a1, a2, a3;
     ldmatrix_x4_trans(va_addr + mt * 32, a0, a1, a2, a3);
-    mma16816_bf16(accO[mt], a0, a1, a2, a3, bh0, bh1);
-    mma16816_bf16(accO[mt], a0, a1, a2, a3, bl0, bl1);
+    mma16816_io<F16>(accO[mt], a0, a1, a2, a3, bh0, bh1);
+    mma16816_io<F16>(accO[mt], a0, a1, a2, a3, bl0, bl1);
   }
 }
 
 // The window warp: this CTA's share [wt0, wt1) of the window, tile by tile; leaves one state row per head
 // (acc[HD], m, l) in `wst` (heads without tokens: m = -inf, l = 0).
-template <bool SP>
+template <bool SP, bool F16>
 __device__ __forceinline__ void window_warp(const DecodeParams& p, int wt0, int wt1, int hk, int b, uint32_t wbuf,
                                             float* wst, int lane) {
   const Dims& dm = p.dm;
@@ -481,7 +503,7 @@ __device__ __forceinline__ void window_warp(const DecodeParams& p, int wt0, int 
     cp_async_wait_all();
     __syncwarp();
     if (p.K_new != nullptr && tb + 16 > p.r - 1 && wt1 == p.r) window_store_new(p, tb, hk, b, wbuf, lane);
-    window_tile<SP>(wbuf, wt1 - tb, raw, scale2, accO, accZ, m0, m1, lane);
+    window_tile<SP, F16>(wbuf, wt1 - tb, raw, scale2, accO, accZ, m0, m1, lane);
   }
   const float l0 = __shfl_sync(0xffffffffu, accZ[2], tig), l1 = __shfl_sync(0xffffffffu, accZ[3], tig);
   const int h0 = SP ? tig : 2 * tig, h1 = 2 * tig + 1;
@@ -564,9 +586,15 @@ __device__ __forceinline__ void ticket_merge(const DecodeParams& p, int ns, int 
     if (p.out_f32) {
       *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + hq * HD + lane * 4) = acc;
     } else {
-      __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
-      uint2 pk = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
-      *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + hq * HD + lane * 4) = pk;
+      uint2 pk;
+      if (p.f16) {
+        __half2 lo = __floats2half2_rn(acc.x, acc.y), hi = __floats2half2_rn(acc.z, acc.w);
+        pk = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+      } else {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+        pk = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+      }
+      *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(p.out) + hq * HD + lane * 4) = pk;
     }
   }
   if (threadIdx.x == 0) p.tickets[bh] = 0u;  // ready for the next launch on this stream
@@ -831,7 +859,8 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
     int wt0, wt1;
     share_of(p.r, ns, split, wt0, wt1);
     if (wt0 < wt1) {
-      window_warp<SP>(p, wt0, wt1, hk, b, sm_base + Pl::OFF_WIN, wst, lane);
+      if (p.f16) window_warp<SP, true>(p, wt0, wt1, hk, b, sm_base + Pl::OFF_WIN, wst, lane);
+      else window_warp<SP, false>(p, wt0, wt1, hk, b, sm_base + Pl::OFF_WIN, wst, lane);
     } else {
       for (int h = 0; h < G; ++h) {
         for (int c = lane; c < HD; c += 32) wst[h * MS + c] = 0.f;
@@ -852,8 +881,8 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         const int pos = 16 * (i >> 1) + 8 * (i & 1) + 2 * tig;  // staged position -> channel (pos % 4) * 32 + pos / 4
-        const float q0 = real ? bf16_to_f(qp[(pos & 3) * 32 + (pos >> 2)]) : 0.f;
-        const float q1 = real ? bf16_to_f(qp[((pos + 1) & 3) * 32 + ((pos + 1) >> 2)]) : 0.f;
+        const float q0 = real ? io_to_f(qp[(pos & 3) * 32 + (pos >> 2)], p.f16) : 0.f;
+        const float q1 = real ? io_to_f(qp[((pos + 1) & 3) * 32 + ((pos + 1) >> 2)], p.f16) : 0.f;
         const __half2 h2 = __floats2half2_rn(q0, q1);
         qf[i] = *reinterpret_cast<const uint32_t*>(&h2);
       }
@@ -902,7 +931,7 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
         float qv[4], am = 0.f;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          qv[j] = h0 + h < G ? bf16_to_f(p.q[((size_t)b * dm.Hq + hk * G + h0 + h) * HD + lane + 32 * j]) : 0.f;
+          qv[j] = h0 + h < G ? io_to_f(p.q[((size_t)b * dm.Hq + hk * G + h0 + h) * HD + lane + 32 * j], p.f16) : 0.f;
           am = fmaxf(am, fabsf(qv[j]));
         }
         const float qmax = __uint_as_float(redux_max_u32(__float_as_uint(am)));

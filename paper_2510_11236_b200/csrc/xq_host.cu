@@ -19,7 +19,20 @@ namespace {
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 inline int layer_bits(int l, int q) { return l < q ? 2 : 1; }
-inline bool owns_codes(int l, int m) { return l < m || (l % 2) == 0; }
+
+// The layer whose integer codes layer l reads (l itself when it keeps its own), for one cache kind with sharing
+// from layer m on.  Groups of two follow Algorithm 1's dequantize loop (the layers of a pair differ in parity;
+// the dominant one has parity k), larger groups are contiguous runs counted from m (Section 3.3.4, Table group).
+inline int code_owner(int l, int m, int group, int k) {
+  if (l < m) return l;
+  if (group == 2) return l - (l % 2) + k;
+  return l - (l - m) % group + k;
+}
+inline int share_group_of(const xq_config* c) { return c->share_group == 0 ? 2 : c->share_group; }
+inline int k_owner(const xq_config* c, int l) { return code_owner(l, c->km, share_group_of(c), c->share_dominant); }
+inline int v_owner(const xq_config* c, int l) { return code_owner(l, c->vm, share_group_of(c), c->share_dominant); }
+// Weighted-average merging (Appendix F): the pair's second layer rewrites the shared codes of a cache kind
+inline bool merges_codes(const xq_config* c, int l, int m) { return c->gamma1 > 0.f && l >= m && (l % 2) == 1; }
 
 struct LayerRegions {
   size_t win_k, win_v, k_meta, v_meta, k_codes, v_codes;  // byte offsets; codes: of the owning layer
@@ -48,12 +61,19 @@ bool check(const xq_config* c) {
   if (!(c->eta1 >= 0.f && c->eta1 <= 0.5f) || !(c->eta2 >= 0.f && c->eta2 <= 0.5f)) return false;
   if (!(c->sm_scale >= 0.f) || isinf(c->sm_scale)) return false;
   if (c->n_splits < 0 || c->n_splits > XQ_MAX_SPLITS) return false;
-  if (c->io_dtype != XQ_BF16) return false;
+  if (c->io_dtype != XQ_BF16 && c->io_dtype != XQ_F16) return false;
   if (c->kernel < XQ_KERNEL_AUTO || c->kernel > XQ_KERNEL_MMA) return false;
-  // both layers of a sharing pair must have the same bit-width
-  for (int l = 1; l < c->n_layers; l += 2) {
-    if (!owns_codes(l, c->km) && layer_bits(l, c->kq) != layer_bits(l - 1, c->kq)) return false;
-    if (!owns_codes(l, c->vm) && layer_bits(l, c->vq) != layer_bits(l - 1, c->vq)) return false;
+  const int group = share_group_of(c);
+  if (group < 2 || group > 4) return false;
+  if (c->share_dominant < 0 || c->share_dominant >= group) return false;
+  if (!(c->gamma1 >= 0.f && c->gamma1 <= 1.f)) return false;
+  if (c->gamma1 > 0.f && (group != 2 || c->share_dominant != 0)) return false;
+  if (group > 2 && ((c->n_layers - c->km) % group || (c->n_layers - c->vm) % group)) return false;
+  // every layer reads the codes of a layer that exists and has its bit-width
+  for (int l = 0; l < c->n_layers; ++l) {
+    const int ok = k_owner(c, l), ov = v_owner(c, l);
+    if (ok < 0 || ok >= c->n_layers || ov < 0 || ov >= c->n_layers) return false;
+    if (layer_bits(l, c->kq) != layer_bits(ok, c->kq) || layer_bits(l, c->vq) != layer_bits(ov, c->vq)) return false;
   }
   return true;
 }
@@ -80,8 +100,12 @@ void make_plan(const xq_config* c, Plan& pl) {
     r.v_meta = take(BH * r.stride[3]);
     r.stride[0] = (size_t)dm.nq_cap * dm.D * bk / 8;
     r.stride[1] = (size_t)dm.nq_cap * dm.D * bv / 8;
-    if (owns_codes(l, c->km)) r.k_codes = take(BH * r.stride[0]); else r.k_codes = pl.layers[l - 1].k_codes;
-    if (owns_codes(l, c->vm)) r.v_codes = take(BH * r.stride[1]); else r.v_codes = pl.layers[l - 1].v_codes;
+    r.k_codes = k_owner(c, l) == l ? take(BH * r.stride[0]) : 0;
+    r.v_codes = v_owner(c, l) == l ? take(BH * r.stride[1]) : 0;
+  }
+  for (int l = 0; l < c->n_layers; ++l) {  // the other layers of a group read the dominant layer's codes
+    if (k_owner(c, l) != l) pl.layers[l].k_codes = pl.layers[k_owner(c, l)].k_codes;
+    if (v_owner(c, l) != l) pl.layers[l].v_codes = pl.layers[v_owner(c, l)].v_codes;
   }
   pl.part_acc = take((size_t)dm.B * dm.Hq * XQ_MAX_SPLITS * dm.D * 4);
   pl.part_ml = take((size_t)dm.B * dm.Hq * XQ_MAX_SPLITS * 2 * 4);
@@ -296,9 +320,8 @@ int prepare_decode(const xq_cache* c, int layer, const void* q, void* out, int o
   if (S < 1) return XQ_ERR_ARG;
   const int r = residual_count(S, dm.R), nq = S - r;
   // a code-borrowing layer needs the owning layer's codes for all of its quantized tokens
-  if (!owns_codes(layer, c->cfg.km) || !owns_codes(layer, c->cfg.vm)) {
-    const int So = c->seq[layer - 1];
-    if (So - residual_count(So, dm.R) < nq) return XQ_ERR_ORDER;
+  for (int o : {k_owner(&c->cfg, layer), v_owner(&c->cfg, layer)}) {
+    if (o != layer && c->seq[o] - residual_count(c->seq[o], dm.R) < nq) return XQ_ERR_ORDER;
   }
   use_mma = layer_uses_mma(c, layer) && nq > 0;
   if (c->cfg.kernel >= XQ_KERNEL_MMA && !layer_uses_mma(c, layer)) return XQ_ERR_CONFIG;
@@ -321,6 +344,7 @@ int prepare_decode(const xq_cache* c, int layer, const void* q, void* out, int o
   p.out = out;
   p.out_f32 = out_f32;
   p.early_fetch = 0;
+  p.f16 = c->cfg.io_dtype == XQ_F16;
   p.K_new = (const uint16_t*)K_new;
   p.V_new = (const uint16_t*)V_new;
   return XQ_OK;
@@ -343,6 +367,7 @@ int launch_decode(xq_cache* c, DecodeParams& p, bool use_mma, const Scratch& s, 
   MergeParams m;
   m.dm = p.dm;
   m.ns = p.ns_q + p.ns_w;
+  m.f16 = p.f16;
   m.part_acc = p.part_acc;
   m.part_ml = p.part_ml;
   m.out = p.out;
@@ -373,6 +398,71 @@ int ensure_clean_scratch(xq_cache* c, cudaStream_t st) {
   if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + c->plan.status, 0, 4, st);
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->tickets_clean = true;
+  return XQ_OK;
+}
+
+// Merged code of (e0, e1) for every pair of B-bit codes, at bits 2 * (4 e0 + e1): round(gamma_0 e0 + gamma_1 e1) in
+// double precision, ties to even (Appendix F).
+uint32_t merge_table(float gamma1, int bits) {
+  const double g1 = (double)gamma1, g0 = 1.0 - g1;
+  uint32_t lut = 0u;
+  for (int e0 = 0; e0 < (1 << bits); ++e0)
+    for (int e1 = 0; e1 < (1 << bits); ++e1) {
+      const double v = g0 * (double)e0 + g1 * (double)e1;
+      lut |= ((uint32_t)nearbyint(v) & 3u) << (2 * (4 * e0 + e1));
+    }
+  return lut;
+}
+
+// One quantize-and-pack launch for `n` layers of equal length that each receive n_tokens new tokens (layer i's at
+// K + i * layer_stride bytes), at least one window block of which fills.  The launch also moves the tokens that
+// follow the quantized blocks into the window.  Layers that merge codes (gamma1 > 0) need their dominant layer's
+// blocks in place: they go one per launch, after it.
+int pack_layers(xq_cache* c, const int* layers, int n, const void* K, const void* V, size_t layer_stride, int n_tokens,
+                cudaStream_t st) {
+  const Dims& dm = c->plan.dm;
+  const int s_old = c->seq[layers[0]], s_new = s_old + n_tokens;
+  const int nq_old = s_old - residual_count(s_old, dm.R), nq_new = s_new - residual_count(s_new, dm.R);
+  PackParams p;
+  p.dm = dm;
+  p.n_layers = n;
+  p.n_in = n_tokens; p.s_old = s_old; p.nq_old = nq_old; p.n_blocks = (nq_new - nq_old) / dm.R;
+  p.tb = dm.g > 32 ? dm.g : 32;  // tokens per CTA: whole key groups, whole words of either kind
+  p.f16 = c->cfg.io_dtype == XQ_F16;
+  p.win_count = s_new - nq_new;
+  p.nq_new = nq_new;
+  p.merge_lut[0] = merge_table(c->cfg.gamma1, 1);
+  p.merge_lut[1] = merge_table(c->cfg.gamma1, 2);
+  for (int i = 0; i < n; ++i) {
+    const int l = layers[i];
+    if (c->seq[l] != s_old) return XQ_ERR_ARG;
+    PackLayer& pl = p.layer[i];
+    pl.L = layer_ptrs(c, l);
+    pl.K_in = (const uint16_t*)((const uint8_t*)K + (size_t)i * layer_stride);
+    pl.V_in = (const uint16_t*)((const uint8_t*)V + (size_t)i * layer_stride);
+    pl.own_k = k_owner(&c->cfg, l) == l ? 1 : (merges_codes(&c->cfg, l, c->cfg.km) ? 2 : 0);
+    pl.own_v = v_owner(&c->cfg, l) == l ? 1 : (merges_codes(&c->cfg, l, c->cfg.vm) ? 2 : 0);
+    if (pl.own_k == 2 || pl.own_v == 2) {
+      if (n != 1) return XQ_ERR_ARG;
+      const int o = l - 1;  // the pair's first layer must hold the blocks this layer merges into
+      if (c->seq[o] - residual_count(c->seq[o], dm.R) < nq_new) return XQ_ERR_ORDER;
+    }
+    pl.eta_k = pl.L.bk == 1 ? c->cfg.eta1 : c->cfg.eta2;
+    pl.eta_v = pl.L.bv == 1 ? c->cfg.eta1 : c->cfg.eta2;
+  }
+  cudaError_t e;
+  {
+    Timer t(c, st, 2);
+    e = launch_pack(p, st);
+  }
+  c->launches++;
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  // every layer that reads what this launch wrote must wait for it before its next decode fetches packed data
+  for (int i = 0; i < n; ++i)
+    for (int l2 = 0; l2 < c->cfg.n_layers; ++l2)
+      if (l2 == layers[i] || k_owner(&c->cfg, l2) == layers[i] || v_owner(&c->cfg, l2) == layers[i] ||
+          k_owner(&c->cfg, layers[i]) == l2 || v_owner(&c->cfg, layers[i]) == l2)
+        c->repacked[l2] = 1;
   return XQ_OK;
 }
 
@@ -482,33 +572,16 @@ int xq_append_kv(xq_cache* c, int layer, const void* K, const void* V, int n_tok
   int nq_old = s_old - residual_count(s_old, dm.R);
   int nq_new = s_new - residual_count(s_new, dm.R);
   int n_blocks = (nq_new - nq_old) / dm.R;
-  LayerPtrs L = layer_ptrs(c, layer);
   if (n_blocks > 0) {
-    PackParams p;
-    p.dm = dm; p.L = L;
-    p.K_in = (const uint16_t*)K; p.V_in = (const uint16_t*)V;
-    p.n_in = n_tokens; p.s_old = s_old; p.nq_old = nq_old; p.n_blocks = n_blocks;
-    p.own_k = owns_codes(layer, c->cfg.km); p.own_v = owns_codes(layer, c->cfg.vm);
-    p.eta_k = L.bk == 1 ? c->cfg.eta1 : c->cfg.eta2;
-    p.eta_v = L.bv == 1 ? c->cfg.eta1 : c->cfg.eta2;
-    p.tb = dm.g > 32 ? dm.g : 32;  // tokens per CTA: whole key groups, whole words of either kind
-    cudaError_t e;
-    {
-      Timer t(c, st, 2);
-      e = launch_pack(p, st);
-    }
-    c->launches++;
-    if (e != cudaSuccess) return fail_cuda(c, e);
-    c->repacked[layer] = 1;
-    if (layer + 1 < c->cfg.n_layers) c->repacked[layer + 1] = 1;  // it may read this layer's codes
-  }
-  {
+    int rc = pack_layers(c, &layer, 1, K, V, 0, n_tokens, st);
+    if (rc != XQ_OK) return rc;
+  } else {
     WindowParams w;
-    w.dm = dm; w.L = L;
+    w.dm = dm; w.L = layer_ptrs(c, layer);
     w.K_in = (const uint16_t*)K; w.V_in = (const uint16_t*)V;
     w.n_in = n_tokens; w.s_old = s_old;
-    w.first = s_old > nq_new ? s_old : nq_new;
-    w.count = s_new - w.first;
+    w.first = s_old;
+    w.count = n_tokens;
     w.nq_new = nq_new;
     cudaError_t e;
     {
@@ -583,9 +656,10 @@ int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void
       seen[l] = 1;
       if (len[l] + 1 > c->cfg.max_seq) return XQ_ERR_CAPACITY;
       len[l] += 1;
-      if (!owns_codes(l, c->cfg.km) || !owns_codes(l, c->cfg.vm)) {
-        if (!seen[l - 1]) return XQ_ERR_ORDER;
-        const int nq = len[l] - residual_count(len[l], dm.R), nqo = len[l - 1] - residual_count(len[l - 1], dm.R);
+      for (int o : {k_owner(&c->cfg, l), v_owner(&c->cfg, l)}) {
+        if (o == l) continue;
+        if (!seen[o]) return XQ_ERR_ORDER;
+        const int nq = len[l] - residual_count(len[l], dm.R), nqo = len[o] - residual_count(len[o], dm.R);
         if (nqo < nq) return XQ_ERR_ORDER;
       }
       if (c->cfg.kernel >= XQ_KERNEL_MMA && !layer_uses_mma(c, l)) return XQ_ERR_CONFIG;
@@ -606,9 +680,34 @@ int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void
     if (e != cudaSuccess) return fail_cuda(c, e);
     dk = sk; dv = sv; dq = sq; dout = so;
   }
-  // Only a CUDA error can stop the loop below (the cache is then in an undefined state, as after any XQ_ERR_CUDA).
+  // Only a CUDA error can stop what follows (the cache is then in an undefined state, as after any XQ_ERR_CUDA).
+  // The step on which every layer's window block fills: one quantize-and-pack launch for all layers (it also moves
+  // the new token into the emptied windows), then the decode launches.
+  bool appended = false;
+  {
+    bool same = true;
+    for (int l = 1; l < L; ++l) same = same && c->seq[l] == c->seq[0];
+    const int s_old = c->seq[0];
+    const int nq_old = s_old - residual_count(s_old, dm.R), nq_new = s_old + 1 - residual_count(s_old + 1, dm.R);
+    if (same && nq_new > nq_old && c->cfg.gamma1 == 0.f) {
+      for (int c0 = 0; c0 < L; c0 += PACK_MAX_LAYERS) {
+        int idx[PACK_MAX_LAYERS];
+        const int n = L - c0 < PACK_MAX_LAYERS ? L - c0 : PACK_MAX_LAYERS;
+        for (int i = 0; i < n; ++i) idx[i] = c0 + i;
+        const int rc = pack_layers(c, idx, n, dk + c0 * kv_layer, dv + c0 * kv_layer, kv_layer, 1, st);
+        if (rc != XQ_OK) return rc;
+      }
+      for (int l = 0; l < L; ++l) c->seq[l] += 1;
+      appended = true;
+    }
+  }
   for (int i = 0; i < L; ++i) {
     const int l = layer_order ? layer_order[i] : i;
+    if (appended) {
+      const int rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st);
+      if (rc != XQ_OK) return rc;
+      continue;
+    }
     // One token that neither fills a window block nor is the layer's first quantized step goes into the window
     // inside the tensor-core decode kernel; every other case appends with its own kernels first.
     const int s_old = c->seq[l];
@@ -645,8 +744,8 @@ double xq_equiv_bits(const xq_config* cfg) {
   if (!check(cfg)) return -1.0;
   long long k = 0, v = 0;
   for (int l = 0; l < cfg->n_layers; ++l) {
-    if (owns_codes(l, cfg->km)) k += layer_bits(l, cfg->kq);
-    if (owns_codes(l, cfg->vm)) v += layer_bits(l, cfg->vq);
+    if (k_owner(cfg, l) == l) k += layer_bits(l, cfg->kq);
+    if (v_owner(cfg, l) == l) v += layer_bits(l, cfg->vq);
   }
   return 0.5 * ((double)k + (double)v) / (double)cfg->n_layers;
 }

@@ -21,18 +21,35 @@ struct LayerPtrs {
   int bk, bv;
 };
 
-struct PackParams {
-  Dims dm;
+// One layer of a quantize-and-pack launch.
+struct PackLayer {
   LayerPtrs L;
   const uint16_t* K_in;  // [B,Hkv,n_in,D] new tokens (absolute positions s_old ..)
   const uint16_t* V_in;
+  // codes of a cache kind: 0 = none (the layer keeps scale and zero-point only), 1 = written, 2 = merged into the
+  // codes the dominant layer wrote (weighted average, Appendix F)
+  int own_k, own_v;
+  float eta_k, eta_v;
+};
+
+constexpr int PACK_MAX_LAYERS = 32;  // layers one launch can take (they share every length below)
+
+struct PackParams {
+  Dims dm;
+  int n_layers;
   int n_in;
   int s_old;     // tokens cached before this append
   int nq_old;    // quantized tokens before this append
   int n_blocks;  // R-token blocks to quantize, starting at absolute token nq_old
-  int own_k, own_v;
-  float eta_k, eta_v;
   int tb;        // tokens per CTA tile (32 or 64)
+  int f16;       // inputs and window are IEEE half precision (else bfloat16)
+  // tokens nq_new .. s_new - 1 of the input go into window rows 0 .. win_count - 1 (the CTAs that staged those rows
+  // of the old window copy them); 0: the caller copies
+  int win_count;
+  int nq_new;
+  // merged code of (e0, e1) at bits 2 * (4 e0 + e1), for 1-bit and 2-bit codes
+  uint32_t merge_lut[2];
+  PackLayer layer[PACK_MAX_LAYERS];
 };
 
 struct WindowParams {
@@ -71,11 +88,13 @@ struct DecodeParams {
   const uint16_t* K_new;
   const uint16_t* V_new;
   int* status;  // device word the tensor-core kernel sets when one of its bounded waits gave up
+  int f16;      // q, the window and the 16-bit output are IEEE half precision (else bfloat16)
 };
 
 struct MergeParams {
   Dims dm;
   int ns;
+  int f16;
   const float* part_acc;
   const float* part_ml;
   void* out;

@@ -17,6 +17,36 @@ namespace xq {
 
 __device__ __forceinline__ float bf16_bits(uint16_t u) { return __uint_as_float(((uint32_t)u) << 16); }
 
+// The 16-bit input type: widening to fp32 (exact) and packed min / max of two elements.
+template <bool F16>
+struct In16;
+template <>
+struct In16<false> {
+  using V2 = __nv_bfloat162;
+  static __device__ __forceinline__ float lo(uint32_t w) { return __uint_as_float(w << 16); }
+  static __device__ __forceinline__ float hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+  static __device__ __forceinline__ float one(uint16_t u) { return bf16_bits(u); }
+};
+template <>
+struct In16<true> {
+  using V2 = __half2;
+  static __device__ __forceinline__ float lo(uint32_t w) { return __half2float(__ushort_as_half((unsigned short)(w & 0xffffu))); }
+  static __device__ __forceinline__ float hi(uint32_t w) { return __half2float(__ushort_as_half((unsigned short)(w >> 16))); }
+  static __device__ __forceinline__ float one(uint16_t u) { return __half2float(__ushort_as_half(u)); }
+};
+
+// Merged words of a sharing pair (Appendix F): field by field, the code of (e0, e1) from the table.
+template <int BITS>
+__device__ __forceinline__ uint32_t merge_words(uint32_t w0, uint32_t w1, uint32_t lut) {
+  uint32_t out = 0u;
+#pragma unroll
+  for (int f = 0; f < 32; f += BITS) {
+    const uint32_t e0 = (w0 >> f) & ((1u << BITS) - 1u), e1 = (w1 >> f) & ((1u << BITS) - 1u);
+    out |= ((lut >> (2u * (4u * e0 + e1))) & ((1u << BITS) - 1u)) << f;
+  }
+  return out;
+}
+
 // Eq. 1 and Eq. 12 for one group: z = min, s = (max - min)/(2^B - 1),
 // z_hat = z + (eta * s) * (2^B - 1), s_hat = (1 - 2 eta) * s.
 __device__ __forceinline__ void group_params(float mn, float mx, int bits, float eta, float& z, float& s,
@@ -77,9 +107,13 @@ __device__ __forceinline__ uint32_t code_pair(float x0, float x1, const float4& 
 // rows are padded.  Keys: a thread builds whole words of a token's row (four consecutive channels per bit
 // offset), the words are collected in shared memory in stream order and leave in 16-byte vectors.  Values: a
 // thread builds whole words of a channel's row over the tile's tokens and stores them itself.
-// G: group size; T = p.tb: a multiple of G and of 32.
-template <int D, int G, int T>
-__global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
+// G: group size; T = p.tb: a multiple of G and of 32; F16: the 16-bit type is IEEE half precision.
+// blockIdx.z runs over (layer of the launch, sequence).  With p.win_count > 0 the CTAs of the first block also copy
+// the new window rows that replace the rows they staged.
+template <int D, int G, int T, bool F16>
+__global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constant__ PackParams p) {
+  using I16 = In16<F16>;
+  using V2 = typename I16::V2;
   constexpr int ROWB = D * 2 + PACK_ROW_PAD;
   constexpr int NG = D / G;
   constexpr int CB = D / 16;
@@ -96,14 +130,15 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
   const int R = dm.R;
   const int kind = blockIdx.x & 1;  // 0 keys, 1 values
   const int tile_idx = blockIdx.x >> 1;
-  const int h = blockIdx.y, b = blockIdx.z;
+  const int h = blockIdx.y, b = blockIdx.z % dm.B;
+  const PackLayer& pl = p.layer[blockIdx.z / dm.B];
   const int bh = b * dm.Hkv + h;
   const int tid = threadIdx.x;
   const int tq0 = p.nq_old + tile_idx * T;  // absolute index of the tile's first token
 
   {
-    const uint16_t* win = kind ? p.L.win_v : p.L.win_k;
-    const uint16_t* in = kind ? p.V_in : p.K_in;
+    const uint16_t* win = kind ? pl.L.win_v : pl.L.win_k;
+    const uint16_t* in = kind ? pl.V_in : pl.K_in;
     constexpr int VPR = D / 8;
 #pragma unroll
     for (int k = 0; k < T * VPR / PACK_THREADS; ++k) {
@@ -116,10 +151,22 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
     }
   }
   __syncthreads();
+  // the window rows this CTA staged are free: the tokens that follow the quantized blocks take them
+  if (p.win_count > 0 && tile_idx * T < p.win_count) {
+    uint16_t* win = kind ? pl.L.win_v : pl.L.win_k;
+    const uint16_t* in = kind ? pl.V_in : pl.K_in;
+    constexpr int VPR = D / 8;
+    const int rows = min(T, p.win_count - tile_idx * T);
+    for (int idx = tid; idx < rows * VPR; idx += PACK_THREADS) {
+      const int r = tile_idx * T + idx / VPR, c8 = idx % VPR;
+      const uint4* src = reinterpret_cast<const uint4*>(in + ((size_t)bh * p.n_in + (p.nq_new + r - p.s_old)) * D) + c8;
+      reinterpret_cast<uint4*>(win + ((size_t)bh * R + r) * D)[c8] = *src;
+    }
+  }
 
-  const int bits = kind ? p.L.bv : p.L.bk;
-  const float eta = kind ? p.eta_v : p.eta_k;
-  const int own = kind ? p.own_v : p.own_k;
+  const int bits = kind ? pl.L.bv : pl.L.bk;
+  const float eta = kind ? pl.eta_v : pl.eta_k;
+  const int own = kind ? pl.own_v : pl.own_k;
 
   if (kind == 0) {
     // keys: one group per (channel, run of G tokens).  First bf16x2 min / max of a channel pair over a part of the
@@ -128,10 +175,10 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
       const int dp = tid % (D / 2), rest = tid / (D / 2);
       const int gl = rest / KP, part = rest % KP;
       const uint8_t* col = tile + (gl * G + part * (G / KP)) * ROWB + dp * 4;
-      __nv_bfloat162 mn2 = *reinterpret_cast<const __nv_bfloat162*>(col), mx2 = mn2;
+      V2 mn2 = *reinterpret_cast<const V2*>(col), mx2 = mn2;
 #pragma unroll
       for (int j = 1; j < G / KP; ++j) {
-        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(col + j * ROWB);
+        const V2 v = *reinterpret_cast<const V2*>(col + j * ROWB);
         mn2 = __hmin2(mn2, v);
         mx2 = __hmax2(mx2, v);
       }
@@ -139,7 +186,7 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
       wbuf[(rest * (D / 2) + dp) * 2 + 1] = *reinterpret_cast<uint32_t*>(&mx2);
     }
     __syncthreads();
-    __half* meta = reinterpret_cast<__half*>(p.L.k_meta);
+    __half* meta = reinterpret_cast<__half*>(pl.L.k_meta);
     const size_t cap_g = (size_t)(dm.nq_cap / G);
 #pragma unroll
     for (int k = 0; k < ((T / G) * D + PACK_THREADS - 1) / PACK_THREADS; ++k) {
@@ -150,8 +197,8 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
 #pragma unroll
         for (int part = 0; part < KP; ++part) {
           const uint32_t a2 = wbuf[((gl * KP + part) * (D / 2) + d / 2) * 2], b2 = wbuf[((gl * KP + part) * (D / 2) + d / 2) * 2 + 1];
-          const float lo = __uint_as_float((d & 1) ? (a2 & 0xffff0000u) : (a2 << 16));
-          const float hi = __uint_as_float((d & 1) ? (b2 & 0xffff0000u) : (b2 << 16));
+          const float lo = (d & 1) ? I16::hi(a2) : I16::lo(a2);
+          const float hi = (d & 1) ? I16::hi(b2) : I16::lo(b2);
           mn = part == 0 ? lo : fminf(mn, lo);
           mx = part == 0 ? hi : fmaxf(mx, hi);
         }
@@ -167,29 +214,30 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
     }
   } else {
     // values: one group per (token, run of G channels); consecutive threads take consecutive tokens
-    __half* meta = reinterpret_cast<__half*>(p.L.v_meta);
+    __half* meta = reinterpret_cast<__half*>(pl.L.v_meta);
 #pragma unroll
     for (int k = 0; k < (T * NG + PACK_THREADS - 1) / PACK_THREADS; ++k) {
       const int item = tid + k * PACK_THREADS;
       if (item < T * NG) {
         const int tl = item % T, gi = item / T;
         const uint4* row = reinterpret_cast<const uint4*>(tile + tl * ROWB + gi * G * 2);
-        __nv_bfloat162 mn2, mx2;
+        V2 mn2, mx2;
         {
           uint4 v = row[0];
-          const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&v);
+          const V2* e = reinterpret_cast<const V2*>(&v);
           mn2 = __hmin2(__hmin2(e[0], e[1]), __hmin2(e[2], e[3]));
           mx2 = __hmax2(__hmax2(e[0], e[1]), __hmax2(e[2], e[3]));
         }
 #pragma unroll
         for (int j = 1; j < G / 8; ++j) {
           uint4 v = row[j];
-          const __nv_bfloat162* e = reinterpret_cast<const __nv_bfloat162*>(&v);
+          const V2* e = reinterpret_cast<const V2*>(&v);
           mn2 = __hmin2(mn2, __hmin2(__hmin2(e[0], e[1]), __hmin2(e[2], e[3])));
           mx2 = __hmax2(mx2, __hmax2(__hmax2(e[0], e[1]), __hmax2(e[2], e[3])));
         }
-        const float mn = fminf(__low2float(mn2), __high2float(mn2));
-        const float mx = fmaxf(__low2float(mx2), __high2float(mx2));
+        const uint32_t mnw = *reinterpret_cast<const uint32_t*>(&mn2), mxw = *reinterpret_cast<const uint32_t*>(&mx2);
+        const float mn = fminf(I16::lo(mnw), I16::hi(mnw));
+        const float mx = fmaxf(I16::lo(mxw), I16::hi(mxw));
         float z, sc;
         __half zh, sh;
         group_params(mn, mx, bits, eta, z, sc, zh, sh);
@@ -205,7 +253,8 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
   __syncthreads();
 
   // codes
-  uint32_t* codes = kind ? p.L.v_codes : p.L.k_codes;
+  uint32_t* codes = kind ? pl.L.v_codes : pl.L.k_codes;
+  const bool merge = own == 2;
   const size_t stream_words = (size_t)dm.nq_cap * D * bits / 32;
   auto build = [&](auto bits_c) {
     constexpr int BITS = decltype(bits_c)::value;
@@ -227,8 +276,8 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
             const int d = i * N + 4 * s4;
             const uint2 xx = *reinterpret_cast<const uint2*>(row + d * 2);
             const float4 p0 = par[gl * D + d], p1 = par[gl * D + d + 1], p2 = par[gl * D + d + 2], p3 = par[gl * D + d + 3];
-            const uint32_t lo = code_pair<BITS>(__uint_as_float(xx.x << 16), __uint_as_float(xx.x & 0xffff0000u), p0, p1, doubt);
-            const uint32_t hi = code_pair<BITS>(__uint_as_float(xx.y << 16), __uint_as_float(xx.y & 0xffff0000u), p2, p3, doubt);
+            const uint32_t lo = code_pair<BITS>(I16::lo(xx.x), I16::hi(xx.x), p0, p1, doubt);
+            const uint32_t hi = code_pair<BITS>(I16::lo(xx.y), I16::hi(xx.y), p2, p3, doubt);
             word |= (lo | (hi << 16)) << (BITS * s4);
           }
           if (doubt) {  // rare: the word again, with the division
@@ -237,7 +286,7 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
             for (int e = 0; e < N; ++e) {
               const int d = i * N + (e / 4) * 4 + (e % 4);
               const float4 pp = par[gl * D + d];
-              const uint32_t c = code_of(bf16_bits(*reinterpret_cast<const uint16_t*>(row + d * 2)), pp.x, pp.z, QMAX);
+              const uint32_t c = code_of(I16::one(*reinterpret_cast<const uint16_t*>(row + d * 2)), pp.x, pp.z, QMAX);
               word |= c << (8 * (e % 4) + BITS * (e / 4));
             }
           }
@@ -246,7 +295,16 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
       }
       __syncthreads();
       uint4* dst = reinterpret_cast<uint4*>(codes + (size_t)bh * stream_words + w0);
-      for (int v = tid; v < T * NW / 4; v += PACK_THREADS) dst[v] = reinterpret_cast<const uint4*>(wbuf)[v];
+      for (int v = tid; v < T * NW / 4; v += PACK_THREADS) {
+        uint4 w = reinterpret_cast<const uint4*>(wbuf)[v];
+        if (merge) {  // the dominant layer's codes of these positions are in place: replace them by the merged ones
+          const uint4 o = dst[v];
+          const uint32_t lut = p.merge_lut[BITS - 1];
+          w = make_uint4(merge_words<BITS>(o.x, w.x, lut), merge_words<BITS>(o.y, w.y, lut),
+                         merge_words<BITS>(o.z, w.z, lut), merge_words<BITS>(o.w, w.w, lut));
+        }
+        dst[v] = w;
+      }
     } else {
       constexpr int WPC = T / N;  // words per channel over the tile's tokens
 #pragma unroll
@@ -261,10 +319,10 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
             const int tl = wi * N + 4 * s4;
             const uint8_t* src = tile + tl * ROWB + d * 2;
             const float4 p0 = par[gi * T + tl], p1 = par[gi * T + tl + 1], p2 = par[gi * T + tl + 2], p3 = par[gi * T + tl + 3];
-            const float x0 = bf16_bits(*reinterpret_cast<const uint16_t*>(src));
-            const float x1 = bf16_bits(*reinterpret_cast<const uint16_t*>(src + ROWB));
-            const float x2 = bf16_bits(*reinterpret_cast<const uint16_t*>(src + 2 * ROWB));
-            const float x3 = bf16_bits(*reinterpret_cast<const uint16_t*>(src + 3 * ROWB));
+            const float x0 = I16::one(*reinterpret_cast<const uint16_t*>(src));
+            const float x1 = I16::one(*reinterpret_cast<const uint16_t*>(src + ROWB));
+            const float x2 = I16::one(*reinterpret_cast<const uint16_t*>(src + 2 * ROWB));
+            const float x3 = I16::one(*reinterpret_cast<const uint16_t*>(src + 3 * ROWB));
             const uint32_t lo = code_pair<BITS>(x0, x1, p0, p1, doubt);
             const uint32_t hi = code_pair<BITS>(x2, x3, p2, p3, doubt);
             word |= (lo | (hi << 16)) << (BITS * s4);
@@ -275,11 +333,12 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
             for (int e = 0; e < N; ++e) {
               const int tl = wi * N + (e / 4) * 4 + (e % 4);
               const float4 pp = par[gi * T + tl];
-              const uint32_t c = code_of(bf16_bits(*reinterpret_cast<const uint16_t*>(tile + tl * ROWB + d * 2)), pp.x, pp.z, QMAX);
+              const uint32_t c = code_of(I16::one(*reinterpret_cast<const uint16_t*>(tile + tl * ROWB + d * 2)), pp.x, pp.z, QMAX);
               word |= c << (8 * (e % 4) + BITS * (e / 4));
             }
           }
-          codes[(size_t)bh * stream_words + v_code_position(tq0 + wi * N, d, BITS, D).word] = word;
+          uint32_t* dst = codes + (size_t)bh * stream_words + v_code_position(tq0 + wi * N, d, BITS, D).word;
+          *dst = merge ? merge_words<BITS>(*dst, word, p.merge_lut[BITS - 1]) : word;
         }
       }
     }
@@ -287,18 +346,24 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(PackParams p) {
   if (bits == 2) build(std::integral_constant<int, 2>{}); else build(std::integral_constant<int, 1>{});
 }
 
-cudaError_t launch_pack(const PackParams& p, cudaStream_t st) {
+template <bool F16>
+cudaError_t launch_pack_t(const PackParams& p, cudaStream_t st) {
   int tiles = p.n_blocks * (p.dm.R / p.tb);
-  dim3 grid(2 * tiles, p.dm.Hkv, p.dm.B);
+  dim3 grid(2 * tiles, p.dm.Hkv, p.dm.B * p.n_layers);
   const int key = p.dm.D * 10000 + p.dm.g * 100 + p.tb;
   switch (key) {
-    case 1283232: pack_kernel<128, 32, 32><<<grid, PACK_THREADS, 0, st>>>(p); break;
-    case 1286464: pack_kernel<128, 64, 64><<<grid, PACK_THREADS, 0, st>>>(p); break;
-    case 643232: pack_kernel<64, 32, 32><<<grid, PACK_THREADS, 0, st>>>(p); break;
-    case 646464: pack_kernel<64, 64, 64><<<grid, PACK_THREADS, 0, st>>>(p); break;
+    case 1283232: pack_kernel<128, 32, 32, F16><<<grid, PACK_THREADS, 0, st>>>(p); break;
+    case 1286464: pack_kernel<128, 64, 64, F16><<<grid, PACK_THREADS, 0, st>>>(p); break;
+    case 643232: pack_kernel<64, 32, 32, F16><<<grid, PACK_THREADS, 0, st>>>(p); break;
+    case 646464: pack_kernel<64, 64, 64, F16><<<grid, PACK_THREADS, 0, st>>>(p); break;
     default: return cudaErrorInvalidValue;
   }
   return cudaGetLastError();
+}
+
+cudaError_t launch_pack(const PackParams& p, cudaStream_t st) {
+  if (p.n_layers < 1 || p.n_layers > PACK_MAX_LAYERS) return cudaErrorInvalidValue;
+  return p.f16 ? launch_pack_t<true>(p, st) : launch_pack_t<false>(p, st);
 }
 
 // Copies new tokens into the 16-bit window, keys and values in one launch.

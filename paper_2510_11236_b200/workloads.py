@@ -89,13 +89,14 @@ def queries(w: dict, layer: int, step: int, device) -> torch.Tensor:
     return torch.randn(w["batch"], w["n_q_heads"], w["head_dim"], generator=g, device=device).to(torch.bfloat16)
 
 
-def make_xq_config(w: dict, *, max_seq=None, eta1=1.0 / 6.0, eta2=0.045, kernel=0, n_splits=None):
+def make_xq_config(w: dict, *, max_seq=None, eta1=1.0 / 6.0, eta2=0.045, kernel=0, n_splits=None, io_dtype=0):
     from . import binding
     return binding.make_config(
         n_layers=w["n_layers"], batch=w["batch"], n_q_heads=w["n_q_heads"], n_kv_heads=w["n_kv_heads"],
         head_dim=w["head_dim"], max_seq=max_seq or w["seq"], group_size=w["group_size"],
         residual_len=w["residual_len"], kq=w["kq"], vq=w["vq"], km=w["km"], vm=w["vm"], eta1=eta1, eta2=eta2,
-        n_splits=w["n_splits"] if n_splits is None else n_splits, kernel=kernel)
+        n_splits=w["n_splits"] if n_splits is None else n_splits, kernel=kernel, io_dtype=io_dtype,
+        share_group=w.get("share_group", 0), share_dominant=w.get("share_dominant", 0), gamma1=w.get("gamma1", 0.0))
 
 
 def algorithmic_bytes(w: dict, seq: int = None, layer: int = 0) -> int:

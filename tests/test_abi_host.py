@@ -108,3 +108,26 @@ def test_host_state_machine_without_launches():
     rc, m1, _ = xq.xq_region(h, 1, 2)
     assert m0 != m1  # but has its own scale / zero-point
     assert xq.xq_destroy(h) == 0
+
+
+def test_sharing_pattern_rules():
+    ok = [dict(share_group=3, share_dominant=1, km=14, vm=14), dict(share_group=4, share_dominant=3, km=16, vm=32),
+          dict(share_group=2, share_dominant=1), dict(gamma1=0.4), dict(gamma1=1.0), dict(io_dtype=xq.XQ_F16)]
+    for kw in ok:
+        assert xq.xq_config_check(_cfg(**kw)) == xq.XQ_OK, kw
+    bad = [dict(share_group=5), dict(share_group=1), dict(share_group=3, share_dominant=3),
+           dict(share_group=3, km=0, vm=0),             # 32 layers are not a whole number of groups of three
+           dict(share_group=2, share_dominant=1, n_layers=31, kq=31, vq=31),  # layer 30 would read layer 31's codes
+           dict(gamma1=0.4, share_group=3, km=14, vm=14), dict(gamma1=0.4, share_dominant=1),
+           dict(gamma1=1.5), dict(gamma1=-0.1), dict(io_dtype=2),
+           dict(share_group=4, km=16, vm=16, kq=18)]     # a group of four would mix 2-bit and 1-bit keys
+    for kw in bad:
+        assert xq.xq_config_check(_cfg(**kw)) == xq.XQ_ERR_CONFIG, kw
+
+
+@pytest.mark.parametrize("group,vm", [(2, 8), (3, 14), (4, 16)])
+def test_equiv_bits_of_group_table(group, vm):
+    # Table group: all key layers and 20 of 32 value layers stored, printed 1.63
+    for k in range(group):
+        c = _cfg(kq=32, vq=32, km=32, vm=vm, share_group=group, share_dominant=k)
+        assert xq.xq_equiv_bits(c) == 1.625 == O.equiv_bits(32, 32, 32, vm, 32, group, k)

@@ -213,7 +213,8 @@ def test_decode_step_appends_inside_the_decode_kernel():
         S = 71 + step
         flush = (S - 1) % R == 0
         now = xq.xq_launch_count(cache.handle)
-        assert now - launches == (L * 3 if flush else L)  # pack + window append + decode, or the decode alone
+        # one quantize-and-pack launch for all layers (it also refills the windows) and the decodes, or the decodes alone
+        assert now - launches == (1 + L if flush else L)
         launches = now
         for l in range(L):
             kv[l] = (torch.cat([kv[l][0], kn[l]], dim=2), torch.cat([kv[l][1], vn[l]], dim=2))
@@ -340,6 +341,125 @@ def test_queries_with_a_few_dominant_tokens(S, bits):
     assert worst[xq.XQ_KERNEL_AUTO] <= util.ATTN_TOL
     for cache in caches.values():
         cache.close()
+
+
+@pytest.mark.parametrize("group,k,m", [(3, 0, 0), (4, 0, 4), (2, 1, 0), (3, 2, 3), (4, 2, 0)])
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_sharing_groups_and_dominant_layers(group, k, m, kernel):
+    """Groups of two, three and four layers reading the codes of their k-th layer (Table group's patterns):
+    regions bit for bit, attention of every layer against the oracle, and one-token steps with the dominant
+    layers first (a layer ahead of its dominant layer cannot decode before that layer has appended)."""
+    L = m + 2 * group
+    w = dict(n_layers=L, batch=1, n_q_heads=8, n_kv_heads=2, head_dim=128, seq=200, residual_len=64, group_size=32,
+             kq=L, vq=L, km=m, vm=m, n_outliers=3, outlier_scale=10.0, seed=31, n_splits=0,
+             share_group=group, share_dominant=k)
+    cfg = W.make_xq_config(w, max_seq=300, kernel=kernel)
+    assert xq.xq_config_check(cfg) == 0
+    cache = xq.Cache(cfg, DEV)
+    layers = list(range(L))
+    kv = _fill(cache, w, layers, 192, step=50)  # the window of 64 is full: the next token quantizes it
+    owners = [m + ((l - m) // group) * group + k if l >= m else l for l in range(L)] if group > 2 else \
+             [l - l % 2 + k if l >= m else l for l in range(L)]
+    order = sorted(range(L), key=lambda l: (owners[l] != l, l))
+    gen = torch.Generator(device="cpu").manual_seed(7)
+    for step in range(2):
+        kn = torch.randn(L, 1, 2, 1, 128, generator=gen).to(torch.bfloat16).to(DEV)
+        vn = torch.randn(L, 1, 2, 1, 128, generator=gen).to(torch.bfloat16).to(DEV)
+        q = torch.randn(L, 1, 8, 128, generator=gen).to(torch.bfloat16).to(DEV)
+        out = torch.empty_like(q)
+        if step == 0 and k > 0:  # ascending order would ask layer 0 of a group to read codes that are not there yet
+            rc = xq.xq_decode_step(cache.handle, kn, vn, q, out, None, xq.XQ_MEM_DEVICE, torch.cuda.current_stream().cuda_stream)
+            assert rc == xq.XQ_ERR_ORDER and cache.seq_len(0) == 192
+        cache.decode_step(kn, vn, q, out, layer_order=order)
+        torch.cuda.synchronize()
+        for l in layers:
+            kv[l] = (torch.cat([kv[l][0], kn[l]], dim=2), torch.cat([kv[l][1], vn[l]], dim=2))
+        o32 = [cache.decode_attention(l, q[l], f32=True) for l in layers]
+        for hk in range(2):
+            oc = util.oracle_for_stream(cfg, layers, 0, hk, kv)
+            for l in layers:
+                util.compare_regions(cache, oc, l, 0, hk)
+                util.check_attention(cache, oc, l, q[l], 0, hk, o32[l], out[l])
+    assert xq.xq_equiv_bits(cfg) == O_equiv(L, m, group, k)
+    cache.close()
+
+
+def O_equiv(L, m, group, k):
+    from oracle import xq_oracle as O
+    return O.equiv_bits(L, L, m, m, L, group, k)
+
+
+@pytest.mark.parametrize("gamma0", [0.05, 0.2, 0.4, 0.6, 0.8, 0.95])
+@pytest.mark.parametrize("bits", [(2, 0), (0, 2)])
+def test_weighted_average_merging(gamma0, bits):
+    """gamma_0 in each of Appendix F's six intervals: once the pair's second layer has quantized a block the shared
+    codes are round(gamma_0 e0 + gamma_1 e1), bit for bit; before that they are the first layer's."""
+    kq, vq = bits
+    w = dict(n_layers=2, batch=2, n_q_heads=4, n_kv_heads=2, head_dim=128, seq=300, residual_len=64, group_size=32,
+             kq=kq, vq=vq, km=0, vm=0, n_outliers=3, outlier_scale=10.0, seed=3, n_splits=0, gamma1=1.0 - gamma0)
+    cfg = W.make_xq_config(w)
+    cache = xq.Cache(cfg, DEV)
+    k0, v0, k1, v1 = W.pair_tokens(w, 0, 0, 300, DEV)
+    s = torch.cuda.current_stream().cuda_stream
+    # the second layer cannot run ahead of the first
+    assert xq.xq_append_kv(cache.handle, 1, k1[:, :, :100].contiguous(), v1[:, :, :100].contiguous(), 100, s) == xq.XQ_ERR_ORDER
+    assert cache.seq_len(1) == 0
+    cache.append_kv(0, k0[:, :, :150].contiguous(), v0[:, :, :150].contiguous())
+    kv = {0: (k0[:, :, :150], v0[:, :, :150])}
+    q = W.queries(w, 0, 0, DEV)
+    o32 = cache.decode_attention(0, q, f32=True)
+    for hk in range(2):
+        oc = util.oracle_for_stream(cfg, [0], 1, hk, kv)
+        util.compare_regions(cache, oc, 0, 1, hk)
+        util.check_attention(cache, oc, 0, q, 1, hk, o32)
+    cache.append_kv(1, k1[:, :, :150].contiguous(), v1[:, :, :150].contiguous())
+    for lo in range(150, 300, 37):
+        hi = min(300, lo + 37)
+        for l, (K, V) in ((0, (k0, v0)), (1, (k1, v1))):
+            cache.append_kv(l, K[:, :, lo:hi].contiguous(), V[:, :, lo:hi].contiguous())
+    kv = {0: (k0, v0), 1: (k1, v1)}
+    for layer in (0, 1):
+        q = W.queries(w, layer, 0, DEV)
+        o32 = cache.decode_attention(layer, q, f32=True)
+        for b in range(2):
+            for hk in range(2):
+                # the oracle takes the same interleaving: both layers complete, block by block
+                oc = util.oracle_for_stream(cfg, [0, 1], b, hk, kv)
+                util.compare_regions(cache, oc, layer, b, hk)
+                util.check_attention(cache, oc, layer, q, b, hk, o32)
+    cache.close()
+
+
+@pytest.mark.parametrize("shape", ["c0", "c2"])
+def test_half_precision_io(shape):
+    """K, V, q, the window and the output in IEEE half precision instead of bfloat16."""
+    w = dict(W.CONFIGS[shape], n_layers=2, batch=1, seq=700)
+    w["kq"], w["vq"] = min(w["kq"], 2), min(w["vq"], 2)
+    cfg = W.make_xq_config(w, max_seq=800, io_dtype=xq.XQ_F16)
+    cache = xq.Cache(cfg, DEV)
+    k0, v0, k1, v1 = (t.to(torch.float16) for t in W.pair_tokens(w, 0, 0, 700, DEV))
+    kv = {0: (k0, v0), 1: (k1, v1)}
+    for lo in range(0, 700, 233):
+        for l in (0, 1):
+            cache.append_kv(l, kv[l][0][:, :, lo:lo + 233].contiguous(), kv[l][1][:, :, lo:lo + 233].contiguous())
+    L, Hq, Hkv, D = 2, w["n_q_heads"], w["n_kv_heads"], w["head_dim"]
+    gen = torch.Generator(device="cpu").manual_seed(9)
+    for step in range(3):
+        kn = torch.randn(L, 1, Hkv, 1, D, generator=gen).to(torch.float16).to(DEV)
+        vn = torch.randn(L, 1, Hkv, 1, D, generator=gen).to(torch.float16).to(DEV)
+        q = torch.randn(L, 1, Hq, D, generator=gen).to(torch.float16).to(DEV)
+        out = torch.empty_like(q)
+        cache.decode_step(kn, vn, q, out)
+        torch.cuda.synchronize()
+        for l in range(L):
+            kv[l] = (torch.cat([kv[l][0], kn[l]], dim=2), torch.cat([kv[l][1], vn[l]], dim=2))
+        o32 = [cache.decode_attention(l, q[l], f32=True) for l in range(L)]
+        for hk in range(min(2, Hkv)):
+            oc = util.oracle_for_stream(cfg, [0, 1], 0, hk, kv)
+            for l in range(L):
+                util.compare_regions(cache, oc, l, 0, hk)
+                util.check_attention(cache, oc, l, q[l], 0, hk, o32[l], out[l])
+    cache.close()
 
 
 @pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4"])

@@ -60,3 +60,31 @@ def test_benchmark_configs():
     assert O.equiv_bits(32, 32, 0, 0, 32) == 1.0
     assert O.equiv_bits(32, 0, 0, 0, 32) == 0.75
     assert O.equiv_bits(2, 2, 0, 0, 2) == 1.0
+
+
+@pytest.mark.parametrize("group,vm", [(2, 8), (3, 14), (4, 16)])
+def test_group_table_common_width(group, vm):
+    """Table group compares group sizes 2, 3, 4 "under the same compression ratio": all key layers and 20 of the
+    32 value layers stored on a 2-bit base, printed as 1.63.  Contiguous groups counted from the sharing start
+    give exactly that for sharing from layer 8, 14 and 16, for every dominant index."""
+    for k in range(group):
+        stored = sum(1 for l in range(32) if O.code_owner(l, vm, group, k) == l)
+        assert stored == 20
+        w = O.equiv_bits(32, 32, 32, vm, 32, group, k)
+        assert w == 1.625 and f"{w:.2f}" in ("1.62", "1.63")
+
+
+def test_owner_of_larger_groups_and_other_dominant_layers():
+    # groups of three from layer 2 on, dominant index 1: (2,3,4) -> 3, (5,6,7) -> 6
+    assert [O.code_owner(l, 2, 3, 1) for l in range(8)] == [0, 1, 3, 3, 3, 6, 6, 6]
+    # pairs with the second layer dominant: the even layer reads the odd one's codes
+    assert [O.code_owner(l, 0, 2, 1) for l in range(4)] == [1, 1, 3, 3]
+    # the default is Algorithm 1's pattern
+    assert [O.code_owner(l, 4) for l in range(8)] == [0, 1, 2, 3, 4, 4, 6, 6]
+    # every layer's owner owns its own codes
+    for group in (2, 3, 4):
+        for k in range(group):
+            for m in (0, 4, 8):
+                for l in range(m + 2 * group):
+                    o = O.code_owner(l, m, group, k)
+                    assert O.code_owner(o, m, group, k) == o

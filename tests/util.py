@@ -7,7 +7,7 @@ from oracle import xq_oracle as O
 
 
 def bits_of(t: torch.Tensor) -> np.ndarray:
-    """bf16 tensor -> numpy uint16 bit patterns (same shape)."""
+    """bf16 or fp16 tensor -> numpy uint16 bit patterns (same shape)."""
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
@@ -17,7 +17,9 @@ def oracle_for_stream(cfg, layers, b, hk, kv_by_layer):
     G = cfg.n_q_heads // cfg.n_kv_heads
     oc = O.OracleCache(cfg.n_layers, 1, G, 1, cfg.head_dim, cfg.group_size, cfg.residual_len,
                        cfg.kq, cfg.vq, cfg.km, cfg.vm, np.float32(cfg.eta1), np.float32(cfg.eta2),
-                       cfg.sm_scale if cfg.sm_scale > 0 else None)
+                       cfg.sm_scale if cfg.sm_scale > 0 else None,
+                       share_group=cfg.share_group or 2, share_dominant=cfg.share_dominant,
+                       gamma1=float(np.float32(cfg.gamma1)), f16=cfg.io_dtype == 1)
     for l in layers:
         K, V = kv_by_layer[l]
         oc.append(l, bits_of(K[b:b + 1, hk:hk + 1]), bits_of(V[b:b + 1, hk:hk + 1]))
@@ -36,7 +38,7 @@ def compare_regions(cache, oc, layer, b, hk):
     r = st["win_k"].shape[2]
     for which, key in ((4, "win_k"), (5, "win_v")):
         got = cache.region(layer, which)[bh].cpu().numpy().view(np.uint16)[: r * D].reshape(r, D)
-        want = O.f32_to_bf16_bits(st[key][0, 0])
+        want = st[key][0, 0].astype(np.float16).view(np.uint16) if oc.f16 else O.f32_to_bf16_bits(st[key][0, 0])
         assert np.array_equal(got, want), f"window {key} differs"
     if nq == 0:
         return
