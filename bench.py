@@ -33,8 +33,38 @@ METRIC = "decode-attention GB/s at 32k ctx"
 APPEND_BLOCKS = 6  # window blocks quantized per layer in the append pass, one block per call
 BULK_BLOCKS = 16   # then two calls per layer of this many blocks each (a prefill-sized append)
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the decode kernel (ncu, same launch shape as the
-# timed one; see profiles/).  Valid only for the kernel version the counters were taken on.
-NCU_TRAFFIC_BYTES = {"c2": 84.03e6 + 2.59e6}
+# timed one; see profiles/), with the SHA-256 of the kernel's sources at the time the counters were taken: the
+# figure is reported only while the sources still hash to that.
+NCU_TRAFFIC = {"c2": {"bytes": 84.07e6 + 2.63e6,
+                      "sources_sha256": "unset"}}
+KERNEL_SOURCES = ("xq_decode_umma.cu", "xq_layout.cuh", "xq_internal.h")
+
+
+def _kernel_sources_hash():
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2510_11236_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def _ncu_traffic(config):
+    t = NCU_TRAFFIC.get(config)
+    if t is None or t["sources_sha256"] != _kernel_sources_hash():
+        return None
+    return t["bytes"]
+
+
+def _config_block(args, w):
+    """What both arms print as `config`: the workload by name and its shape."""
+    return {"workload": f"{args.config}: BASELINE.json configs[{args.config[1:]}]",
+            **{k: w[k] for k in ("n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "seq", "residual_len",
+                                 "group_size", "kq", "vq", "km", "vm")},
+            "eta1": args.eta1, "eta2": args.eta2,
+            "step": "per layer: append 1 token (+ quantize-and-pack when the window block fills) and decode attention",
+            "l2": "inputs larger than L2: every step streams the whole packed cache (GBs against 126 MB of L2); "
+                  "owners-first layer order keeps a pair's shared codes from being re-served by L2"}
 
 
 def _peaks():
@@ -47,7 +77,7 @@ def _peaks():
 
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while a region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -60,7 +90,11 @@ class ClockSampler:
         except Exception:
             self.p = None
 
-    def stop(self):
+    def stop(self, t_lo=None, t_hi=None):
+        """Median SM clock and the throttle reasons seen.  With a window [t_lo, t_hi] (datetime, local time) the
+        figures come from the samples inside it when there are any (`window`: "timed region"), else from every
+        sample since the sampler started (`window`: "whole run": warm-up and all passes)."""
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
         if self.p is None:
             return out
@@ -71,16 +105,22 @@ class ClockSampler:
             self.p.kill()
         self.f.flush()
         self.f.seek(0)
-        clocks, mx, reasons = [], [], set()
+        rows = []
         for line in self.f.read().splitlines():
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 9:
                 continue
             try:
-                clocks.append(float(parts[1])); mx.append(float(parts[2]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f")
+                rows.append((ts, float(parts[1]), float(parts[2]), parts[5:9]))
             except ValueError:
                 continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+        inside = [r for r in rows if t_lo is not None and t_lo <= r[0] <= t_hi]
+        out["window"] = "timed region" if inside else "whole run"
+        clocks, mx, reasons = [], [], set()
+        for ts, c, m, flags in (inside or rows):
+            clocks.append(c); mx.append(m)
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), flags):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         try:
@@ -140,6 +180,30 @@ class OracleSample:
         return time.perf_counter() - t0
 
 
+def _oracle_worker(job):
+    """One process of the all-cores figure: builds one stream's oracle cache, then runs decode passes for about
+    `seconds`; returns (passes, seconds spent in them, bytes per pass)."""
+    w, eta1, eta2, seconds = job
+    smp = OracleSample(w, 1, eta1, eta2)
+    smp.run()
+    dt, passes = 0.0, 0
+    while dt < seconds:
+        dt += smp.run()
+        passes += 1
+    return passes, dt, smp.bytes
+
+
+def oracle_all_cores(w, eta1, eta2, seconds=6.0):
+    """The oracle on every host core at once: one single-threaded process per core (at most 32), each on its own
+    stream; the figure is the sum of the processes' rates."""
+    import multiprocessing as mp
+    n = max(1, min(os.cpu_count() or 1, 32))
+    ctx = mp.get_context("spawn")
+    with ctx.Pool(n) as pool:
+        res = pool.map(_oracle_worker, [(w, eta1, eta2, seconds)] * n)
+    return sum(p * b / dt for p, dt, b in res) / 1e9, n
+
+
 def run_reference(args, w):
     """The reference arm: the CPU oracle timed on this machine's host cores."""
     rank = int(os.environ.get("RANK", "0"))
@@ -160,8 +224,9 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": T * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.config, **{k: w[k] for k in ("n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "seq", "residual_len", "group_size", "kq", "vq", "km", "vm")}},
-        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "config": _config_block(args, w),
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": 1, "host_cores": os.cpu_count(), "kind": "oracle",
+                         "sample": sample},
         "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -263,6 +328,8 @@ def main():
                 tot += W.algorithmic_bytes(w, first_seq + i, l)
         return tot
 
+    import datetime
+    sampler = ClockSampler(local) if rank == 0 else None  # runs from before the warm-up to the end of pass 3
     for _ in range(Wm):
         device_step()
     barrier()
@@ -270,16 +337,16 @@ def main():
     # ---- pass 1: whole steps, inputs resident in HBM
     seq_before = cache.seq_len(0)
     launches_before = xq.xq_launch_count(cache.handle)
-    sampler = ClockSampler(local) if rank == 0 else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    t_lo = datetime.datetime.now()
     e0.record()
     for _ in range(K):
         device_step()
     e1.record()
     barrier()
+    t_hi = datetime.datetime.now()
     ms = e0.elapsed_time(e1)
-    clocks = sampler.stop() if sampler else None
     launches = xq.xq_launch_count(cache.handle) - launches_before
     bytes_pass1 = step_bytes(seq_before + 1, K)
     ms_max = sharding.max_over_ranks(ms, dev)
@@ -327,6 +394,7 @@ def main():
     ms3_max = sharding.max_over_ranks(ms3, dev)
     e2e_val = sharding.aggregate_rate(step_bytes(seq_before3 + 1, K), ms3_max, world) / 1e9
 
+    clocks = sampler.stop(t_lo, t_hi) if sampler else None
     rc, nsq, nsw = xq.xq_split_plan(cache.handle, 0)  # the decode launches' split plan (before the appends below)
 
     # ---- pass 4: the quantize-and-pack path: every layer receives whole window blocks (R tokens per call), so each
@@ -374,16 +442,13 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f16 mma operands, f32 accumulate, bf16 io", "data": "synthetic",
-            "config": {"workload": f"{args.config}: BASELINE.json configs[{args.config[1:]}]",
-                       **{k: w[k] for k in ("n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "seq",
-                                            "residual_len", "group_size", "kq", "vq", "km", "vm")},
-                       "eta1": args.eta1, "eta2": args.eta2, "equiv_bits": xq.xq_equiv_bits(cfg),
-                       "step": "per layer: append 1 token (+ quantize-and-pack when the window block fills) and decode attention",
-                       "layer_order": args.layer_order,
-                       "l2": "inputs larger than L2: each step streams ~%.1f GB of cache; owners-first layer order keeps a pair's shared codes from being re-served by L2" % (bytes_pass1 / K / 1e9),
-                       "splits_quantized": nsq, "splits_window": nsw,
-                       "algorithmic_bytes_per_layer_call": W.algorithmic_bytes(w, S, 0)},
+            "dtype": "u8 x u8 -> s32 tensor-core products (24-bit fixed-point operands), f32 softmax, bf16 io",
+            "data": "synthetic",
+            "config": _config_block(args, w),
+            "run": {"equiv_bits": xq.xq_equiv_bits(cfg), "layer_order": args.layer_order,
+                    "bytes_streamed_per_step_gb": bytes_pass1 / K / 1e9,
+                    "splits_quantized": nsq, "splits_window": nsw,
+                    "algorithmic_bytes_per_layer_call": W.algorithmic_bytes(w, S, 0)},
             "frac_of_8TBps": value / world / 8000.0,
             "frac_of_measured_hbm": value / world / peak,
             "attended_tokens_per_s": tokens_per_s,
@@ -394,7 +459,7 @@ def main():
             "roofline": {"bound": "hbm", "kernel": "decode split kernel", "achieved": achieved, "peak": peak,
                          "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                          "frac_of_8TBps": achieved / 8000.0,
-                         "traffic": NCU_TRAFFIC_BYTES.get(args.config) if not (args.layers or args.seq or args.splits) else None,
+                         "traffic": _ncu_traffic(args.config) if not (args.layers or args.seq or args.splits) else None,
                          "algorithmic_bytes_per_launch": bytes_pass1 / decode_launches_pass1,
                          "avg_launch_us": avg_launch_us, "launches": decode_launches_pass1,
                          "timing": "CUDA events around the timed region of back-to-back launches, divided by the decode launches in it",
@@ -402,6 +467,11 @@ def main():
                                       "launches": dec["launches"],
                                       "timing": "CUDA events around every launch (no overlap of a launch's prologue with its predecessor's tail)"}},
             "kernels": kinds,
+            "flush_step": {"what": "the step on which every layer's window block fills: one quantize-and-pack launch for "
+                                   "all layers before that step's decode launches",
+                           "pack_launches": kinds["quantize_pack"]["launches"],
+                           "pack_avg_us": kinds["quantize_pack"]["avg_us"],
+                           "step_ms_without_it": ms_max / K},
             "append": append,
         }
         if not args.no_cpu_baseline and world == 1:
@@ -411,10 +481,14 @@ def main():
             while dt < 12.0 and passes < 16:  # about 10-30 s of CPU work
                 dt += smp.run()
                 passes += 1
+            all_val, all_n = oracle_all_cores(w, args.eta1, args.eta2)
             line["cpu_baseline"] = {
                 "value": passes * smp.bytes / dt / 1e9, "unit": "GB/s", "cores": smp.cores, "kind": "oracle",
+                "host_cores": os.cpu_count(),
                 "sample": f"decode attention of one layer for {n_streams} of {B * Hkv} (sequence, kv head) streams at S={S} "
-                          f"(dequantize + attention, fp64 numpy), {passes} passes, {dt:.1f} s"}
+                          f"(dequantize + attention, fp64 numpy), {passes} passes, {dt:.1f} s",
+                "all_cores": {"value": all_val, "unit": "GB/s", "cores": all_n,
+                              "sample": f"{all_n} single-threaded processes, one stream each at S={S}, ~6 s of passes each"}}
         print(json.dumps(line), flush=True)
     cache.close()
     if world > 1:

@@ -164,6 +164,19 @@ int xq_decode_attention(xq_cache* c, int layer, const void* q, void* out, void* 
  * head_dim] (the accumulator before the final rounding to bfloat16). */
 int xq_decode_attention_f32(xq_cache* c, int layer, const void* q, float* out, void* stream);
 
+/* Attention of the last n_q_tokens tokens of `layer` as queries (a prefill chunk,
+ * or the prompt / output workload of Appendix D), causal inside the chunk: the
+ * keys and values of these tokens are already in the cache (xq_append_kv), and
+ * query token j (0 .. n_q_tokens - 1) attends to the tokens 0 .. S - n_q_tokens + j,
+ * S the layer's length -- packed tokens through their codes, window tokens as they
+ * are, exactly as xq_decode_attention does for the tokens it sees; n_q_tokens = 1
+ * is xq_decode_attention.  q, out: device, [n_q_tokens, batch, n_q_heads, head_dim]
+ * contiguous (token-major: one token's slice is a decode call's q), io_dtype;
+ * 16-byte aligned.  The _f32 variant writes float results (tests).  Errors as
+ * xq_decode_attention; 1 <= n_q_tokens <= S. */
+int xq_attention_chunk(xq_cache* c, int layer, const void* q, void* out, int n_q_tokens, void* stream);
+int xq_attention_chunk_f32(xq_cache* c, int layer, const void* q, float* out, int n_q_tokens, void* stream);
+
 /* xq_decode_attention for callers that cannot provide scratch memory of their
  * own.  (The paper has no counterpart: this is a deployment variant, not part of
  * the method.)  Some hosts hand every byte of device memory to their own pools at

@@ -400,6 +400,24 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, sm_scale: float) -> n
     return p @ v
 
 
+def attention_chunk(q: np.ndarray, k: np.ndarray, v: np.ndarray, sm_scale: float) -> np.ndarray:
+    """The last T cached tokens as queries, causal inside the chunk (the prompt /
+    output workload of Appendix D processed a chunk at a time): query j sees the
+    tokens 0 .. S - T + j.  Plain definition: masked softmax attention in fp64.
+    q: [T, D], k, v: [S, D] -> [T, D]."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    T, S = q.shape[0], k.shape[0]
+    logits = sm_scale * (q @ k.T)
+    visible = np.arange(S)[None, :] <= (S - T + np.arange(T))[:, None]
+    logits = np.where(visible, logits, -np.inf)
+    logits = logits - logits.max(axis=1, keepdims=True)
+    p = np.exp(logits)
+    p = p / p.sum(axis=1, keepdims=True)
+    return p @ v
+
+
 # --------------------------------------------------------------------------
 # Whole cache: Algorithm 1 with the residual window
 # --------------------------------------------------------------------------
@@ -564,4 +582,22 @@ class OracleCache:
                 cache[(b, hk)] = self.dequantized(l, b, hk)
             kh, vh = cache[(b, hk)]
             out[b, h] = attention(q[b, h], kh, vh, self.sm_scale)
+        return out
+
+    def attention_chunk(self, l: int, q_bits16: np.ndarray, pairs=None) -> np.ndarray:
+        """q_bits16: [T, B, H_q, D] bit patterns: the queries of the layer's last T
+        tokens.  Returns fp64 [T, B, H_q, D]; packed tokens enter through their
+        dequantized values, window tokens as they are, as in decode."""
+        q = self._widen(q_bits16).astype(np.float64)
+        T = q.shape[0]
+        G = self.Hq // self.Hkv
+        out = np.full((T, self.B, self.Hq, self.D), np.nan, dtype=np.float64)
+        todo = pairs if pairs is not None else [(b, h) for b in range(self.B) for h in range(self.Hq)]
+        cache = {}
+        for (b, h) in todo:
+            hk = h // G
+            if (b, hk) not in cache:
+                cache[(b, hk)] = self.dequantized(l, b, hk)
+            kh, vh = cache[(b, hk)]
+            out[:, b, h] = attention_chunk(q[:, b, h], kh, vh, self.sm_scale)
         return out

@@ -49,6 +49,10 @@ _SIGNATURES = {
                                                ctypes.c_void_p]),
     "xq_decode_attention_static": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
                                                   ctypes.c_void_p]),
+    "xq_attention_chunk": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                                          ctypes.c_void_p]),
+    "xq_attention_chunk_f32": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                              ctypes.c_int, ctypes.c_void_p]),
     "xq_decode_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                       ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.c_int,
                                       ctypes.c_void_p]),
@@ -143,6 +147,14 @@ def xq_decode_attention_f32(handle, layer: int, q, out, stream: int = 0) -> int:
 
 def xq_decode_attention_static(handle, layer: int, q, out, stream: int = 0) -> int:
     return lib().xq_decode_attention_static(handle, layer, _ptr(q), _ptr(out), stream)
+
+
+def xq_attention_chunk(handle, layer: int, q, out, n_q_tokens: int, stream: int = 0) -> int:
+    return lib().xq_attention_chunk(handle, layer, _ptr(q), _ptr(out), n_q_tokens, stream)
+
+
+def xq_attention_chunk_f32(handle, layer: int, q, out, n_q_tokens: int, stream: int = 0) -> int:
+    return lib().xq_attention_chunk_f32(handle, layer, _ptr(q), _ptr(out), n_q_tokens, stream)
 
 
 def xq_decode_step(handle, K_new, V_new, q, out, layer_order=None, mem: int = XQ_MEM_DEVICE, stream: int = 0) -> int:
@@ -263,6 +275,17 @@ class Cache:
         rc = fn(self.handle, layer, q, out, self._stream())
         if rc:
             raise XQError(rc, "xq_decode_attention")
+        return out
+
+    def attention_chunk(self, layer, q, out=None, f32=False):
+        """q: [n_q_tokens, batch, n_q_heads, head_dim]."""
+        import torch
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32 if f32 else q.dtype, device=q.device)
+        fn = xq_attention_chunk_f32 if f32 else xq_attention_chunk
+        rc = fn(self.handle, layer, q, out, q.shape[0], self._stream())
+        if rc:
+            raise XQError(rc, "xq_attention_chunk")
         return out
 
     def decode_step(self, K_new, V_new, q, out, layer_order=None, mem=XQ_MEM_DEVICE):

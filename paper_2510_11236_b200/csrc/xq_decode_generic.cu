@@ -41,10 +41,10 @@ __global__ void __launch_bounds__(GEN_WARPS * 32) decode_generic_kernel(DecodePa
   bool quant = split < p.ns_q;
   int t0, t1;
   if (quant) {
-    int units = p.n_q / 32;
+    int units = (p.n_q + 31) / 32;  // the last unit is ragged when a visibility limit cuts the packed region
     share_of(units, p.ns_q, split, t0, t1);
     t0 *= 32;
-    t1 *= 32;
+    t1 = min(t1 * 32, p.n_q);
   } else {
     int sw = split - p.ns_q;
     int tiles = (p.r + 15) / 16;

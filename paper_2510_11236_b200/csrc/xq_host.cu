@@ -210,11 +210,10 @@ int mma_ctas_per_sm(const xq_cache* c, int l) {
 // tokens): every split takes whole batches of the packed region and a share of the
 // window (ns_w = 0), sized towards whole waves of resident CTAs.  Generic kernel:
 // separate splits for the packed region and for the window, in proportion to their bytes.
-void plan_splits(const xq_cache* c, int l, int& ns_q, int& ns_w, int* n_ctas_out = nullptr) {
+// nq packed tokens and r window tokens are visible to the call.
+void plan_splits(const xq_cache* c, int l, int nq, int r, int& ns_q, int& ns_w, int* n_ctas_out = nullptr) {
   const Dims& dm = c->plan.dm;
-  int S = c->seq[l];
-  int r = residual_count(S, dm.R), nq = S - r;
-  int units = nq / 32, tiles = (r + 15) / 16;
+  int units = (nq + 31) / 32, tiles = (r + 15) / 16;
   const int streams = dm.B * dm.Hkv;
   if (layer_uses_mma(c, l) && nq > 0) {
     // the tensor-core kernel: whole 128-token batches per CTA, every CTA also takes a share of the window
@@ -308,9 +307,10 @@ struct Scratch {
 
 // Checks a decode call and fills the kernel parameters (everything but the scratch).  Touches no state.
 // K_new / V_new: one new token per stream that the tensor-core kernel appends itself; S_eff is the layer's
-// length with that token counted.
+// length with that token counted.  vis >= 0: only the first vis tokens are visible to the query (a query token of
+// a chunk that is followed by later tokens in the cache).
 int prepare_decode(const xq_cache* c, int layer, const void* q, void* out, int out_f32, const void* K_new,
-                   const void* V_new, int S_eff, DecodeParams& p, bool& use_mma) {
+                   const void* V_new, int S_eff, DecodeParams& p, bool& use_mma, int vis = -1) {
   if (!c || !q || !out) return XQ_ERR_ARG;
   if (layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
   if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return XQ_ERR_ARG;
@@ -318,7 +318,11 @@ int prepare_decode(const xq_cache* c, int layer, const void* q, void* out, int o
   const Dims& dm = c->plan.dm;
   const int S = S_eff;
   if (S < 1) return XQ_ERR_ARG;
-  const int r = residual_count(S, dm.R), nq = S - r;
+  int r = residual_count(S, dm.R), nq = S - r;
+  if (vis >= 0) {
+    if (vis < 1 || vis > S) return XQ_ERR_ARG;
+    if (vis < nq) { nq = vis; r = 0; } else { r = vis - nq; }
+  }
   // a code-borrowing layer needs the owning layer's codes for all of its quantized tokens
   for (int o : {k_owner(&c->cfg, layer), v_owner(&c->cfg, layer)}) {
     if (o != layer && c->seq[o] - residual_count(c->seq[o], dm.R) < nq) return XQ_ERR_ORDER;
@@ -332,14 +336,7 @@ int prepare_decode(const xq_cache* c, int layer, const void* q, void* out, int o
   p.n_q = nq;
   p.r = r;
   p.n_ctas = 0;
-  {
-    // plan_splits reads the layer's length from the handle: give it the effective one
-    xq_cache* cc = const_cast<xq_cache*>(c);
-    const int keep = cc->seq[layer];
-    cc->seq[layer] = S;
-    plan_splits(c, layer, p.ns_q, p.ns_w, &p.n_ctas);
-    cc->seq[layer] = keep;
-  }
+  plan_splits(c, layer, nq, r, p.ns_q, p.ns_w, &p.n_ctas);
   p.scale = c->scale;
   p.out = out;
   p.out_f32 = out_f32;
@@ -467,12 +464,12 @@ int pack_layers(xq_cache* c, const int* layers, int n, const void* K, const void
 }
 
 int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, cudaStream_t st,
-                const void* K_new = nullptr, const void* V_new = nullptr) {
+                const void* K_new = nullptr, const void* V_new = nullptr, int vis = -1) {
   if (!c) return XQ_ERR_ARG;
   if (layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
   DecodeParams p;
   bool use_mma = false;
-  int rc = prepare_decode(c, layer, q, out, out_f32, K_new, V_new, c->seq[layer] + (K_new ? 1 : 0), p, use_mma);
+  int rc = prepare_decode(c, layer, q, out, out_f32, K_new, V_new, c->seq[layer] + (K_new ? 1 : 0), p, use_mma, vis);
   if (rc != XQ_OK) return rc;
   if (use_mma) {
     rc = ensure_clean_scratch(c, st);
@@ -601,6 +598,43 @@ int xq_decode_attention(xq_cache* c, int layer, const void* q, void* out, void* 
 
 int xq_decode_attention_f32(xq_cache* c, int layer, const void* q, float* out, void* stream) {
   return decode_impl(c, layer, q, out, 1, (cudaStream_t)stream);
+}
+
+namespace {
+// Query token j of n sees the cache up to its own position; one decode launch per token (their visible ranges
+// differ), all on the same stream.
+int chunk_impl(xq_cache* c, int layer, const void* q, void* out, int n, int out_f32, void* stream) {
+  if (!c || !q || !out) return XQ_ERR_ARG;
+  if (layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
+  const int S = c->seq[layer];
+  if (n < 1 || n > S) return XQ_ERR_ARG;
+  if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return XQ_ERR_ARG;
+  const Dims& dm = c->plan.dm;
+  // everything that can be refused is the same for every token: check the first and the last before any launch
+  {
+    DecodeParams p;
+    bool use_mma;
+    int rc = prepare_decode(c, layer, q, out, out_f32, nullptr, nullptr, S, p, use_mma, S - n + 1);
+    if (rc == XQ_OK) rc = prepare_decode(c, layer, q, out, out_f32, nullptr, nullptr, S, p, use_mma, S);
+    if (rc != XQ_OK) return rc;
+  }
+  const size_t row = (size_t)dm.B * dm.Hq * dm.D;  // elements of one token's queries: [batch, heads, head_dim]
+  for (int j = 0; j < n; ++j) {
+    const uint8_t* qj = (const uint8_t*)q + (size_t)j * row * 2;
+    uint8_t* oj = (uint8_t*)out + (size_t)j * row * (out_f32 ? 4 : 2);
+    const int rc = decode_impl(c, layer, qj, oj, out_f32, (cudaStream_t)stream, nullptr, nullptr, S - n + 1 + j);
+    if (rc != XQ_OK) return rc;
+  }
+  return XQ_OK;
+}
+}  // namespace
+
+int xq_attention_chunk(xq_cache* c, int layer, const void* q, void* out, int n_q_tokens, void* stream) {
+  return chunk_impl(c, layer, q, out, n_q_tokens, 0, stream);
+}
+
+int xq_attention_chunk_f32(xq_cache* c, int layer, const void* q, float* out, int n_q_tokens, void* stream) {
+  return chunk_impl(c, layer, q, out, n_q_tokens, 1, stream);
 }
 
 int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out, void* stream) {
@@ -764,7 +798,10 @@ int xq_quantized_len(const xq_cache* c, int layer) {
 int xq_split_plan(const xq_cache* c, int layer, int* nsq, int* nsw) {
   if (!c || !nsq || !nsw || layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
   if (c->seq[layer] < 1) return XQ_ERR_ARG;
-  plan_splits(c, layer, *nsq, *nsw);
+  {
+    const int S = c->seq[layer], r = residual_count(S, c->plan.dm.R);
+    plan_splits(c, layer, S - r, r, *nsq, *nsw);
+  }
   return XQ_OK;
 }
 

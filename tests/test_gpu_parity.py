@@ -462,6 +462,44 @@ def test_half_precision_io(shape):
     cache.close()
 
 
+@pytest.mark.parametrize("T", [1, 4, 16, 64])
+@pytest.mark.parametrize("shape", ["mha", "gqa", "d64"])
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_attention_chunk(T, shape, kernel):
+    """The last T tokens as queries, causal inside the chunk, on MHA and GQA shapes: every row against the oracle.
+    With a window of 32 and 9 tokens in it, chunks of 16 and 64 reach into the packed region (their first queries
+    see only a part of it)."""
+    Hq, Hkv, D = {"mha": (4, 4, 128), "gqa": (8, 2, 128), "d64": (6, 2, 64)}[shape]
+    S = 393  # 384 quantized + 9 in the window
+    w = dict(n_layers=2, batch=2, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, seq=S, residual_len=32, group_size=32,
+             kq=2, vq=0, km=0, vm=0, n_outliers=3, outlier_scale=10.0, seed=41, n_splits=0)
+    cfg = W.make_xq_config(w, kernel=kernel)
+    cache = xq.Cache(cfg, DEV)
+    kv = _fill(cache, w, [0, 1], S, step=131)
+    gen = torch.Generator(device="cpu").manual_seed(T)
+    for layer in (0, 1):
+        q = torch.randn(T, 2, Hq, D, generator=gen).to(torch.bfloat16).to(DEV)
+        o32 = cache.attention_chunk(layer, q, f32=True)
+        o16 = cache.attention_chunk(layer, q)
+        torch.cuda.synchronize()
+        if T == 1:
+            assert torch.equal(o16[0], cache.decode_attention(layer, q[0]))
+        G = Hq // Hkv
+        for b in range(2):
+            for hk in range(Hkv):
+                oc = util.oracle_for_stream(cfg, [0, 1], b, hk, kv)
+                ref = oc.attention_chunk(layer, util.bits_of(q[:, b:b + 1, hk * G:(hk + 1) * G]))[:, 0]
+                got = o32[:, b, hk * G:(hk + 1) * G].double().cpu().numpy()
+                assert np.abs(got - ref).max() <= util.ATTN_TOL
+                got16 = o16[:, b, hk * G:(hk + 1) * G].double().cpu().numpy()
+                assert (np.abs(got16 - ref) <= util.ATTN_TOL + 2.0 ** -8 * np.abs(ref)).all()
+    s = torch.cuda.current_stream().cuda_stream
+    q = torch.zeros(2, 2, Hq, D, dtype=torch.bfloat16, device=DEV)
+    assert xq.xq_attention_chunk(cache.handle, 0, q, q.clone(), S + 1, s) == xq.XQ_ERR_ARG
+    assert xq.xq_attention_chunk(cache.handle, 0, q, q.clone(), 0, s) == xq.XQ_ERR_ARG
+    cache.close()
+
+
 @pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4"])
 def test_full_size_configs_sampled(name):
     """The benchmark's shapes and launch configuration (library-chosen splits, tensor-core kernel), one layer

@@ -165,3 +165,64 @@ def test_quantization_error_is_small_relative_to_two_bit_step():
     rng_k = kf[:32].max(axis=0) - kf[:32].min(axis=0)
     assert (np.abs(kh[:32] - kf[:32]) <= (rng_k / 3) * (0.5 + 0.045 * 3) * 1.01 + 1e-3).all()
     assert np.array_equal(kh[32:], kf[32:])
+
+
+# ---- chunk attention (the last T tokens as queries, causal inside the chunk)
+
+def test_chunk_of_one_is_decode():
+    rng = np.random.default_rng(0)
+    q, k, v = rng.standard_normal((1, 16)), rng.standard_normal((9, 16)), rng.standard_normal((9, 16))
+    assert np.array_equal(O.attention_chunk(q, k, v, 0.25)[0], O.attention(q[0], k, v, 0.25))
+
+
+def test_chunk_against_explicit_loops():
+    rng = np.random.default_rng(1)
+    S, T, D = 11, 4, 8
+    q, k, v = rng.standard_normal((T, D)), rng.standard_normal((S, D)), rng.standard_normal((S, D))
+    got = O.attention_chunk(q, k, v, 0.3)
+    for j in range(T):
+        n = S - T + j + 1  # tokens visible to query j
+        logit = [0.3 * sum(q[j][d] * k[t][d] for d in range(D)) for t in range(n)]
+        mx = max(logit)
+        w = [np.exp(x - mx) for x in logit]
+        for d in range(D):
+            want = sum(w[t] * v[t][d] for t in range(n)) / sum(w)
+            assert abs(got[j][d] - want) < 1e-12
+
+
+def test_chunk_rows_ignore_later_tokens_and_the_last_row_sees_all():
+    rng = np.random.default_rng(2)
+    S, T, D = 20, 5, 8
+    q, k, v = rng.standard_normal((T, D)), rng.standard_normal((S, D)), rng.standard_normal((S, D))
+    base = O.attention_chunk(q, k, v, 0.5)
+    assert np.allclose(base[T - 1], O.attention(q[T - 1], k, v, 0.5), rtol=0, atol=1e-14)
+    for j in range(T - 1):
+        k2, v2 = k.copy(), v.copy()
+        k2[S - T + j + 1:] += 100.0  # tokens after query j's own position
+        v2[S - T + j + 1:] -= 50.0
+        again = O.attention_chunk(q, k2, v2, 0.5)
+        assert np.array_equal(again[j], base[j])
+        assert not np.allclose(again[T - 1], base[T - 1])
+    # a row equals a decode call over its visible prefix
+    for j in range(T):
+        n = S - T + j + 1
+        assert np.allclose(base[j], O.attention(q[j], k[:n], v[:n], 0.5), rtol=0, atol=1e-14)
+
+
+def test_cache_chunk_matches_cache_decode_for_one_token():
+    rng = np.random.default_rng(3)
+    D, S = 64, 75
+    oc = O.OracleCache(1, 1, 2, 1, D, 32, 32, 1, 1, 1, 1, np.float32(1 / 6), np.float32(0.045))
+    x = O.f32_to_bf16_bits(rng.standard_normal((1, 1, S, D)).astype(np.float32))
+    y = O.f32_to_bf16_bits(rng.standard_normal((1, 1, S, D)).astype(np.float32))
+    oc.append(0, x, y)
+    q = O.f32_to_bf16_bits(rng.standard_normal((1, 1, 2, D)).astype(np.float32))
+    assert np.array_equal(oc.attention_chunk(0, q)[0], oc.decode(0, q[0]))
+    # a chunk longer than the window reaches into the quantized region
+    q = O.f32_to_bf16_bits(rng.standard_normal((40, 1, 2, D)).astype(np.float32))
+    got = oc.attention_chunk(0, q)
+    kh, vh = oc.dequantized(0, 0, 0)
+    qf = O.bf16_bits_to_f32(q).astype(np.float64)
+    for j in (0, 17, 39):
+        n = S - 40 + j + 1
+        assert np.allclose(got[j, 0, 1], O.attention(qf[j, 0, 1], kh[:n], vh[:n], oc.sm_scale), rtol=0, atol=1e-13)
