@@ -113,6 +113,12 @@ typedef struct xq_config {
                              pair's codes by round(gamma_0 e_0 + gamma1 e_1), ties to even
                              (evaluated in double precision); until then the block holds
                              the first layer's codes e_0                                  */
+  int32_t delta_stats;    /* 1: every layer that reads another layer's codes also quantizes
+                             its own blocks (codes not stored) and counts, per cache kind,
+                             the elements by |own code - shared code| -- the statistic of
+                             Section 3.3.1 (Figure delta) on the caller's own data, read
+                             with xq_delta_histogram.  Costs the code computation the
+                             accelerated scheme saves; 0 (default): off                  */
 } xq_config;
 
 #define XQ_MAX_SPLITS 256
@@ -233,6 +239,15 @@ int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void
  * has an iteration limit instead of the ability to hang the GPU.  XQ_OK otherwise.
  * Synchronizes; not for the hot path. */
 int xq_check_device(xq_cache* c, void* stream);
+
+/* Code-similarity statistic of Section 3.3.1 (needs delta_stats = 1 in the
+ * configuration): counts[d], d = 0..3, is the number of quantized elements of
+ * `layer` (kind 0: keys, 1: values; all sequences and heads, every block packed
+ * since xq_create or xq_reset) whose own code differs by d from the code it reads
+ * from its group's dominant layer (before any merging of that block).  Zero for a
+ * layer that keeps its own codes.  Waits for `stream`; not for the hot path.
+ * XQ_ERR_CONFIG without delta_stats. */
+int xq_delta_histogram(xq_cache* c, int layer, int kind, unsigned long long counts[4], void* stream);
 
 /* Equivalent bit-width of Appendix C: stored code bits per cached element,
  * averaged over layers and over keys and values; scale / zero-point excluded,

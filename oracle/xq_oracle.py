@@ -435,7 +435,7 @@ class OracleCache:
 
     def __init__(self, n_layers, batch, n_q_heads, n_kv_heads, head_dim, group_size,
                  residual_len, kq, vq, km, vm, eta1, eta2, sm_scale=None,
-                 share_group=2, share_dominant=0, gamma1=0.0, f16=False):
+                 share_group=2, share_dominant=0, gamma1=0.0, f16=False, delta_stats=False):
         self.L, self.B, self.Hq, self.Hkv, self.D = n_layers, batch, n_q_heads, n_kv_heads, head_dim
         self.g, self.R = group_size, residual_len
         self.kq, self.vq, self.km, self.vm = kq, vq, km, vm
@@ -445,6 +445,10 @@ class OracleCache:
         # merged codes (0: the dominant layer's codes are shared as they are); f16: inputs are IEEE half precision
         self.share_group, self.share_dominant, self.gamma1 = share_group or 2, share_dominant, gamma1
         self.f16 = f16
+        # Section 3.3.1: per layer and cache kind, the number of quantized elements whose own code differs by
+        # d = 0..3 from the code the layer reads from its dominant layer (layers that keep their codes: zeros)
+        self.delta_stats = delta_stats
+        self.delta = np.zeros((n_layers, 2, 4), dtype=np.int64)
         assert self.gamma1 == 0.0 or (self.share_group == 2 and self.share_dominant == 0)
         assert n_q_heads % n_kv_heads == 0 and residual_len % group_size == 0
         assert head_dim % group_size == 0
@@ -483,7 +487,9 @@ class OracleCache:
         st = self.layers[l]
         B, H = self.B, self.Hkv
         mrg_k, mrg_v = self._merges(l, self.km), self._merges(l, self.vm)
-        own_k, own_v = self.k_owner(l) == l or mrg_k, self.v_owner(l) == l or mrg_v
+        cmp_k = self.delta_stats and self.k_owner(l) != l
+        cmp_v = self.delta_stats and self.v_owner(l) != l
+        own_k, own_v = self.k_owner(l) == l or mrg_k or cmp_k, self.v_owner(l) == l or mrg_v or cmp_v
         bk, bv = self.k_bits(l), self.v_bits(l)
         kc, ks, kz, vc, vs, vz = [], [], [], [], [], []
         for b in range(B):
@@ -498,6 +504,16 @@ class OracleCache:
 
         blk = len(st["k_s"])  # index of the block being quantized
         kcs, vcs = stack(kc), stack(vc)
+        for kind, cmp, own, key, mine in ((0, cmp_k, self.k_owner(l), "k_codes", kcs), (1, cmp_v, self.v_owner(l), "v_codes", vcs)):
+            if cmp:
+                shared = self.layers[own][key]
+                assert len(shared) > blk, "the dominant layer must have quantized this block"
+                d = np.abs(shared[blk].astype(np.int64) - mine.astype(np.int64))
+                self.delta[l, kind] += np.bincount(d.reshape(-1), minlength=4)[:4]
+        if not mrg_k and self.k_owner(l) != l:
+            kcs = None
+        if not mrg_v and self.v_owner(l) != l:
+            vcs = None
         if mrg_k:  # the pair's codes of this block: weighted average with the first layer's, rounded
             first = self.layers[l - 1]["k_codes"]
             assert len(first) > blk, "the pair's first layer must have quantized this block"

@@ -31,6 +31,7 @@ class xq_config(ctypes.Structure):
         ("eta1", ctypes.c_float), ("eta2", ctypes.c_float), ("sm_scale", ctypes.c_float),
         ("n_splits", ctypes.c_int32), ("io_dtype", ctypes.c_int32), ("kernel", ctypes.c_int32),
         ("share_group", ctypes.c_int32), ("share_dominant", ctypes.c_int32), ("gamma1", ctypes.c_float),
+        ("delta_stats", ctypes.c_int32),
     ]
 
 
@@ -57,6 +58,8 @@ _SIGNATURES = {
                                       ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.c_int,
                                       ctypes.c_void_p]),
     "xq_check_device": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
+    "xq_delta_histogram": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                          ctypes.POINTER(ctypes.c_ulonglong), ctypes.c_void_p]),
     "xq_equiv_bits": (ctypes.c_double, [ctypes.POINTER(xq_config)]),
     "xq_seq_len": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
     "xq_quantized_len": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int]),
@@ -168,6 +171,12 @@ def xq_check_device(handle, stream: int = 0) -> int:
     return lib().xq_check_device(handle, stream)
 
 
+def xq_delta_histogram(handle, layer: int, kind: int, stream: int = 0):
+    counts = (ctypes.c_ulonglong * 4)()
+    rc = lib().xq_delta_histogram(handle, layer, kind, counts, stream)
+    return rc, [int(x) for x in counts]
+
+
 def xq_equiv_bits(cfg: xq_config) -> float:
     return lib().xq_equiv_bits(ctypes.byref(cfg))
 
@@ -216,10 +225,12 @@ def xq_strerror(code: int) -> str:
 
 def make_config(*, n_layers, batch, n_q_heads, n_kv_heads, head_dim, max_seq, group_size=32, residual_len=128,
                 kq=None, vq=None, km=0, vm=0, eta1=0.0, eta2=0.0, sm_scale=0.0, n_splits=0,
-                kernel=XQ_KERNEL_AUTO, io_dtype=XQ_BF16, share_group=0, share_dominant=0, gamma1=0.0) -> xq_config:
+                kernel=XQ_KERNEL_AUTO, io_dtype=XQ_BF16, share_group=0, share_dominant=0, gamma1=0.0,
+                delta_stats=0) -> xq_config:
     return xq_config(n_layers, batch, n_q_heads, n_kv_heads, head_dim, max_seq, group_size, residual_len,
                      n_layers if kq is None else kq, n_layers if vq is None else vq, km, vm,
-                     eta1, eta2, sm_scale, n_splits, io_dtype, kernel, share_group, share_dominant, gamma1)
+                     eta1, eta2, sm_scale, n_splits, io_dtype, kernel, share_group, share_dominant, gamma1,
+                     delta_stats)
 
 
 class Cache:

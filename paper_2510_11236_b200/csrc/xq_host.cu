@@ -42,7 +42,7 @@ struct LayerRegions {
 struct Plan {
   Dims dm;
   std::vector<LayerRegions> layers;
-  size_t part_acc, part_ml, tickets, status, staging, total;
+  size_t part_acc, part_ml, tickets, status, delta, staging, total;
   size_t staging_kv_bytes, staging_q_bytes;
 };
 
@@ -68,6 +68,7 @@ bool check(const xq_config* c) {
   if (c->share_dominant < 0 || c->share_dominant >= group) return false;
   if (!(c->gamma1 >= 0.f && c->gamma1 <= 1.f)) return false;
   if (c->gamma1 > 0.f && (group != 2 || c->share_dominant != 0)) return false;
+  if (c->delta_stats != 0 && c->delta_stats != 1) return false;
   if (group > 2 && ((c->n_layers - c->km) % group || (c->n_layers - c->vm) % group)) return false;
   // every layer reads the codes of a layer that exists and has its bit-width
   for (int l = 0; l < c->n_layers; ++l) {
@@ -111,6 +112,7 @@ void make_plan(const xq_config* c, Plan& pl) {
   pl.part_ml = take((size_t)dm.B * dm.Hq * XQ_MAX_SPLITS * 2 * 4);
   pl.tickets = take(BH * 4);
   pl.status = take(4);
+  pl.delta = take((size_t)c->n_layers * 2 * 4 * 8);  // per layer and cache kind: elements by code difference 0..3
   pl.staging_kv_bytes = (size_t)c->n_layers * BH * dm.D * 2;
   pl.staging_q_bytes = (size_t)c->n_layers * dm.B * dm.Hq * dm.D * 2;
   pl.staging = take(2 * align_up(pl.staging_kv_bytes, 256) + 2 * align_up(pl.staging_q_bytes, 256));
@@ -157,6 +159,7 @@ struct xq_cache {
   int device;            // CUDA device the handle was created on (-1: none)
   uint8_t* static_base;  // device address of the library's static scratch array on that device (null: not resolved)
   bool tickets_clean;  // the ticket counters have been zeroed on a stream
+  bool delta_clean;    // the code-difference counters have been zeroed on a stream
   std::vector<uint8_t> repacked;  // per layer: codes or parameters it reads were written since its last decode
   int mma_ctas[2][2];  // resident CTAs per SM of the tensor-core kernel by (key bits - 1, value bits - 1); 0 = not asked yet
   // timing
@@ -437,17 +440,28 @@ int pack_layers(xq_cache* c, const int* layers, int n, const void* K, const void
     pl.L = layer_ptrs(c, l);
     pl.K_in = (const uint16_t*)((const uint8_t*)K + (size_t)i * layer_stride);
     pl.V_in = (const uint16_t*)((const uint8_t*)V + (size_t)i * layer_stride);
-    pl.own_k = k_owner(&c->cfg, l) == l ? 1 : (merges_codes(&c->cfg, l, c->cfg.km) ? 2 : 0);
-    pl.own_v = v_owner(&c->cfg, l) == l ? 1 : (merges_codes(&c->cfg, l, c->cfg.vm) ? 2 : 0);
-    if (pl.own_k == 2 || pl.own_v == 2) {
+    const int ok = k_owner(&c->cfg, l), ov = v_owner(&c->cfg, l);
+    const int stat = c->cfg.delta_stats ? 4 : 0;
+    pl.own_k = ok == l ? 1 : ((merges_codes(&c->cfg, l, c->cfg.km) ? 2 : 0) | stat);
+    pl.own_v = ov == l ? 1 : ((merges_codes(&c->cfg, l, c->cfg.vm) ? 2 : 0) | stat);
+    pl.delta_k = (unsigned long long*)(c->ws + c->plan.delta) + (size_t)(l * 2 + 0) * 4;
+    pl.delta_v = (unsigned long long*)(c->ws + c->plan.delta) + (size_t)(l * 2 + 1) * 4;
+    if (pl.own_k > 1 || pl.own_v > 1) {
+      // the layer reads the codes its dominant layer wrote for these blocks: that layer must hold them, and the
+      // launch that wrote them must be another one
       if (n != 1) return XQ_ERR_ARG;
-      const int o = l - 1;  // the pair's first layer must hold the blocks this layer merges into
-      if (c->seq[o] - residual_count(c->seq[o], dm.R) < nq_new) return XQ_ERR_ORDER;
+      for (int o : {ok, ov})
+        if (o != l && c->seq[o] - residual_count(c->seq[o], dm.R) < nq_new) return XQ_ERR_ORDER;
     }
     pl.eta_k = pl.L.bk == 1 ? c->cfg.eta1 : c->cfg.eta2;
     pl.eta_v = pl.L.bv == 1 ? c->cfg.eta1 : c->cfg.eta2;
   }
   cudaError_t e;
+  if (c->cfg.delta_stats && !c->delta_clean) {
+    e = cudaMemsetAsync(c->ws + c->plan.delta, 0, (size_t)c->cfg.n_layers * 2 * 4 * 8, st);
+    if (e != cudaSuccess) return fail_cuda(c, e);
+    c->delta_clean = true;
+  }
   {
     Timer t(c, st, 2);
     e = launch_pack(p, st);
@@ -521,6 +535,7 @@ int xq_create(const xq_config* cfg, void* dev_workspace, size_t bytes, xq_cache*
   c->used = 0;
   c->sm_count = 148;
   c->tickets_clean = false;
+  c->delta_clean = false;
   c->device = -1;
   c->static_base = nullptr;
   memset(c->mma_ctas, 0, sizeof(c->mma_ctas));
@@ -554,6 +569,7 @@ int xq_reset(xq_cache* c) {
   for (auto& s : c->seq) s = 0;
   for (auto& r : c->repacked) r = 1;  // as after xq_create: the first decode of a layer waits for its predecessor
   c->tickets_clean = false;           // tickets and status are cleared again before their next use
+  c->delta_clean = false;             // and so are the code-difference counters
   return XQ_OK;
 }
 
@@ -723,7 +739,7 @@ int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void
     for (int l = 1; l < L; ++l) same = same && c->seq[l] == c->seq[0];
     const int s_old = c->seq[0];
     const int nq_old = s_old - residual_count(s_old, dm.R), nq_new = s_old + 1 - residual_count(s_old + 1, dm.R);
-    if (same && nq_new > nq_old && c->cfg.gamma1 == 0.f) {
+    if (same && nq_new > nq_old && c->cfg.gamma1 == 0.f && !c->cfg.delta_stats) {
       for (int c0 = 0; c0 < L; c0 += PACK_MAX_LAYERS) {
         int idx[PACK_MAX_LAYERS];
         const int n = L - c0 < PACK_MAX_LAYERS ? L - c0 : PACK_MAX_LAYERS;
@@ -772,6 +788,19 @@ int xq_check_device(xq_cache* c, void* stream) {
   e = cudaMemcpy(&status, c->ws + c->plan.status, 4, cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return fail_cuda(c, e);
   return status ? XQ_ERR_DEVICE : XQ_OK;
+}
+
+int xq_delta_histogram(xq_cache* c, int layer, int kind, unsigned long long counts[4], void* stream) {
+  if (!c || !counts) return XQ_ERR_ARG;
+  if (layer < 0 || layer >= c->cfg.n_layers || kind < 0 || kind > 1) return XQ_ERR_ARG;
+  if (!c->cfg.delta_stats) return XQ_ERR_CONFIG;
+  for (int k = 0; k < 4; ++k) counts[k] = 0ull;
+  cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (!c->delta_clean) return XQ_OK;  // nothing has been counted yet
+  e = cudaMemcpy(counts, c->ws + c->plan.delta + (size_t)(layer * 2 + kind) * 4 * 8, 4 * 8, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  return XQ_OK;
 }
 
 double xq_equiv_bits(const xq_config* cfg) {

@@ -27,9 +27,13 @@ struct PackLayer {
   const uint16_t* K_in;  // [B,Hkv,n_in,D] new tokens (absolute positions s_old ..)
   const uint16_t* V_in;
   // codes of a cache kind: 0 = none (the layer keeps scale and zero-point only), 1 = written, 2 = merged into the
-  // codes the dominant layer wrote (weighted average, Appendix F)
+  // codes the dominant layer wrote (weighted average, Appendix F); 4 = computed for the statistic only; 6 = both
   int own_k, own_v;
   float eta_k, eta_v;
+  // with bit 2 set in own_*: count the elements by |own code - stored code| into these four counters (before the
+  // codes are merged, if they are)
+  unsigned long long* delta_k;
+  unsigned long long* delta_v;
 };
 
 constexpr int PACK_MAX_LAYERS = 32;  // layers one launch can take (they share every length below)

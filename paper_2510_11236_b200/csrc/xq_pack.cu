@@ -103,6 +103,18 @@ __device__ __forceinline__ uint32_t code_pair(float x0, float x1, const float4& 
   return __byte_perm(__float_as_uint(u0), __float_as_uint(u1), 0x0040) & (QM | (QM << 8));
 }
 
+// Adds to hist[d] the number of fields of the two words whose codes differ by d.
+template <int BITS>
+__device__ __forceinline__ void delta_count(uint32_t w0, uint32_t w1, uint32_t (&hist)[4]) {
+#pragma unroll
+  for (int f = 0; f < 32; f += BITS) {
+    const int e0 = (int)((w0 >> f) & ((1u << BITS) - 1u)), e1 = (int)((w1 >> f) & ((1u << BITS) - 1u));
+    const int d = e0 > e1 ? e0 - e1 : e1 - e0;
+#pragma unroll
+    for (int k = 0; k < (1 << BITS); ++k) hist[k] += d == k;
+  }
+}
+
 // One CTA: T tokens x D channels of one (sequence, kv head), keys (blockIdx.x even) or values (odd).  Staged
 // rows are padded.  Keys: a thread builds whole words of a token's row (four consecutive channels per bit
 // offset), the words are collected in shared memory in stream order and leave in 16-byte vectors.  Values: a
@@ -254,7 +266,8 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
 
   // codes
   uint32_t* codes = kind ? pl.L.v_codes : pl.L.k_codes;
-  const bool merge = own == 2;
+  const bool merge = (own & 2) != 0, stats = (own & 4) != 0, store = (own & 3) != 0;
+  uint32_t hist[4] = {0u, 0u, 0u, 0u};
   const size_t stream_words = (size_t)dm.nq_cap * D * bits / 32;
   auto build = [&](auto bits_c) {
     constexpr int BITS = decltype(bits_c)::value;
@@ -297,13 +310,17 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
       uint4* dst = reinterpret_cast<uint4*>(codes + (size_t)bh * stream_words + w0);
       for (int v = tid; v < T * NW / 4; v += PACK_THREADS) {
         uint4 w = reinterpret_cast<const uint4*>(wbuf)[v];
-        if (merge) {  // the dominant layer's codes of these positions are in place: replace them by the merged ones
+        if (merge || stats) {  // the dominant layer's codes of these positions are in place
           const uint4 o = dst[v];
+          if (stats) {
+            delta_count<BITS>(o.x, w.x, hist); delta_count<BITS>(o.y, w.y, hist);
+            delta_count<BITS>(o.z, w.z, hist); delta_count<BITS>(o.w, w.w, hist);
+          }
           const uint32_t lut = p.merge_lut[BITS - 1];
           w = make_uint4(merge_words<BITS>(o.x, w.x, lut), merge_words<BITS>(o.y, w.y, lut),
                          merge_words<BITS>(o.z, w.z, lut), merge_words<BITS>(o.w, w.w, lut));
         }
-        dst[v] = w;
+        if (store) dst[v] = w;
       }
     } else {
       constexpr int WPC = T / N;  // words per channel over the tile's tokens
@@ -338,12 +355,25 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
             }
           }
           uint32_t* dst = codes + (size_t)bh * stream_words + v_code_position(tq0 + wi * N, d, BITS, D).word;
-          *dst = merge ? merge_words<BITS>(*dst, word, p.merge_lut[BITS - 1]) : word;
+          if (merge || stats) {
+            const uint32_t o = *dst;
+            if (stats) delta_count<BITS>(o, word, hist);
+            word = merge_words<BITS>(o, word, p.merge_lut[BITS - 1]);
+          }
+          if (store) *dst = word;
         }
       }
     }
   };
   if (bits == 2) build(std::integral_constant<int, 2>{}); else build(std::integral_constant<int, 1>{});
+  if (stats) {
+    unsigned long long* out = kind ? pl.delta_v : pl.delta_k;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t tot = __reduce_add_sync(0xffffffffu, hist[k]);
+      if ((tid & 31) == 0 && tot) atomicAdd(out + k, (unsigned long long)tot);
+    }
+  }
 }
 
 template <bool F16>

@@ -31,6 +31,10 @@ CONFIGS = {
     # long context, 64 splits per head
     "c4": dict(n_layers=32, batch=1, n_q_heads=32, n_kv_heads=8, head_dim=128, seq=131072, residual_len=128,
                group_size=32, kq=32, vq=0, km=0, vm=0, n_outliers=3, outlier_scale=10.0, seed=4, n_splits=64),
+    # Qwen2.5-14B-shaped GQA (48 layers, 40 query heads on 8 kv heads: groups of five), the paper's second model
+    # family (Table qwen); 2-bit keys, the upper half of the value layers 1-bit
+    "q14": dict(n_layers=48, batch=4, n_q_heads=40, n_kv_heads=8, head_dim=128, seq=16384, residual_len=128,
+                group_size=32, kq=48, vq=24, km=0, vm=0, n_outliers=3, outlier_scale=10.0, seed=5, n_splits=0),
 }
 
 NOISE_SIGMA = 0.1
@@ -96,7 +100,8 @@ def make_xq_config(w: dict, *, max_seq=None, eta1=1.0 / 6.0, eta2=0.045, kernel=
         head_dim=w["head_dim"], max_seq=max_seq or w["seq"], group_size=w["group_size"],
         residual_len=w["residual_len"], kq=w["kq"], vq=w["vq"], km=w["km"], vm=w["vm"], eta1=eta1, eta2=eta2,
         n_splits=w["n_splits"] if n_splits is None else n_splits, kernel=kernel, io_dtype=io_dtype,
-        share_group=w.get("share_group", 0), share_dominant=w.get("share_dominant", 0), gamma1=w.get("gamma1", 0.0))
+        share_group=w.get("share_group", 0), share_dominant=w.get("share_dominant", 0), gamma1=w.get("gamma1", 0.0),
+        delta_stats=w.get("delta_stats", 0))
 
 
 def algorithmic_bytes(w: dict, seq: int = None, layer: int = 0) -> int:

@@ -500,6 +500,119 @@ def test_attention_chunk(T, shape, kernel):
     cache.close()
 
 
+@pytest.mark.parametrize("bits", [(2, 2), (2, 0), (0, 0)])
+def test_delta_histogram(bits):
+    """The pack kernel's optional statistic (Section 3.3.1): per layer and cache kind the elements by
+    |own code - shared code|, against the oracle's count, exactly; the cache's contents are unchanged by it."""
+    kq, vq = bits
+    w = dict(n_layers=4, batch=2, n_q_heads=4, n_kv_heads=2, head_dim=128, seq=333, residual_len=64, group_size=32,
+             kq=kq, vq=vq, km=2, vm=0, n_outliers=3, outlier_scale=10.0, seed=13, n_splits=0, delta_stats=1)
+    cfg = W.make_xq_config(w)
+    cache = xq.Cache(cfg, DEV)
+    layers = [0, 1, 2, 3]
+    kv = _fill(cache, w, layers, 333, step=77)
+    s = torch.cuda.current_stream().cuda_stream
+    want = np.zeros((4, 2, 4), dtype=np.int64)
+    for b in range(2):
+        for hk in range(2):
+            oc = util.oracle_for_stream(cfg, layers, b, hk, kv)
+            want += oc.delta
+            for l in layers:
+                util.compare_regions(cache, oc, l, b, hk)
+    for l in layers:
+        for kind in (0, 1):
+            rc, got = xq.xq_delta_histogram(cache.handle, l, kind, s)
+            assert rc == 0 and got == list(want[l, kind]), (l, kind, got, list(want[l, kind]))
+    assert want[1, 0].sum() == 0 and want[1, 1].sum() == 2 * 2 * 320 * 128  # keys shared from layer 2 on, values from 0
+    plain = xq.Cache(W.make_xq_config(dict(w, delta_stats=0)), DEV)
+    assert xq.xq_delta_histogram(plain.handle, 1, 0, s)[0] == xq.XQ_ERR_CONFIG
+    plain.close()
+    cache.close()
+
+
+def test_decode_right_after_the_pack_of_the_layer_it_reads():
+    """A layer that reads another layer's codes decodes immediately after that layer packed a large append, many
+    times on one stream with nothing in between: the decode kernel must not fetch packed data ahead of the pack
+    kernel that is still writing it.  Every result against the oracle."""
+    w = dict(W.CONFIGS["c2"], n_layers=2, batch=4, seq=8192 + 100)
+    w["kq"], w["vq"] = 2, 0
+    R = w["residual_len"]
+    cfg = W.make_xq_config(w, max_seq=8192 + 16 * 4 * R + 200)
+    cache = xq.Cache(cfg, DEV)
+    kv = _fill(cache, w, [0, 1], 8192 + 100, step=2048)
+    gen = torch.Generator(device="cpu").manual_seed(21)
+    B, Hkv, Hq, D = 4, w["n_kv_heads"], w["n_q_heads"], w["head_dim"]
+    outs, qs = [], []
+    for it in range(4):
+        n = 16 * R  # sixteen window blocks per append: a pack launch of several microseconds
+        newk = [torch.randn(B, Hkv, n, D, generator=gen).to(torch.bfloat16).to(DEV) for _ in range(2)]
+        newv = [torch.randn(B, Hkv, n, D, generator=gen).to(torch.bfloat16).to(DEV) for _ in range(2)]
+        q = torch.randn(B, Hq, D, generator=gen).to(torch.bfloat16).to(DEV)
+        # warm decodes so that neither layer is flagged as repacked when the appends start
+        cache.decode_attention(0, q, f32=True); cache.decode_attention(1, q, f32=True)
+        cache.append_kv(1, newk[1], newv[1])   # the borrowing layer's own parameters
+        cache.append_kv(0, newk[0], newv[0])   # the pack of the codes layer 1 reads ...
+        first = cache.decode_attention(1, q, f32=True).clone()  # ... and at once the decode that reads them
+        again = cache.decode_attention(1, q, f32=True)  # the next one may fetch early: the pack is long complete
+        outs.append(first)
+        assert torch.equal(first, again)
+        qs.append(q)
+        for l in (0, 1):
+            kv[l] = (torch.cat([kv[l][0], newk[l]], dim=2), torch.cat([kv[l][1], newv[l]], dim=2))
+        if it < 3:
+            continue
+        torch.cuda.synchronize()
+    # the last state against the oracle, and each earlier result against a replay at its own length
+    G = Hq // Hkv
+    for it in range(4):
+        S_it = 8192 + 100 + (it + 1) * 16 * R
+        part = {l: (kv[l][0][:, :, :S_it], kv[l][1][:, :, :S_it]) for l in (0, 1)}
+        for (b, hk) in ((0, 0), (3, Hkv - 1)):
+            oc = util.oracle_for_stream(cfg, [0, 1], b, hk, part)
+            ref = oc.decode(1, util.bits_of(qs[it][b:b + 1, hk * G:(hk + 1) * G]))[0]
+            got = outs[it][b, hk * G:(hk + 1) * G].double().cpu().numpy()
+            assert np.abs(got - ref).max() <= util.ATTN_TOL, (it, b, hk)
+    cache.close()
+
+
+def test_decode_step_from_host_buffers_at_full_size():
+    """xq_decode_step with pinned host buffers (the end-to-end path the benchmark times) on the 32k GQA shape with
+    one layer pair: three steps, sampled streams against the oracle."""
+    w = dict(W.CONFIGS["c2"], n_layers=2)
+    w["kq"], w["vq"] = 2, 0
+    S, B, Hkv, Hq, D = w["seq"], w["batch"], w["n_kv_heads"], w["n_q_heads"], w["head_dim"]
+    cfg = W.make_xq_config(w, max_seq=S + 8)
+    cache = xq.Cache(cfg, DEV)
+    streams = [(0, 0), (B - 1, Hkv - 1)]
+    parts = {s: [[], [], [], []] for s in streams}
+    for c0 in range(0, S, W.CHUNK):
+        k0, v0, k1, v1 = W.pair_tokens(w, 0, c0, min(S, c0 + W.CHUNK), DEV)
+        cache.append_kv(0, k0, v0)
+        cache.append_kv(1, k1, v1)
+        for (b, h) in streams:
+            for lst, t in zip(parts[(b, h)], (k0, v0, k1, v1)):
+                lst.append(t[b:b + 1, h:h + 1].cpu())
+    gen = torch.Generator(device="cpu").manual_seed(2)
+    G = Hq // Hkv
+    for step in range(3):  # the first step quantizes the full windows
+        kn = torch.randn(2, B, Hkv, 1, D, generator=gen).to(torch.bfloat16).pin_memory()
+        vn = torch.randn(2, B, Hkv, 1, D, generator=gen).to(torch.bfloat16).pin_memory()
+        q = torch.randn(2, B, Hq, D, generator=gen).to(torch.bfloat16).pin_memory()
+        out = torch.empty(2, B, Hq, D, dtype=torch.bfloat16).pin_memory()
+        cache.decode_step(kn, vn, q, out, mem=xq.XQ_MEM_HOST)
+        torch.cuda.synchronize()
+        for (b, h) in streams:
+            for i, t in enumerate((kn[0], vn[0], kn[1], vn[1])):
+                parts[(b, h)][i].append(t[b:b + 1, h:h + 1])
+            k0, v0, k1, v1 = (torch.cat(x, dim=2) for x in parts[(b, h)])
+            oc = util.oracle_for_stream(cfg, [0, 1], 0, 0, {0: (k0, v0), 1: (k1, v1)})
+            for l in (0, 1):
+                ref = oc.decode(l, util.bits_of(q[l, b:b + 1, h * G:(h + 1) * G]))[0]
+                got = out[l, b, h * G:(h + 1) * G].double().numpy()
+                assert (np.abs(got - ref) <= util.ATTN_TOL + 2.0 ** -8 * np.abs(ref)).all(), (step, b, h, l)
+    cache.close()
+
+
 @pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4"])
 def test_full_size_configs_sampled(name):
     """The benchmark's shapes and launch configuration (library-chosen splits, tensor-core kernel), one layer
@@ -507,6 +620,19 @@ def test_full_size_configs_sampled(name):
     sampled streams' query heads against the oracle."""
     w = dict(W.CONFIGS[name], n_layers=2)
     w["kq"], w["vq"] = min(w["kq"], 2), min(w["vq"], 2)
+    _full_size_pair(name, w, pair=0)
+
+
+@pytest.mark.parametrize("name,kq,pair", [("c2", 0, 0), ("c2", 2, 1), ("c1", 0, 1)])
+def test_full_size_other_layers(name, kq, pair):
+    """The same at full size for a layer pair with 1-bit keys (layers at or above kq) and for the workload's
+    second layer pair (other outlier channels, other data)."""
+    w = dict(W.CONFIGS[name], n_layers=2)
+    w["kq"], w["vq"] = kq, min(w["vq"], 2)
+    _full_size_pair(name, w, pair=pair)
+
+
+def _full_size_pair(name, w, pair):
     cfg = W.make_xq_config(w)  # n_splits as the workload names it (0 = library's choice, c4: 64)
     cache = xq.Cache(cfg, DEV)
     S, B, Hkv = w["seq"], w["batch"], w["n_kv_heads"]
@@ -514,7 +640,7 @@ def test_full_size_configs_sampled(name):
     kv = {0: {}, 1: {}}  # per layer, per stream: the tokens of that stream only (host side)
     parts = {s: [[], [], [], []] for s in streams}
     for c0 in range(0, S, W.CHUNK):
-        k0, v0, k1, v1 = W.pair_tokens(w, 0, c0, min(S, c0 + W.CHUNK), DEV)
+        k0, v0, k1, v1 = W.pair_tokens(w, pair, c0, min(S, c0 + W.CHUNK), DEV)
         cache.append_kv(0, k0, v0)
         cache.append_kv(1, k1, v1)
         for (b, h) in streams:

@@ -106,3 +106,27 @@ def test_half_precision_inputs_are_widened_exactly():
     ck, sk, zk, _, _, _ = a.codes_and_meta(0)
     assert np.array_equal(ck[0, 0], codes) and np.array_equal(sk[0, 0], s) and np.array_equal(zk[0, 0], z)
     assert np.array_equal(a.layers[0]["win_k"][0, 0], x[0, 0, 32:].astype(np.float32))
+
+
+def test_delta_histogram_counts_code_differences():
+    """Section 3.3.1's statistic: elements by |own code - shared code|.  Identical layers differ nowhere; the
+    counts of a pair add up to the quantized elements; they equal a direct count over standalone quantizations."""
+    rng = np.random.default_rng(8)
+    D, S = 64, 100
+    k0, v0 = _tokens(rng, S, D), _tokens(rng, S, D)
+    k1, v1 = _tokens(rng, S, D), _tokens(rng, S, D)
+    oc = _cache(delta_stats=True)
+    oc.append(0, k0, v0); oc.append(1, k1, v1)
+    a0, a1 = _cache(L=1), _cache(L=1)
+    a0.append(0, k0, v0); a1.append(0, k1, v1)
+    nq = oc.n_quantized(1)
+    assert nq == 96 and (oc.delta[0] == 0).all()
+    for kind, idx in ((0, 0), (1, 3)):
+        e0, e1 = a0.codes_and_meta(0)[idx], a1.codes_and_meta(0)[idx]
+        want = [int(np.count_nonzero(np.abs(e0.astype(int) - e1.astype(int)) == d)) for d in range(4)]
+        assert list(oc.delta[1, kind]) == want and sum(want) == nq * D
+    # the shared codes are untouched by the statistic
+    assert np.array_equal(oc.codes_and_meta(1)[0], a0.codes_and_meta(0)[0])
+    same = _cache(delta_stats=True)
+    same.append(0, k0, v0); same.append(1, k0, v0)
+    assert list(same.delta[1, 0]) == [nq * D, 0, 0, 0]

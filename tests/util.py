@@ -19,7 +19,7 @@ def oracle_for_stream(cfg, layers, b, hk, kv_by_layer):
                        cfg.kq, cfg.vq, cfg.km, cfg.vm, np.float32(cfg.eta1), np.float32(cfg.eta2),
                        cfg.sm_scale if cfg.sm_scale > 0 else None,
                        share_group=cfg.share_group or 2, share_dominant=cfg.share_dominant,
-                       gamma1=float(np.float32(cfg.gamma1)), f16=cfg.io_dtype == 1)
+                       gamma1=float(np.float32(cfg.gamma1)), f16=cfg.io_dtype == 1, delta_stats=bool(cfg.delta_stats))
     for l in layers:
         K, V = kv_by_layer[l]
         oc.append(l, bits_of(K[b:b + 1, hk:hk + 1]), bits_of(V[b:b + 1, hk:hk + 1]))
