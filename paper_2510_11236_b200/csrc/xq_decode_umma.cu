@@ -27,18 +27,30 @@
 //            S[token][(group, head, byte)]: a token reads the columns of its own group (its warp's);
 //   values:  A_V[128 channels x 128 tokens],  B_V[token x (channel group, head, byte)]
 //            O[channel][(channel group, head, byte)] accumulates over all batches in tensor memory.
-// Warps: 0..3 compute (thread = tensor-memory lane), 4 issues the MMAs (one
-// elected lane, everything else of the issue loop warp-uniform), 5 feeds the
-// stage ring with bulk copies (cp.async.bulk + mbarrier transaction counts),
-// 6 folds the CTA's share of the 16-bit window (bf16 mma.sync over 16-token
-// tiles) beside the main loop.  The loop is software-pipelined: while the tensor
-// core multiplies the keys of batch i+1, the compute warps run the softmax of
-// batch i and expand its values.  Softmax keeps one integer reference per head
-// for the whole CTA, raised only when a logit exceeds it by more than TAU; the
-// value scales are normalised by a power of two per channel group, raised the
-// same way; raising either rescales O in tensor memory (rare).  Split-K partials
-// are merged by the last CTA of a stream (atomic ticket; nobody waits for
+// Warps: the compute warps (thread = tensor-memory lane; four, or two teams of four that split the heads and
+// the columns of every expansion -- measured slower, kept as a template parameter), one warp that folds the
+// CTA's share of the 16-bit window (bf16 or f16 mma.sync over 16-token tiles), one that turns the staged key
+// zero-points into the logit biases sigma * sum_d q_d z_d (one row of mma.sync products per batch), and one that
+// issues the bulk copies of the stage ring (cp.async.bulk + mbarrier transaction counts) and, from one elected
+// lane, the matrix products.  The loop is software-pipelined: while the tensor core multiplies the keys of batch
+// i + 1, the compute warps run the softmax of batch i and expand its values.  Softmax keeps one integer reference
+// per head for the whole team, raised only when a logit exceeds it by more than TAU; the value scales are
+// normalised by a power of two per channel group, raised the same way; raising either rescales O in tensor
+// memory (rare).  Split-K partials are merged by the last CTA of a stream (atomic ticket; nobody waits for
 // another CTA).
+//
+// What bounds it (32k context, four heads per kv head): tensor memory holds two CTAs per SM (64 + 3 * 64 columns
+// each), and a batch takes a CTA about 2000 cycles whether or not it shares its SM, spread evenly over its phases
+// (wait for the stage ~150, expand keys ~190, B_K ~270, publish ~120, read S ~130, logits and the team's vote
+// ~250, exponentials and sums ~280, B_V and expand values ~280, publish ~130, loop and wait for S ~230).  Each
+// phase is the latency of its own instruction chain and of a hand-over (tcgen05.wait, proxy fence, mbarrier,
+// named barrier) between warps that run out of step, not issue bandwidth (issue slots 45 % busy, tensor pipe
+// 17 %, DRAM 24 %).  Variants built and measured on that shape, per launch, back to back: this one 40 us; two
+// teams of four compute warps 50 us; separate expansion and softmax warps with their own hand-overs 50 us; the
+// last arriving compute warp issuing the products itself 63 us (a tcgen05.mma costs its issuing thread ~60
+// cycles); every load of an iteration issued at its top with the team's vote cast early and read late 46 us;
+// four CTAs per SM for a single head per kv head (72 registers) 45 us against 36 us with two; polling warps
+// that sleep between polls: no change.
 //
 // Every wait on an mbarrier is bounded: a thread that gives up sets the status
 // word in global memory and a flag in shared memory that makes every other wait
@@ -1237,6 +1249,8 @@ cudaError_t launch_gp(const DecodeParams& p, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Pl::TOTAL);
+    // the largest shared-memory carve-out: several CTAs of this size are to share an SM
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -1252,11 +1266,23 @@ int ctas_per_sm_gp() {
     cudaGetLastError();
     return 0;
   }
-  int n = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, Va::THREADS, Pl::TOTAL) != cudaSuccess) {
+  // Residency from the kernel's own figures (the occupancy calculator answers 1 for this kernel although two
+  // CTAs do share an SM): registers, shared memory with the 1 KB the system keeps per CTA, threads.
+  cudaFuncAttributes fa;
+  int dev = 0, regs_sm = 0, smem_sm = 0, thr_sm = 0;
+  if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess || cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&regs_sm, cudaDevAttrMaxRegistersPerMultiprocessor, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&thr_sm, cudaDevAttrMaxThreadsPerMultiProcessor, dev) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
+  const int warps = Va::THREADS / 32;
+  const int regs_cta = warps * ((fa.numRegs * 32 + 511) / 512 * 512);  // allocated per warp in units of 512
+  const int smem_cta = (int)Pl::TOTAL + (int)fa.sharedSizeBytes + 1024;
+  int n = regs_sm / regs_cta;
+  if (smem_sm / smem_cta < n) n = smem_sm / smem_cta;
+  if (thr_sm / Va::THREADS < n) n = thr_sm / Va::THREADS;
   const int by_tmem = 512 / (int)Pl::TM_COLS;  // a CTA beyond this would wait for tensor memory
   return n < by_tmem ? n : by_tmem;
 }
