@@ -31,12 +31,13 @@ if ROOT not in sys.path:
 
 METRIC = "decode-attention GB/s at 32k ctx"
 APPEND_BLOCKS = 6  # window blocks quantized per layer in the append pass, one block per call
-BULK_BLOCKS = 16   # then two calls per layer of this many blocks each (a prefill-sized append)
+BULK_BYTES = 256e6  # then two calls per layer of about this much 16-bit input each (a prefill-sized append):
+BULK_MIN, BULK_MAX = 16, 64  # between 16 and 64 window blocks per call
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the decode kernel (ncu, same launch shape as the
 # timed one; see profiles/), with the SHA-256 of the kernel's sources at the time the counters were taken: the
 # figure is reported only while the sources still hash to that.
-NCU_TRAFFIC = {"c2": {"bytes": 84.07e6 + 2.63e6,
-                      "sources_sha256": "unset"}}
+NCU_TRAFFIC = {"c2": {"bytes": 84.04e6 + 2.56e6,
+                      "sources_sha256": "15d7cb099cbabe3ca3f23dc17e890996747600d97841974245b17acb3bec4161"}}
 KERNEL_SOURCES = ("xq_decode_umma.cu", "xq_layout.cuh", "xq_internal.h")
 
 
@@ -277,6 +278,7 @@ def main():
     L, B, Hq, Hkv, D, S = w["n_layers"], w["batch"], w["n_q_heads"], w["n_kv_heads"], w["head_dim"], w["seq"]
     K, Wm = args.steps, args.warmup
     R = w["residual_len"]
+    BULK_BLOCKS = int(max(BULK_MIN, min(BULK_MAX, BULK_BYTES // (2 * B * Hkv * R * D * 2))))
     n_total = Wm + 3 * K + 8 + (APPEND_BLOCKS + 1 + 2 * BULK_BLOCKS) * R  # warm-up, three timed passes, then the append pass
     cfg = W.make_xq_config(w, max_seq=S + n_total + 1, eta1=args.eta1, eta2=args.eta2, kernel=args.kernel,
                            n_splits=args.splits)

@@ -1236,7 +1236,9 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
 template <int BK, int BV, int GS, int GP>
 struct Variant {
   static constexpr bool SP = GP <= 4;
-  static constexpr int NT = 1;
+  // two teams of four compute warps where one CTA has the SM to itself (groups of 5..8 heads); with two CTAs per SM
+  // two teams were measured slower on every shape (50 us against 40 us per launch at 32k, four heads)
+  static constexpr int NT = GP == 8 ? 2 : 1;
   static constexpr int THREADS = (4 * NT + 3) * 32;
   static auto kernel() { return decode_umma_kernel<BK, BV, GS, GP, SP, NT>; }
 };

@@ -46,9 +46,14 @@ def test_static_scratch_matches_workspace_scratch_twice_in_a_row(kernel):
             q = W.queries(w, layer, call, DEV)
             want = cache.decode_attention(layer, q)
             got = torch.full_like(want, float("nan"))
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             rc = xq.xq_decode_attention_static(cache.handle, layer, q, got, stream)
             assert rc == xq.XQ_OK, xq.xq_strerror(rc)
             torch.cuda.synchronize()
+            # the handle was created before this call, so the array is already on the device: the call itself
+            # must leave the device's free memory as it found it
+            assert torch.cuda.mem_get_info()[0] == free_before
             assert torch.isfinite(got.float()).all()
             diff = (got.float() - want.float()).abs().max().item()
             assert diff <= TOL, f"call {call}, layer {layer}, n_splits {n_splits}: max abs difference {diff}"
