@@ -397,6 +397,26 @@ def main():
     e2e_val = sharding.aggregate_rate(step_bytes(seq_before3 + 1, K), ms3_max, world) / 1e9
 
     clocks = sampler.stop(t_lo, t_hi) if sampler else None
+
+    # ---- chunk attention: the last CHUNK_T tokens of a layer as queries, causal inside the chunk (a prefill
+    # ---- chunk / Appendix D's prompt workload), on the first layers of the model
+    CHUNK_T, chunk_layers = 16, min(L, 4)
+    qc = torch.randn(CHUNK_T, B, Hq, D, generator=g, device=dev).to(torch.bfloat16)
+    oc = torch.empty_like(qc)
+    for l in range(chunk_layers):
+        cache.attention_chunk(l, qc, oc)
+    barrier()
+    e0.record()
+    for l in range(chunk_layers):
+        cache.attention_chunk(l, qc, oc)
+    e1.record()
+    barrier()
+    ms_chunk = sharding.max_over_ranks(e0.elapsed_time(e1), dev)
+    S_now = cache.seq_len(0)
+    chunk = {"n_q_tokens": CHUNK_T, "layers": chunk_layers, "context": S_now,
+             "us_per_query_token_and_layer": ms_chunk * 1e3 / (CHUNK_T * chunk_layers),
+             "attended_tokens_per_s": world * B * CHUNK_T * chunk_layers * (S_now - (CHUNK_T - 1) / 2.0) / (ms_chunk * 1e-3),
+             "how": "one decode launch per query token with its visibility limit"}
     rc, nsq, nsw = xq.xq_split_plan(cache.handle, 0)  # the decode launches' split plan (before the appends below)
 
     # ---- pass 4: the quantize-and-pack path: every layer receives whole window blocks (R tokens per call), so each
@@ -468,6 +488,7 @@ def main():
                          "isolated": {"avg_launch_us": dec["avg_us"], "achieved": isolated, "frac": isolated / peak,
                                       "launches": dec["launches"],
                                       "timing": "CUDA events around every launch (no overlap of a launch's prologue with its predecessor's tail)"}},
+            "chunk": chunk,
             "kernels": kinds,
             "flush_step": {"what": "the step on which every layer's window block fills: one quantize-and-pack launch for "
                                    "all layers before that step's decode launches",

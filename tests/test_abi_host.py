@@ -131,3 +131,31 @@ def test_equiv_bits_of_group_table(group, vm):
     for k in range(group):
         c = _cfg(kq=32, vq=32, km=32, vm=vm, share_group=group, share_dominant=k)
         assert xq.xq_equiv_bits(c) == 1.625 == O.equiv_bits(32, 32, 32, vm, 32, group, k)
+
+
+def test_decode_step_refuses_before_it_touches_anything():
+    """xq_decode_step checks pointers, layer order, capacity and kernel choice for every layer before its first
+    copy or launch: a refused call leaves every layer's length as it was (no device is needed to see that)."""
+    import ctypes as C
+    c = _cfg(n_layers=4, max_seq=8)
+    rc, h = xq.xq_create(c, 256, 1 << 40)
+    assert rc == 0
+    launches = xq.xq_launch_count(h)
+    a = 1 << 20  # an aligned, never dereferenced address
+    assert xq.xq_decode_step(h, a + 2, a, a, a) == xq.XQ_ERR_ARG      # misaligned K_new
+    assert xq.xq_decode_step(h, a, a + 8, a, a) == xq.XQ_ERR_ARG      # misaligned V_new
+    assert xq.xq_decode_step(h, a, a, a + 4, a) == xq.XQ_ERR_ARG      # misaligned q
+    assert xq.xq_decode_step(h, a, a, a, a + 6) == xq.XQ_ERR_ARG      # misaligned out
+    assert xq.xq_decode_step(h, a, a, a, a, [0, 1, 1, 2]) == xq.XQ_ERR_ARG    # a layer twice
+    assert xq.xq_decode_step(h, a, a, a, a, [1, 0, 2, 3]) == xq.XQ_ERR_ORDER  # layer 1 reads layer 0's codes
+    assert xq.xq_decode_step(h, a, a, a, a, None, 7) == xq.XQ_ERR_ARG         # unknown memory kind
+    assert [xq.xq_seq_len(h, l) for l in range(4)] == [0, 0, 0, 0]
+    assert xq.xq_launch_count(h) == launches
+    assert xq.xq_destroy(h) == 0
+    # a tensor-core-only configuration on a shape that kernel does not take is refused for every layer up front
+    c = _cfg(n_layers=2, head_dim=64, kernel=xq.XQ_KERNEL_MMA)
+    rc, h = xq.xq_create(c, 256, 1 << 40)
+    assert rc == 0
+    assert xq.xq_decode_step(h, a, a, a, a) == xq.XQ_ERR_CONFIG
+    assert xq.xq_seq_len(h, 0) == 0 and xq.xq_reset(h) == 0
+    assert xq.xq_destroy(h) == 0
