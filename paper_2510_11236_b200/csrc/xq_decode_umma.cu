@@ -49,8 +49,9 @@
 // teams of four compute warps 50 us; separate expansion and softmax warps with their own hand-overs 50 us; the
 // last arriving compute warp issuing the products itself 63 us (a tcgen05.mma costs its issuing thread ~60
 // cycles); every load of an iteration issued at its top with the team's vote cast early and read late 46 us;
-// four CTAs per SM for a single head per kv head (72 registers) 45 us against 36 us with two; polling warps
-// that sleep between polls: no change.
+// four (72 registers) or three (80) CTAs per SM for a single head per kv head 45 us and 44 us against 36 us with
+// two; one S buffer read before the keys are handed over, with two buffers for A_V and B_V instead, 42.5 us;
+// polling warps that sleep between polls: no change.
 //
 // Every wait on an mbarrier is bounded: a thread that gives up sets the status
 // word in global memory and a flag in shared memory that makes every other wait
