@@ -11,11 +11,15 @@
  * and, for each adjacent layer pair (2p, 2p+1) at or above the sharing start,
  * stores the integer codes once, in layer 2p, while both layers keep their own
  * scale and zero-point (Section 3.3.3 / 3.3.4 with group size G = 2 and dominant
- * layer k = 0; Algorithms 1 and 2).
+ * layer k = 0; Algorithms 1 and 2).  The configuration also takes the paper's
+ * other sharing patterns: groups of three and four layers, another dominant
+ * layer, and a pair's codes merged by a weighted average (Tables group, gamma).
  *
  * Two operations form the hot path: xq_append_kv (window append, and
  * quantize-and-pack of every window block that fills) and xq_decode_attention
- * (one query per head against the packed cache plus the window).
+ * (one query per head against the packed cache plus the window);
+ * xq_decode_step runs both for every layer of a model, xq_attention_chunk
+ * takes several query tokens.
  *
  * Conventions that hold for every entry point:
  *   - "device" pointers are CUDA device addresses valid on the device that was
@@ -34,7 +38,9 @@
  *   - Every function returns XQ_OK (0) or a negative XQ_ERR_* code; a failing
  *     call leaves the cache unchanged.  Nothing is thrown across the boundary.
  *   - A cache handle is not thread-safe; use one host thread per handle.
- *   - 16-bit inputs and outputs are bfloat16 (io_dtype XQ_BF16).
+ *   - 16-bit inputs, outputs and the residual window have the type io_dtype
+ *     names: bfloat16 (XQ_BF16, where a comment below says "bfloat16" read
+ *     "io_dtype") or IEEE half precision (XQ_F16).
  */
 #ifndef XQ_H_
 #define XQ_H_
@@ -151,9 +157,13 @@ int xq_reset(xq_cache* c);
  * until the stream has run the call.  Tokens enter the window; when the window
  * already holds R tokens and a further token arrives, that block of R tokens is
  * quantized (Eq. 1, 2, 12): scale and zero-point always, integer codes only if
- * the layer owns codes (Quantize), not if it borrows them (PseudoQuantize).
- * After S tokens the window holds ((S-1) mod R)+1 tokens.
- * Errors: XQ_ERR_ARG, XQ_ERR_CAPACITY (S would exceed max_seq), XQ_ERR_CUDA. */
+ * the layer owns codes (Quantize), not if it borrows them (PseudoQuantize); with
+ * gamma1 > 0 the second layer of a pair quantizes too and merges its codes into
+ * the pair's (Appendix F), which needs the first layer's blocks in place.
+ * After S tokens the window holds ((S-1) mod R)+1 tokens.  One kernel launch:
+ * the quantize-and-pack launch also refills the window.
+ * Errors: XQ_ERR_ARG, XQ_ERR_CAPACITY (S would exceed max_seq), XQ_ERR_ORDER (a
+ * merging or difference-counting layer ahead of its dominant layer), XQ_ERR_CUDA. */
 int xq_append_kv(xq_cache* c, int layer, const void* K, const void* V, int n_tokens, void* stream);
 
 /* One decode query per head against everything cached in `layer` (Algorithm 1,
@@ -228,8 +238,13 @@ int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out,
  * The result equals xq_append_kv followed by xq_decode_attention per layer, bit
  * for bit; where the tensor-core kernel serves the layer and the token fills no
  * window block, that kernel stores the token into the window itself (one launch
- * per layer).  K_new and V_new must stay unchanged until the step's kernels
- * have run. */
+ * per layer); on the step on which every layer's window block fills (all layers
+ * of equal length, no merging or difference counting), one quantize-and-pack
+ * launch serves all layers before the decode launches.  K_new and V_new must
+ * stay unchanged until the step's kernels have run.
+ * Every layer's capacity, order and kernel are checked before the first copy or
+ * launch: a call refused with XQ_ERR_ARG / CAPACITY / ORDER / CONFIG changes
+ * nothing.  After XQ_ERR_CUDA the cache's state is undefined. */
 int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void* q, void* out,
                    const int32_t* layer_order, int mem, void* stream);
 

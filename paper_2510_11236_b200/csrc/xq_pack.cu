@@ -143,7 +143,7 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
   const int kind = blockIdx.x & 1;  // 0 keys, 1 values
   const int tile_idx = blockIdx.x >> 1;
   const int h = blockIdx.y, b = blockIdx.z % dm.B;
-  const PackLayer& pl = p.layer[blockIdx.z / dm.B];
+  const PackLayer pl = p.layer[blockIdx.z / dm.B];  // by value: its fields are read in every loop below
   const int bh = b * dm.Hkv + h;
   const int tid = threadIdx.x;
   const int tq0 = p.nq_old + tile_idx * T;  // absolute index of the tile's first token
