@@ -494,7 +494,7 @@ def main():
                                    "all layers before that step's decode launches",
                            "pack_launches": kinds["quantize_pack"]["launches"],
                            "pack_avg_us": kinds["quantize_pack"]["avg_us"],
-                           "step_ms_without_it": ms_max / K},
+                           "avg_step_ms_of_the_timed_region": ms_max / K},
             "append": append,
         }
         if not args.no_cpu_baseline and world == 1:
