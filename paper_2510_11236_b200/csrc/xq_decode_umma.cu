@@ -51,7 +51,8 @@
 // cycles); every load of an iteration issued at its top with the team's vote cast early and read late 46 us;
 // four (72 registers) or three (80) CTAs per SM for a single head per kv head 45 us and 44 us against 36 us with
 // two; one S buffer read before the keys are handed over, with two buffers for A_V and B_V instead, 42.5 us;
-// polling warps that sleep between polls: no change.
+// polling warps that sleep between polls: no change; B_K and the logit scales of all four groups written a
+// batch ahead by the warp that computes the biases (two B_K buffers), the compute warps only expanding: 42 us.
 //
 // Every wait on an mbarrier is bounded: a thread that gives up sets the status
 // word in global memory and a flag in shared memory that makes every other wait
@@ -853,7 +854,7 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
         const int k = i - 1;
         const bool ok = mbar_wait(bar_vready, k & 1, &dead_sm);
         tc_fence_after();
-        if (ok && lane == 0) {
+        if (ok && elect_one()) {
           const uint32_t dO = tbase + Pl::COL_O, aV = tbase + Pl::COL_AV;
           if (k == 0) umma_i8<false>(dO, aV, dV, IDESC);
           else umma_i8<true>(dO, aV, dV, IDESC);
@@ -1068,22 +1069,23 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
 
     // ---- prologue: keys of the first batch ----
     float ck[HT], ck_n[HT];
-    mbar_wait(bar_full, 0, &dead_sm);
+    mbar_wait(bar_bias, 0, &dead_sm);  // the biases of a batch are written once its stage has landed
     prep_keys(sm_base, ck);
     publish(bar_kready);
 #pragma unroll
     for (int h = 0; h < HT; ++h) ck_n[h] = ck[h];
+    mbar_wait(bar_sready, 0, &dead_sm);  // S of the first batch
+    tc_fence_after();
 
     // ---- main loop: keys of batch i + 1 go to the tensor core, then softmax and values of batch i ----
 #pragma unroll 1
     for (int i = 0; i < nb; ++i) {
       const int s = i % NSTG;
       const uint32_t st = sm_base + s * St::BYTES;
-      mbar_wait(bar_sready + 8 * (i & 1), (i >> 1) & 1, &dead_sm);  // S of batch i is complete; A_K and B_K are free
-      tc_fence_after();
+      // S of batch i is complete and A_K and B_K are free (waited for in the iteration before)
       if (i + 1 < nb) {
         const int sn = (i + 1) % NSTG;
-        mbar_wait(bar_full + 8 * sn, ((i + 1) / NSTG) & 1, &dead_sm);
+        mbar_wait(bar_bias + 8 * sn, ((i + 1) / NSTG) & 1, &dead_sm);  // stage and biases of batch i + 1
         prep_keys(sm_base + sn * St::BYTES, ck_n);
         publish(bar_kready);
       }
@@ -1108,7 +1110,6 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
         sv[0] = a.x; sv[1] = a.y;
         zv[0] = e.x; zv[1] = e.y;
       }
-      mbar_wait(bar_bias + 8 * s, (i / NSTG) & 1, &dead_sm);
       float bias[HT];
       {
         const float* slot = reinterpret_cast<const float*>(smem + Pl::OFF_META + s * Pl::META_SLOT) + gam * GP + h0;
@@ -1142,7 +1143,11 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
 #pragma unroll
         for (int gi = 0; gi < NGB; ++gi) zacc[gi][h] = fmaf(pe[h], zv[gi], zacc[gi][h]);
       }
-      if (i > 0) mbar_wait(bar_odone, (i - 1) & 1, &dead_sm);  // the value products of batch i - 1 are done with A_V and B_V
+      // The value products of batch i - 1 must be done with A_V and B_V.  They were issued before the key products
+      // of batch i + 1, and a commit covers everything its thread issued before it: S of batch i + 1 being complete
+      // says both, in one wait.
+      if (i + 1 < nb) mbar_wait(bar_sready + 8 * ((i + 1) & 1), ((i + 1) >> 1) & 1, &dead_sm);
+      else if (i > 0) mbar_wait(bar_odone, (i - 1) & 1, &dead_sm);
       tc_fence_after();
       {
         const uint32_t bv = sm_base + Pl::OFF_BV + (ctid >> 3) * LBO + (ctid & 7) * 16;
