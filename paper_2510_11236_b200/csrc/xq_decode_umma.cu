@@ -740,9 +740,10 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = dm.G;
 
-  // The next kernel in the stream may be scheduled at once when this one is sure to fetch nothing that kernel's
-  // predecessors could still be writing; otherwise only after this kernel's own wait (below).
-  if (p.early_fetch) grid_dependents_go();
+  // The next kernel in the stream may be scheduled at once when all work before this kernel's own predecessor is
+  // known to be complete (a chained launch); otherwise only after this kernel's own wait (below), so that a chained
+  // successor never starts before the work this kernel waited for has completed.
+  if (p.late_wait) grid_dependents_go();
 
   // CTA -> (stream, split): p.n_ctas CTAs dealt to the streams in order; the first n_ctas % streams streams get one
   // split more than the others
@@ -869,7 +870,7 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
     }
   } else if (warp == W_WIN) {
     // ================= window warp: this CTA's share of the 16-bit window =================
-    grid_dependency_wait();
+    if (!p.late_wait) grid_dependency_wait();
     int wt0, wt1;
     share_of(p.r, ns, split, wt0, wt1);
     if (wt0 < wt1) {
@@ -883,7 +884,7 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
     }
   } else if (warp == W_BIAS) {
     // ================= bias warp: sigma * sum_d q_d z_d per (token group, head) of a batch =================
-    grid_dependency_wait();  // q comes from the preceding kernel
+    if (!p.late_wait) grid_dependency_wait();  // q may come from the preceding kernel
     // One row of legacy tensor-core products per batch: rows = the batch's token groups (zero-points read as they
     // are staged, fp16), columns = heads (q as fp16: exact for bf16 inputs of ordinary magnitude), fp32 accumulate.
     const int gid = lane >> 2, tig = lane & 3;
@@ -927,8 +928,10 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
     const int team = NT == 1 ? 0 : warp >> 2, qw = warp & 3;  // qw: lane quarter
     const int ctid = qw * 32 + lane;                          // row: token of the batch / channel
     const int h0 = team * HT;                                 // first head of the team
-    grid_dependency_wait();  // q comes from the preceding kernel
-    if (!p.early_fetch) grid_dependents_go();
+    if (!p.late_wait) {
+      grid_dependency_wait();  // q may come from the preceding kernel
+      grid_dependents_go();    // whatever this kernel waited for is complete for its successor too
+    }
     const int gam = qw / WPG;  // this warp's rows: key token group of the batch / channel group of O
     const uint32_t row_t = tbase + ((uint32_t)(qw * 32) << 16);
     const float scale2 = p.scale * 1.4426950408889634f;
@@ -1210,6 +1213,7 @@ __global__ void __launch_bounds__((4 * NT + 3) * 32, GP <= 4 ? 2 : 1) decode_umm
   // ---- all warps: combine the main state with the window state, write the partial, merge ----
   tc_fence_before();
   __syncthreads();
+  if (p.late_wait) grid_dependency_wait();  // the preceding launch still reads and writes the scratch and its result
   const bool dead = dead_sm != 0;
   if (warp < 4 && !dead) {
     const int stride = p.ns_q;

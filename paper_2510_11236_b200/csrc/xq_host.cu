@@ -344,6 +344,7 @@ int prepare_decode(const xq_cache* c, int layer, const void* q, void* out, int o
   p.out = out;
   p.out_f32 = out_f32;
   p.early_fetch = 0;
+  p.late_wait = 0;
   p.f16 = c->cfg.io_dtype == XQ_F16;
   p.K_new = (const uint16_t*)K_new;
   p.V_new = (const uint16_t*)V_new;
@@ -477,8 +478,13 @@ int pack_layers(xq_cache* c, const int* layers, int n, const void* K, const void
   return XQ_OK;
 }
 
+// chained: the launch before this one in the stream is a tensor-core decode launch of the same call, so nothing this
+// launch reads (q, the new token, the window, the packed streams) can still be written when its CTAs start; it
+// waits for that launch only before it writes.  *was_mma tells the caller whether this launch can head such a chain.
 int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, cudaStream_t st,
-                const void* K_new = nullptr, const void* V_new = nullptr, int vis = -1) {
+                const void* K_new = nullptr, const void* V_new = nullptr, int vis = -1, bool chained = false,
+                bool* was_mma = nullptr) {
+  if (was_mma) *was_mma = false;
   if (!c) return XQ_ERR_ARG;
   if (layer < 0 || layer >= c->cfg.n_layers) return XQ_ERR_ARG;
   DecodeParams p;
@@ -491,6 +497,7 @@ int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, c
     // the packed streams may be fetched ahead of the preceding kernel unless a pack kernel wrote them since
     // this layer's last decode (then that kernel may be the writer, or only just behind it)
     p.early_fetch = c->repacked[layer] ? 0 : 1;
+    if (chained) p.early_fetch = p.late_wait = 1;
   }
   rc = launch_decode(c, p, use_mma, workspace_scratch(c), st);
   if (rc != XQ_OK) {
@@ -499,6 +506,7 @@ int decode_impl(xq_cache* c, int layer, const void* q, void* out, int out_f32, c
   }
   if (use_mma) c->repacked[layer] = 0;
   if (K_new) c->seq[layer] += 1;
+  if (was_mma) *was_mma = use_mma;
   return XQ_OK;
 }
 
@@ -751,10 +759,11 @@ int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void
       appended = true;
     }
   }
+  bool chain = false;  // the launch before the next one is a tensor-core decode launch of this call
   for (int i = 0; i < L; ++i) {
     const int l = layer_order ? layer_order[i] : i;
     if (appended) {
-      const int rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st);
+      const int rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st, nullptr, nullptr, -1, chain, &chain);
       if (rc != XQ_OK) return rc;
       continue;
     }
@@ -764,11 +773,12 @@ int xq_decode_step(xq_cache* c, const void* K_new, const void* V_new, const void
     const int nq_old = s_old - residual_count(s_old, dm.R), nq_new = s_old + 1 - residual_count(s_old + 1, dm.R);
     int rc;
     if (nq_new == nq_old && nq_old > 0 && layer_uses_mma(c, l)) {
-      rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st, dk + l * kv_layer, dv + l * kv_layer);
+      rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st, dk + l * kv_layer, dv + l * kv_layer, -1, chain,
+                       &chain);
     } else {
       rc = xq_append_kv(c, l, dk + l * kv_layer, dv + l * kv_layer, 1, stream);
       if (rc != XQ_OK) return rc;
-      rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st);
+      rc = decode_impl(c, l, dq + l * q_layer, dout + l * q_layer, 0, st, nullptr, nullptr, -1, false, &chain);
     }
     if (rc != XQ_OK) return rc;
   }

@@ -86,6 +86,11 @@ struct DecodeParams {
   // 1: the packed streams were complete before the preceding kernel in the stream started, so their first
   // copies may be issued before this kernel has waited for that kernel (programmatic dependent launch)
   int early_fetch;
+  // 1: the preceding kernel in the stream is a decode launch of the same call that itself started only after all
+  // earlier work in the stream had completed, so nothing this launch reads is still being written: it reads at
+  // once and waits for that launch only before its first write that the launch could see (partials, tickets,
+  // result, status).  Implies early_fetch.
+  int late_wait;
   // Fused append of one token per stream (tensor-core kernel with quantized tokens only; else null): the newest
   // window row, index r - 1, is not in the window yet but here, [B,Hkv,D] bf16.  The CTA whose share of the
   // window holds that row reads it from here and stores it into the window.
