@@ -72,7 +72,7 @@ constexpr int HD = 128;
 constexpr int BT = 128;          // tokens per batch
 constexpr int NSTG = 4;          // staged batches
 constexpr int TAU = 3;           // log2 units a logit may exceed the softmax reference before it is raised
-constexpr int MREF = 2;          // a raised reference sits this far below the (rounded-up) largest logit
+constexpr int MREF = 0;           // a raised reference is the largest logit rounded up: three more units before the next raise
 constexpr int FRAC_V = 23 - TAU; // fraction bits of the value-side fixed point
 constexpr int WAIT_LIMIT = 1 << 20;     // polls of a wait before it gives up
 constexpr uint32_t WAIT_HINT_NS = 10000;  // longest suspension of one poll (it ends at once when the phase completes)
