@@ -643,10 +643,11 @@ int chunk_impl(xq_cache* c, int layer, const void* q, void* out, int n, int out_
     if (rc != XQ_OK) return rc;
   }
   const size_t row = (size_t)dm.B * dm.Hq * dm.D;  // elements of one token's queries: [batch, heads, head_dim]
+  bool chain = false;  // launches after the first read what the first one waited for and write their own rows
   for (int j = 0; j < n; ++j) {
     const uint8_t* qj = (const uint8_t*)q + (size_t)j * row * 2;
     uint8_t* oj = (uint8_t*)out + (size_t)j * row * (out_f32 ? 4 : 2);
-    const int rc = decode_impl(c, layer, qj, oj, out_f32, (cudaStream_t)stream, nullptr, nullptr, S - n + 1 + j);
+    const int rc = decode_impl(c, layer, qj, oj, out_f32, (cudaStream_t)stream, nullptr, nullptr, S - n + 1 + j, chain, &chain);
     if (rc != XQ_OK) return rc;
   }
   return XQ_OK;
