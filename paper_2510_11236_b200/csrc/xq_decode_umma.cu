@@ -40,19 +40,29 @@
 // another CTA).
 //
 // What bounds it (32k context, four heads per kv head): tensor memory holds two CTAs per SM (64 + 3 * 64 columns
-// each), and a batch takes a CTA about 2000 cycles whether or not it shares its SM, spread evenly over its phases
-// (wait for the stage ~150, expand keys ~190, B_K ~270, publish ~120, read S ~130, logits and the team's vote
-// ~250, exponentials and sums ~280, B_V and expand values ~280, publish ~130, loop and wait for S ~230).  Each
-// phase is the latency of its own instruction chain and of a hand-over (tcgen05.wait, proxy fence, mbarrier,
-// named barrier) between warps that run out of step, not issue bandwidth (issue slots 45 % busy, tensor pipe
-// 17 %, DRAM 24 %).  Variants built and measured on that shape, per launch, back to back: this one 40 us; two
-// teams of four compute warps 50 us; separate expansion and softmax warps with their own hand-overs 50 us; the
-// last arriving compute warp issuing the products itself 63 us (a tcgen05.mma costs its issuing thread ~60
-// cycles); every load of an iteration issued at its top with the team's vote cast early and read late 46 us;
-// four (72 registers) or three (80) CTAs per SM for a single head per kv head 45 us and 44 us against 36 us with
-// two; one S buffer read before the keys are handed over, with two buffers for A_V and B_V instead, 42.5 us;
-// polling warps that sleep between polls: no change; B_K and the logit scales of all four groups written a
-// batch ahead by the warp that computes the biases (two B_K buffers), the compute warps only expanding: 42 us.
+// each), and a batch takes a CTA about 1600 cycles whether or not it shares its SM.  That time is the latency of
+// the compute warps' own instruction chain (expand keys ~190 cycles, B_K ~270, read S ~130, logits and the team's
+// vote ~250, exponentials and sums ~70, B_V and expand values ~290) plus 100 to 200 cycles for every hand-over on
+// it (a wait on an mbarrier, tcgen05.wait, proxy fence and arrive); the SM's units are far from busy (issue slots
+// 40 %, tensor pipe 20 %, DRAM 25 %).  So the loop keeps the hand-overs few: the bias barrier of a batch also
+// stands for the arrival of its stage, one wait for S of batch i + 1 also covers the value products of batch i - 1
+// (a commit covers everything its thread issued before), and a wait first tests its barrier without suspending
+// (most are complete by then).  A raise of the references costs ~1200 cycles, so a raised reference leaves three
+// units of room.  A CTA lives ~31 us for ~25 us of loop; consecutive launches of a decode step overlap
+// (late_wait), so the next launch's CTAs take the slots as this one's leave.
+// Variants built and measured on that shape, per launch, back to back (the kept loop: 40 us before the hand-overs
+// were thinned out, 34.4 us now): two teams of four compute warps 50 us; separate expansion and softmax warps with
+// their own hand-overs 50 us; the last arriving compute warp issuing the products itself 63 us (a tcgen05.mma
+// costs its issuing thread ~50 cycles); every load of an iteration issued at its top with the team's vote cast
+// early and read late 46 us; four (72 registers) or three (80) CTAs per SM for a single head per kv head 45 us
+// and 44 us against 36 us with two; one S buffer read before the keys are handed over, with two buffers for A_V
+// and B_V instead, 42.5 us; polling warps that sleep between polls: no change; polling warps that never suspend:
+// 0.7 us slower (they take issue slots from the compute warp of their sub-partition); B_K and the logit scales of
+// all four groups written a batch ahead by the bias warp (two B_K buffers) 42 us, only the groups' exponents and
+// logit scales from the bias warp: 1.3 us slower; the team's votes cast a batch ahead through an mbarrier instead
+// of the hardware barrier (logits of batch i + 1 at the end of iteration i) 42.6 us; a warp of its own for the
+// bulk copies: no change; the first copies, or q, fetched before the tensor-memory allocation: no change; the
+// four bulk copies of a batch issued from four lanes instead of one: 40.5 us.
 //
 // Every wait on an mbarrier is bounded: a thread that gives up sets the status
 // word in global memory and a flag in shared memory that makes every other wait
@@ -156,7 +166,15 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 // Bounded wait; gives up as well when another thread of the CTA has (dead flag in shared memory).
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* dead) {
+  if (mbar_test_wait(bar, parity)) return true;  // the usual case on the loop's path: already complete
   for (int i = 0; i < WAIT_LIMIT; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*dead) return false;
