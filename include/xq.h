@@ -241,7 +241,12 @@ int xq_decode_attention_static(xq_cache* c, int layer, const void* q, void* out,
  * per layer); on the step on which every layer's window block fills (all layers
  * of equal length, no merging or difference counting), one quantize-and-pack
  * launch serves all layers before the decode launches.  K_new and V_new must
- * stay unchanged until the step's kernels have run.
+ * stay unchanged until the step's kernels have run.  The tensor-core decode
+ * launches of a step overlap: the first waits for all earlier work in `stream`
+ * before it reads anything; each later one starts while its predecessor still
+ * runs, reads at once (everything before the first launch is complete by then,
+ * and a decode launch writes only its own window row, scratch and result) and
+ * waits for the predecessor before its own first write to scratch or result.
  * Every layer's capacity, order and kernel are checked before the first copy or
  * launch: a call refused with XQ_ERR_ARG / CAPACITY / ORDER / CONFIG changes
  * nothing.  After XQ_ERR_CUDA the cache's state is undefined. */
