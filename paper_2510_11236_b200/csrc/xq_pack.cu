@@ -26,6 +26,11 @@ struct In16<false> {
   static __device__ __forceinline__ float lo(uint32_t w) { return __uint_as_float(w << 16); }
   static __device__ __forceinline__ float hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
   static __device__ __forceinline__ float one(uint16_t u) { return bf16_bits(u); }
+  // pattern of the nearest 16-bit value (of x itself when it is one)
+  static __device__ __forceinline__ uint32_t bits(float x) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x)); }
+  // the nearest 16-bit value at or above / at or below x
+  static __device__ __forceinline__ uint32_t bits_up(float x) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_ru(x)); }
+  static __device__ __forceinline__ uint32_t bits_down(float x) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rd(x)); }
 };
 template <>
 struct In16<true> {
@@ -33,6 +38,9 @@ struct In16<true> {
   static __device__ __forceinline__ float lo(uint32_t w) { return __half2float(__ushort_as_half((unsigned short)(w & 0xffffu))); }
   static __device__ __forceinline__ float hi(uint32_t w) { return __half2float(__ushort_as_half((unsigned short)(w >> 16))); }
   static __device__ __forceinline__ float one(uint16_t u) { return __half2float(__ushort_as_half(u)); }
+  static __device__ __forceinline__ uint32_t bits(float x) { return (uint32_t)__half_as_ushort(__float2half_rn(x)); }
+  static __device__ __forceinline__ uint32_t bits_up(float x) { return (uint32_t)__half_as_ushort(__float2half_ru(x)); }
+  static __device__ __forceinline__ uint32_t bits_down(float x) { return (uint32_t)__half_as_ushort(__float2half_rd(x)); }
 };
 
 // Merged words of a sharing pair (Appendix F): field by field, the code of (e0, e1) from the table.
@@ -60,21 +68,12 @@ __device__ __forceinline__ void group_params(float mn, float mx, int bits, float
   sh = __float2half_rn(__fmul_rn(k, s));
 }
 
-// Eq. 2 with the uncalibrated z, s; ties to even; clamped; constant group -> 0.
-__device__ __forceinline__ uint32_t code_of(float x, float z, float s, float qmax) {
-  if (s == 0.0f) return 0u;
-  float c = rintf(__fdiv_rn(__fsub_rn(x, z), s));
-  c = fminf(fmaxf(c, 0.0f), qmax);
-  return (uint32_t)c;
-}
-
 constexpr int PACK_THREADS = 128;
 constexpr int PACK_ROW_PAD = 16;  // bytes added to each staged row: 8 consecutive rows then fall in 8 different bank groups
-constexpr float PACK_MAGIC = 12582912.0f;  // 1.5 * 2^23: x + MAGIC has rint(x) in its low mantissa bits for |x| < 2^22
 
-// 1/s for the quotient sequence of code_pair: 0 for a constant group (every code 0), NaN where that sequence is
+// 1/s for the quotient sequence of `quotient`: 0 for a constant group (every code 0), NaN where that sequence is
 // not known to round correctly -- a scale whose significand is all ones, or one so small or large that an
-// intermediate could leave the normal range -- which sends the word to the division.
+// intermediate could leave the normal range -- which sends the group to the division.
 __device__ __forceinline__ float safe_rcp(float s) {
   if (s == 0.0f) return 0.0f;
   const uint32_t b = __float_as_uint(s);
@@ -83,24 +82,95 @@ __device__ __forceinline__ float safe_rcp(float s) {
   return __frcp_rn(s);
 }
 
-// Eq. 2 for two elements without a division.  With y = RN(1/s): q = RN(a y), r = a - q s (exact in one fused
-// multiply-add), q' = RN(q + r y) is the correctly rounded quotient RN(a / s) (the classical correction step of
-// division by a correctly rounded reciprocal; the significands it can miss are excluded by safe_rcp), so
-// rint(q') is the code the division gives, ties included.  Adding 1.5 * 2^23 rounds to the nearest integer, ties
-// to even, and leaves it in the low mantissa bits; 0 <= a / s < 2^B - 1/2 holds for every member of the group, so
-// no clamp is needed.  A NaN reciprocal sets `doubt` and the caller recomputes the word with the division.
-// Returns code(x0) | code(x1) << 8: two neighbouring bytes of a packed word.
-template <int BITS>
-__device__ __forceinline__ uint32_t code_pair(float x0, float x1, const float4& p0, const float4& p1, bool& doubt) {
-  const float a0 = __fsub_rn(x0, p0.x), a1 = __fsub_rn(x1, p1.x);
-  float q0 = __fmul_rn(a0, p0.y), q1 = __fmul_rn(a1, p1.y);
-  const float r0 = __fmaf_rn(-q0, p0.z, a0), r1 = __fmaf_rn(-q1, p1.z, a1);
-  q0 = __fmaf_rn(r0, p0.y, q0);
-  q1 = __fmaf_rn(r1, p1.y, q1);
-  const float u0 = __fadd_rn(q0, PACK_MAGIC), u1 = __fadd_rn(q1, PACK_MAGIC);
-  doubt |= (p0.y != p0.y) | (p1.y != p1.y);
-  constexpr uint32_t QM = (1u << BITS) - 1u;
-  return __byte_perm(__float_as_uint(u0), __float_as_uint(u1), 0x0040) & (QM | (QM << 8));
+// Codes by comparison (Eq. 2).  The code of x in a group, c(x) = clamp(rint(RN(RN(x - z) / s)), 0, 2^B - 1), never
+// decreases with x, and x is a 16-bit float, so the group's codes are fixed by B-bit-many thresholds on the input
+// lattice: X_k = the smallest 16-bit value with c(X_k) >= k, and c(x) = #{k : x >= X_k}.  One thread per group
+// finds the X_k: next to z + (k - 1/2) s, from the rounding bounds of the quotient where they decide, else by
+// evaluating c itself (the quotient exactly as the division gives it, ties of rint to even) at lattice points; the
+// elements are then coded two at a time with packed 16-bit compares.
+
+// 16-bit float pattern <-> integer that orders like the value (sign-magnitude to two's complement; -0 and +0 -> 0)
+__device__ __forceinline__ int ord16(uint32_t h) {
+  const int m = (int)(h & 0x7fffu);
+  return (h & 0x8000u) ? -m : m;
+}
+__device__ __forceinline__ uint32_t pat16(int o) { return o >= 0 ? (uint32_t)o : (0x8000u | (uint32_t)(-o)); }
+
+// A group's uncalibrated parameters for the quotient RN(RN(x - z) / s).  With y = RN(1/s): q = RN(a y),
+// r = a - q s (exact in one fused multiply-add), q' = RN(q + r y) is the correctly rounded quotient (the classical
+// correction step of division by a correctly rounded reciprocal; the scales it can miss get a NaN from safe_rcp
+// and take the division).
+struct Quot {
+  float z, s, y;
+  bool fast;
+};
+__device__ __forceinline__ float quotient(const Quot& g, float x) {
+  const float a = __fsub_rn(x, g.z);
+  if (g.fast) {
+    const float q = __fmul_rn(a, g.y);
+    const float r = __fmaf_rn(-q, g.s, a);
+    return __fmaf_rn(r, g.y, q);
+  }
+  return __fdiv_rn(a, g.s);
+}
+
+// X_k as a 16-bit pattern, given lattice points (as ordered integers) with c(o_lo) < k <= c(o_hi).  In real
+// numbers the threshold is tau = z + (k - 1/2) s.  The computed quotient differs from (x - z) / s by less than
+// 2^-23 relative (two roundings), i.e. by less than 3.1 * 2^-23 s in x, and t = RN(tau) from tau by at most
+// 2^-24 |t|: a lattice point at or above t + eps certainly has c >= k, one at or below t - eps certainly has not,
+// for eps = 2^-22 |t| + 2^-20 s (twice what is needed).  Where the lattice is coarser than eps -- almost always --
+// the two certain neighbours are adjacent and nothing is evaluated; otherwise (a threshold next to zero under a
+// large |z|, an exact tie on the lattice) c itself decides, by bisection between them.  Groups whose scale takes
+// the division (safe_rcp) are bisected from the group's ends.
+template <bool F16>
+__device__ __forceinline__ uint32_t threshold16(const Quot& g, int k, int o_lo, int o_hi) {
+  const float kk = (float)k - 0.5f;
+  const bool even = (k & 1) == 0;  // rint takes a tie to the even neighbour: k - 1/2 counts as >= k only for even k
+  int lo = o_lo, hi = o_hi;
+  if (g.fast) {
+    const float t = __fmaf_rn(kk, g.s, g.z);
+    const float eps = __fmaf_rn(fabsf(t), 0x1p-22f, __fmul_rn(g.s, 0x1p-20f));
+    const int o_up = ord16(In16<F16>::bits_up(__fadd_ru(t, eps)));   // the smallest lattice point >= t + eps
+    const int o_dn = ord16(In16<F16>::bits_down(__fadd_rd(t, -eps)));  // the largest one <= t - eps
+    if (o_dn > lo && o_dn < hi) lo = o_dn;
+    if (o_up < hi && o_up > lo) hi = o_up;
+  }
+  while (hi - lo > 1) {
+    const int mid = lo + ((hi - lo) >> 1);
+    const float q = quotient(g, In16<F16>::one((uint16_t)pat16(mid)));
+    if (even ? q >= kk : q > kk) hi = mid; else lo = mid;
+  }
+  return pat16(hi);
+}
+
+// The thresholds of a group with minimum mn and maximum mx (16-bit values, widened) into thr[k * stride]; unused
+// ones (k beyond 2^B - 1, or a constant group: every code 0) are +infinity.
+template <bool F16>
+__device__ __forceinline__ void group_thresholds(float mn, float mx, float z, float sc, int bits, uint16_t* thr, int stride) {
+  constexpr uint16_t INF16 = F16 ? 0x7c00u : 0x7f80u;
+  const float y = safe_rcp(sc);
+  const Quot g{z, sc, y, y == y};
+  const int o_lo = ord16(In16<F16>::bits(mn)), o_hi = ord16(In16<F16>::bits(mx));
+  const int qmax = (1 << bits) - 1;
+#pragma unroll
+  for (int k = 1; k <= 3; ++k)
+    thr[(k - 1) * stride] = (k <= qmax && sc != 0.0f) ? (uint16_t)threshold16<F16>(g, k, o_lo, o_hi) : INF16;
+}
+
+// Codes of two packed 16-bit elements against their groups' packed thresholds: code of the low element at bit 0,
+// of the high element at bit 16.
+template <int BITS, typename V2>
+__device__ __forceinline__ uint32_t code_pair(uint32_t x, uint32_t t1, uint32_t t2, uint32_t t3) {
+  const V2 xv = *reinterpret_cast<const V2*>(&x);
+  const uint32_t m1 = __hge2_mask(xv, *reinterpret_cast<const V2*>(&t1));
+  if constexpr (BITS == 1) {
+    return m1 & 0x00010001u;
+  } else {
+    const uint32_t m2 = __hge2_mask(xv, *reinterpret_cast<const V2*>(&t2));
+    const uint32_t m3 = __hge2_mask(xv, *reinterpret_cast<const V2*>(&t3));
+    // m3 implies m2 implies m1: code bit 0 = (m1 and not m2) or m3, bit 1 = m2
+    return (((m1 & ~m2) | m3) & 0x00010001u) | (m2 & 0x00020002u);
+  }
 }
 
 // Adds to hist[d] the number of fields of the two words whose codes differ by d.
@@ -133,7 +203,8 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
   constexpr int KP = PACK_THREADS / ((T / G) * (D / 2));               // token parts of a key group in the statistics
   static_assert(KP >= 1 && G % KP == 0, "key statistics: 128 threads over (group, channel pair, token part)");
   __shared__ __align__(16) uint8_t tile[T * ROWB];
-  __shared__ __align__(16) float4 par[NPAR];  // (z, 1/s, s, -) of a group; keys: [group][channel], values: [channel group][token]
+  // thresholds X_1..X_3 of a group: [k][group]; keys: group = [token group][channel], values: [channel group][token]
+  __shared__ __align__(16) uint16_t thr[3 * NPAR];
   // packed words (at most T * D * 2 / 32); before that, the key statistics' partial (min, max) pairs, two words per thread
   constexpr int NWBUF = (T * D * 2 / 32) > 2 * PACK_THREADS ? (T * D * 2 / 32) : 2 * PACK_THREADS;
   __shared__ __align__(16) uint32_t wbuf[NWBUF];
@@ -217,7 +288,7 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
         float z, sc;
         __half zh, sh;
         group_params(mn, mx, bits, eta, z, sc, zh, sh);
-        par[item] = make_float4(z, safe_rcp(sc), sc, 0.f);
+        if (own) group_thresholds<F16>(mn, mx, z, sc, bits, thr + item, NPAR);
         const size_t grp = (size_t)bh * cap_g + (tq0 / G + gl);  // per group: D scales, then D zero-points
         const int pos = k_meta_position(d, D);
         meta[grp * 2 * D + pos] = sh;
@@ -253,7 +324,7 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
         float z, sc;
         __half zh, sh;
         group_params(mn, mx, bits, eta, z, sc, zh, sh);
-        par[gi * T + tl] = make_float4(z, safe_rcp(sc), sc, 0.f);
+        if (own) group_thresholds<F16>(mn, mx, z, sc, bits, thr + gi * T + tl, NPAR);
         const int tabs = tq0 + tl;
         __half* mine = meta + (size_t)bh * dm.nq_cap * 2 * NG;
         mine[v_scale_index(tabs, gi, NG)] = sh;
@@ -272,7 +343,6 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
   auto build = [&](auto bits_c) {
     constexpr int BITS = decltype(bits_c)::value;
     constexpr int N = 32 / BITS;        // codes per word
-    constexpr float QMAX = (float)((1 << BITS) - 1);
     if (kind == 0) {
       constexpr int NW = D * BITS / 32;  // words per token row
       const size_t w0 = k_code_position(tq0, 0, BITS, D).word;  // the tile's words are one contiguous run
@@ -283,25 +353,18 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
           const int tl = item % T, i = item / T, gl = tl / G;
           const uint8_t* row = tile + tl * ROWB;
           uint32_t word = 0u;
-          bool doubt = false;
 #pragma unroll
           for (int s4 = 0; s4 < N / 4; ++s4) {
-            const int d = i * N + 4 * s4;
+            const int d = i * N + 4 * s4;  // four consecutive channels: four groups
             const uint2 xx = *reinterpret_cast<const uint2*>(row + d * 2);
-            const float4 p0 = par[gl * D + d], p1 = par[gl * D + d + 1], p2 = par[gl * D + d + 2], p3 = par[gl * D + d + 3];
-            const uint32_t lo = code_pair<BITS>(I16::lo(xx.x), I16::hi(xx.x), p0, p1, doubt);
-            const uint32_t hi = code_pair<BITS>(I16::lo(xx.y), I16::hi(xx.y), p2, p3, doubt);
-            word |= (lo | (hi << 16)) << (BITS * s4);
-          }
-          if (doubt) {  // rare: the word again, with the division
-            word = 0u;
-#pragma unroll 1
-            for (int e = 0; e < N; ++e) {
-              const int d = i * N + (e / 4) * 4 + (e % 4);
-              const float4 pp = par[gl * D + d];
-              const uint32_t c = code_of(I16::one(*reinterpret_cast<const uint16_t*>(row + d * 2)), pp.x, pp.z, QMAX);
-              word |= c << (8 * (e % 4) + BITS * (e / 4));
+            const uint2 t1 = *reinterpret_cast<const uint2*>(thr + gl * D + d);
+            uint2 t2 = t1, t3 = t1;
+            if constexpr (BITS == 2) {
+              t2 = *reinterpret_cast<const uint2*>(thr + NPAR + gl * D + d);
+              t3 = *reinterpret_cast<const uint2*>(thr + 2 * NPAR + gl * D + d);
             }
+            const uint32_t lo = code_pair<BITS, V2>(xx.x, t1.x, t2.x, t3.x), hi = code_pair<BITS, V2>(xx.y, t1.y, t2.y, t3.y);
+            word |= __byte_perm(lo, hi, 0x6420) << (BITS * s4);
           }
           wbuf[k_code_position(tq0 + tl, i * N, BITS, D).word - w0] = word;
         }
@@ -330,29 +393,21 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
         if (item < D * WPC) {
           const int d = item % D, wi = item / D, gi = d / G;
           uint32_t word = 0u;
-          bool doubt = false;
 #pragma unroll
           for (int s4 = 0; s4 < N / 4; ++s4) {
-            const int tl = wi * N + 4 * s4;
+            const int tl = wi * N + 4 * s4;  // four consecutive tokens: four groups
             const uint8_t* src = tile + tl * ROWB + d * 2;
-            const float4 p0 = par[gi * T + tl], p1 = par[gi * T + tl + 1], p2 = par[gi * T + tl + 2], p3 = par[gi * T + tl + 3];
-            const float x0 = I16::one(*reinterpret_cast<const uint16_t*>(src));
-            const float x1 = I16::one(*reinterpret_cast<const uint16_t*>(src + ROWB));
-            const float x2 = I16::one(*reinterpret_cast<const uint16_t*>(src + 2 * ROWB));
-            const float x3 = I16::one(*reinterpret_cast<const uint16_t*>(src + 3 * ROWB));
-            const uint32_t lo = code_pair<BITS>(x0, x1, p0, p1, doubt);
-            const uint32_t hi = code_pair<BITS>(x2, x3, p2, p3, doubt);
-            word |= (lo | (hi << 16)) << (BITS * s4);
-          }
-          if (doubt) {
-            word = 0u;
-#pragma unroll 1
-            for (int e = 0; e < N; ++e) {
-              const int tl = wi * N + (e / 4) * 4 + (e % 4);
-              const float4 pp = par[gi * T + tl];
-              const uint32_t c = code_of(I16::one(*reinterpret_cast<const uint16_t*>(tile + tl * ROWB + d * 2)), pp.x, pp.z, QMAX);
-              word |= c << (8 * (e % 4) + BITS * (e / 4));
+            const uint32_t x0 = *reinterpret_cast<const uint16_t*>(src), x1 = *reinterpret_cast<const uint16_t*>(src + ROWB);
+            const uint32_t x2 = *reinterpret_cast<const uint16_t*>(src + 2 * ROWB), x3 = *reinterpret_cast<const uint16_t*>(src + 3 * ROWB);
+            const uint2 t1 = *reinterpret_cast<const uint2*>(thr + gi * T + tl);
+            uint2 t2 = t1, t3 = t1;
+            if constexpr (BITS == 2) {
+              t2 = *reinterpret_cast<const uint2*>(thr + NPAR + gi * T + tl);
+              t3 = *reinterpret_cast<const uint2*>(thr + 2 * NPAR + gi * T + tl);
             }
+            const uint32_t lo = code_pair<BITS, V2>(x0 | (x1 << 16), t1.x, t2.x, t3.x);
+            const uint32_t hi = code_pair<BITS, V2>(x2 | (x3 << 16), t1.y, t2.y, t3.y);
+            word |= __byte_perm(lo, hi, 0x6420) << (BITS * s4);
           }
           uint32_t* dst = codes + (size_t)bh * stream_words + v_code_position(tq0 + wi * N, d, BITS, D).word;
           if (merge || stats) {
