@@ -114,27 +114,34 @@ __device__ __forceinline__ float quotient(const Quot& g, float x) {
   return __fdiv_rn(a, g.s);
 }
 
-// X_k as a 16-bit pattern, given lattice points (as ordered integers) with c(o_lo) < k <= c(o_hi).  In real
-// numbers the threshold is tau = z + (k - 1/2) s.  The computed quotient differs from (x - z) / s by less than
-// 2^-23 relative (two roundings), i.e. by less than 3.1 * 2^-23 s in x, and t = RN(tau) from tau by at most
-// 2^-24 |t|: a lattice point at or above t + eps certainly has c >= k, one at or below t - eps certainly has not,
-// for eps = 2^-22 |t| + 2^-20 s (twice what is needed).  Where the lattice is coarser than eps -- almost always --
-// the two certain neighbours are adjacent and nothing is evaluated; otherwise (a threshold next to zero under a
-// large |z|, an exact tie on the lattice) c itself decides, by bisection between them.  Groups whose scale takes
-// the division (safe_rcp) are bisected from the group's ends.
+// X_k as a 16-bit pattern for a group with minimum mn and maximum mx.  In real numbers the threshold is
+// tau = z + (k - 1/2) s.  The computed quotient differs from (x - z) / s by less than 2^-23 relative (two
+// roundings), i.e. by less than 3.1 * 2^-23 s in x, and t = RN(tau) from tau by at most 2^-24 |t|: a lattice point
+// at or above t + eps certainly has c >= k, one below t - eps certainly has not, for eps = 2^-22 |t| + 2^-20 s
+// (twice what is needed).  Where the lattice is coarser than eps -- almost always -- no lattice point lies between
+// the bounds and nothing is evaluated; otherwise (a threshold next to zero under a large |z|, an exact tie on the
+// lattice) c itself decides, by bisection between the bounds.  Groups whose scale takes the division (safe_rcp)
+// are bisected from the group's ends (c(mn) = 0, c(mx) = 2^B - 1).
 template <bool F16>
-__device__ __forceinline__ uint32_t threshold16(const Quot& g, int k, int o_lo, int o_hi) {
+__device__ __forceinline__ uint32_t threshold16(const Quot& g, int k, float mn, float mx) {
   const float kk = (float)k - 0.5f;
-  const bool even = (k & 1) == 0;  // rint takes a tie to the even neighbour: k - 1/2 counts as >= k only for even k
-  int lo = o_lo, hi = o_hi;
+  int lo, hi;  // ordered integers of lattice points with c(lo) < k <= c(hi)
   if (g.fast) {
     const float t = __fmaf_rn(kk, g.s, g.z);
     const float eps = __fmaf_rn(fabsf(t), 0x1p-22f, __fmul_rn(g.s, 0x1p-20f));
-    const int o_up = ord16(In16<F16>::bits_up(__fadd_ru(t, eps)));   // the smallest lattice point >= t + eps
-    const int o_dn = ord16(In16<F16>::bits_down(__fadd_rd(t, -eps)));  // the largest one <= t - eps
-    if (o_dn > lo && o_dn < hi) lo = o_dn;
-    if (o_up < hi && o_up > lo) hi = o_up;
+    // the smallest lattice points at or above t + eps and at or above t - eps: the same point when no lattice
+    // point lies between the two bounds, and then it is X_k (mn lies below t - eps, mx above t + eps: the
+    // thresholds are half a step and more away from both)
+    const uint32_t up = In16<F16>::bits_up(__fadd_ru(t, eps)), up_lo = In16<F16>::bits_up(__fadd_rd(t, -eps));
+    constexpr uint32_t INF16 = F16 ? 0x7c00u : 0x7f80u;
+    if (up == up_lo && up != INF16) return up;
+    hi = up != INF16 ? ord16(up) : ord16(In16<F16>::bits(mx));  // (a bound beyond the largest finite value)
+    lo = ord16(up_lo) - 1;  // below t - eps
+  } else {
+    lo = ord16(In16<F16>::bits(mn));
+    hi = ord16(In16<F16>::bits(mx));
   }
+  const bool even = (k & 1) == 0;  // rint takes a tie to the even neighbour: k - 1/2 counts as >= k only for even k
   while (hi - lo > 1) {
     const int mid = lo + ((hi - lo) >> 1);
     const float q = quotient(g, In16<F16>::one((uint16_t)pat16(mid)));
@@ -150,11 +157,10 @@ __device__ __forceinline__ void group_thresholds(float mn, float mx, float z, fl
   constexpr uint16_t INF16 = F16 ? 0x7c00u : 0x7f80u;
   const float y = safe_rcp(sc);
   const Quot g{z, sc, y, y == y};
-  const int o_lo = ord16(In16<F16>::bits(mn)), o_hi = ord16(In16<F16>::bits(mx));
   const int qmax = (1 << bits) - 1;
 #pragma unroll
   for (int k = 1; k <= 3; ++k)
-    thr[(k - 1) * stride] = (k <= qmax && sc != 0.0f) ? (uint16_t)threshold16<F16>(g, k, o_lo, o_hi) : INF16;
+    thr[(k - 1) * stride] = (k <= qmax && sc != 0.0f) ? (uint16_t)threshold16<F16>(g, k, mn, mx) : INF16;
 }
 
 // Codes of two packed 16-bit elements against their groups' packed thresholds: code of the low element at bit 0,
@@ -168,8 +174,11 @@ __device__ __forceinline__ uint32_t code_pair(uint32_t x, uint32_t t1, uint32_t 
   } else {
     const uint32_t m2 = __hge2_mask(xv, *reinterpret_cast<const V2*>(&t2));
     const uint32_t m3 = __hge2_mask(xv, *reinterpret_cast<const V2*>(&t3));
-    // m3 implies m2 implies m1: code bit 0 = (m1 and not m2) or m3, bit 1 = m2
-    return (((m1 & ~m2) | m3) & 0x00010001u) | (m2 & 0x00020002u);
+    // A mask is 0xffff per element that passed.  n = -(m1 + m2 + m3) holds the low element's count in its low
+    // half and (high count - low count) in its high half (the low half borrows); n * 0x10001 adds the low count
+    // back to the high half.
+    const uint32_t n = 0u - m1 - m2 - m3;
+    return n * 0x10001u;
   }
 }
 
@@ -190,7 +199,7 @@ __device__ __forceinline__ void delta_count(uint32_t w0, uint32_t w1, uint32_t (
 // offset), the words are collected in shared memory in stream order and leave in 16-byte vectors.  Values: a
 // thread builds whole words of a channel's row over the tile's tokens and stores them itself.
 // G: group size; T = p.tb: a multiple of G and of 32; F16: the 16-bit type is IEEE half precision.
-// blockIdx.z runs over (layer of the launch, sequence).  With p.win_count > 0 the CTAs of the first block also copy
+// blockIdx.y is the (sequence, kv head) stream, blockIdx.z the layer of the launch.  With p.win_count > 0 the CTAs of the first block also copy
 // the new window rows that replace the rows they staged.
 template <int D, int G, int T, bool F16>
 __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constant__ PackParams p) {
@@ -213,9 +222,8 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
   const int R = dm.R;
   const int kind = blockIdx.x & 1;  // 0 keys, 1 values
   const int tile_idx = blockIdx.x >> 1;
-  const int h = blockIdx.y, b = blockIdx.z % dm.B;
-  const PackLayer pl = p.layer[blockIdx.z / dm.B];  // by value: its fields are read in every loop below
-  const int bh = b * dm.Hkv + h;
+  const PackLayer pl = p.layer[blockIdx.z];  // by value: its fields are read in every loop below
+  const int bh = blockIdx.y;                  // (sequence, kv head) stream
   const int tid = threadIdx.x;
   const int tq0 = p.nq_old + tile_idx * T;  // absolute index of the tile's first token
 
@@ -223,13 +231,15 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
     const uint16_t* win = kind ? pl.L.win_v : pl.L.win_k;
     const uint16_t* in = kind ? pl.V_in : pl.K_in;
     constexpr int VPR = D / 8;
+    // row `pabs` (absolute token) of the stream: in the old window while pabs < s_old, else in the input
+    const uint16_t* const win_rows = win + ((size_t)bh * R - p.nq_old) * D;
+    const uint16_t* const in_rows = in + ((size_t)bh * p.n_in - p.s_old) * D;
 #pragma unroll
     for (int k = 0; k < T * VPR / PACK_THREADS; ++k) {
       const int idx = tid + k * PACK_THREADS;
       const int tl = idx / VPR, c8 = idx % VPR;
       const int pabs = tq0 + tl;
-      const uint16_t* src = (pabs < p.s_old) ? win + ((size_t)bh * R + (pabs - p.nq_old)) * D
-                                             : in + ((size_t)bh * p.n_in + (pabs - p.s_old)) * D;
+      const uint16_t* src = (pabs < p.s_old ? win_rows : in_rows) + (size_t)pabs * D;
       *reinterpret_cast<uint4*>(tile + tl * ROWB + c8 * 16) = reinterpret_cast<const uint4*>(src)[c8];
     }
   }
@@ -434,7 +444,7 @@ __global__ void __launch_bounds__(PACK_THREADS) pack_kernel(const __grid_constan
 template <bool F16>
 cudaError_t launch_pack_t(const PackParams& p, cudaStream_t st) {
   int tiles = p.n_blocks * (p.dm.R / p.tb);
-  dim3 grid(2 * tiles, p.dm.Hkv, p.dm.B * p.n_layers);
+  dim3 grid(2 * tiles, p.dm.B * p.dm.Hkv, p.n_layers);
   const int key = p.dm.D * 10000 + p.dm.g * 100 + p.tb;
   switch (key) {
     case 1283232: pack_kernel<128, 32, 32, F16><<<grid, PACK_THREADS, 0, st>>>(p); break;
