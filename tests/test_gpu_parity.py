@@ -575,6 +575,44 @@ def test_decode_right_after_the_pack_of_the_layer_it_reads():
     cache.close()
 
 
+def test_chained_decode_launches_equal_single_calls():
+    """The decode launches of a step overlap: each after the first reads at once and waits for its predecessor only
+    before it writes the scratch and its result.  Eight layers of the 32k shape at a length where a launch fills
+    every slot of the device, twelve steps back to back on one stream (one of them fills the window blocks and
+    packs): every layer's result of every step equals, bit for bit, what a second cache with the same contents
+    returns through separate xq_append_kv / xq_decode_attention calls, which never overlap."""
+    L = 8
+    w = dict(W.CONFIGS["c2"], n_layers=L, seq=6000)
+    w["kq"], w["vq"] = L, 0
+    cfg = W.make_xq_config(w, max_seq=6000 + 64)
+    a, b = xq.Cache(cfg, DEV), xq.Cache(cfg, DEV)
+    S0 = 6000 + 8  # 6008 = 46 blocks of 128 + 120 in the window: step 9 fills the blocks
+    for cache in (a, b):
+        for pair in range(L // 2):
+            k0, v0, k1, v1 = W.pair_tokens(w, pair, 0, S0, DEV)
+            cache.append_kv(2 * pair, k0, v0)
+            cache.append_kv(2 * pair + 1, k1, v1)
+    B, Hkv, Hq, D = w["batch"], w["n_kv_heads"], w["n_q_heads"], w["head_dim"]
+    gen = torch.Generator(device="cpu").manual_seed(33)
+    steps = 12
+    kn = [torch.randn(L, B, Hkv, 1, D, generator=gen).to(torch.bfloat16).to(DEV) for _ in range(steps)]
+    vn = [torch.randn(L, B, Hkv, 1, D, generator=gen).to(torch.bfloat16).to(DEV) for _ in range(steps)]
+    q = [torch.randn(L, B, Hq, D, generator=gen).to(torch.bfloat16).to(DEV) for _ in range(steps)]
+    outs = [torch.empty_like(q[0]) for _ in range(steps)]
+    torch.cuda.synchronize()
+    for i in range(steps):  # nothing between the steps
+        a.decode_step(kn[i], vn[i], q[i], outs[i])
+    torch.cuda.synchronize()
+    a.check_device()  # raises if a kernel gave up a bounded wait
+    for i in range(steps):
+        for l in range(L):
+            b.append_kv(l, kn[i][l], vn[i][l])
+            ref = b.decode_attention(l, q[i][l])
+            assert torch.equal(ref, outs[i][l]), (i, l)
+    assert a.quantized_len(0) == b.quantized_len(0) == 47 * 128
+    a.close(); b.close()
+
+
 def test_decode_step_from_host_buffers_at_full_size():
     """xq_decode_step with pinned host buffers (the end-to-end path the benchmark times) on the 32k GQA shape with
     one layer pair: three steps, sampled streams against the oracle."""
