@@ -270,6 +270,75 @@ def test_pack_on_lattice_data_with_exact_ties(bits, D, g):
     cache.close()
 
 
+@pytest.mark.filterwarnings("ignore:overflow encountered in cast")  # scales of 1e30 stored as 16-bit floats
+@pytest.mark.parametrize("f16", [False, True])
+@pytest.mark.parametrize("bits", [(2, 2), (0, 0)])
+def test_pack_on_groups_that_are_hard_for_the_thresholds(bits, f16):
+    """The pack kernel codes by comparing against per-group thresholds on the 16-bit input lattice.  Groups where
+    finding them takes the slow paths: a threshold next to zero under a large |z| with elements of every small
+    magnitude around it (the lattice there is far finer than the quotient can tell apart), a scale whose
+    significand is all ones (2 - 2^-23 times a power of two: the reciprocal sequence is not trusted), scales of
+    extreme exponent (bfloat16 only), constant groups.  Codes, scales and zero-points against the oracle, bit for
+    bit; no attention (the magnitudes are not a model's)."""
+    L, B, Hkv, D, g, R = 2, 1, 2, 128, 32, 64
+    kq, vq = bits
+    S = 2 * R + 5
+    dt = torch.float16 if f16 else torch.bfloat16
+    w = dict(n_layers=L, batch=B, n_q_heads=Hkv, n_kv_heads=Hkv, head_dim=D, seq=S, residual_len=R,
+             group_size=g, kq=kq, vq=vq, km=0, vm=0, n_outliers=0, outlier_scale=1.0, seed=1, n_splits=0)
+    cfg = W.make_xq_config(w, io_dtype=xq.XQ_F16 if f16 else xq.XQ_BF16)
+    cache = xq.Cache(cfg, DEV)
+    gen = torch.Generator().manual_seed(7 + kq + 2 * int(f16))
+    lo_exp = -20 if f16 else -120
+    kv = {}
+    for l in range(L):
+        K = torch.randn(B, Hkv, S, D, generator=gen)
+        V = torch.randn(B, Hkv, S, D, generator=gen)
+
+        def tiny(shape):
+            e = torch.randint(lo_exp, -6, shape, generator=gen).float()
+            sign = torch.randint(0, 2, shape, generator=gen).float() * 2 - 1
+            t = sign * torch.exp2(e)
+            t[torch.rand(shape, generator=gen) < 0.2] = 0.0
+            t[torch.rand(shape, generator=gen) < 0.1] = -0.0
+            return t
+
+        # thresholds at zero: the ends +-5 (also +-6 with an odd spacing), everything else tiny or zero
+        for ch, end in ((3, 5.0), (4, 6.0)):
+            K[:, :, :, ch] = tiny((B, Hkv, S))
+            K[:, :, 0::8, ch] = end
+            K[:, :, 1::8, ch] = -end
+        for tok, end in ((5, 5.0), (6, 6.0)):
+            V[:, :, tok::16, :] = tiny(V[:, :, tok::16, :].shape)
+            V[:, :, tok::16, 0::8] = end
+            V[:, :, tok::16, 1::8] = -end
+        # 1-bit scale (max - min) with a significand of 24 ones: min = 2^-22, max = 4 -> 4 - 2^-22
+        mn = 2.0 ** -22 if not f16 else 2.0 ** -14  # (half precision: 4 - 2^-14 has 17 ones; still an odd case)
+        K[:, :, :, 7] = torch.rand(B, Hkv, S, generator=gen) * 3 + 0.5
+        K[:, :, 0::4, 7] = 4.0
+        K[:, :, 1::4, 7] = mn
+        V[:, :, 9::16, :] = torch.rand(V[:, :, 9::16, :].shape, generator=gen) * 3 + 0.5
+        V[:, :, 9::16, 0::4] = 4.0
+        V[:, :, 9::16, 1::4] = mn
+        if not f16:
+            # scales of extreme exponent: the reciprocal sequence is not used
+            K[:, :, :, 11] = (torch.rand(B, Hkv, S, generator=gen) * 2 + 1) * 1e-30
+            K[:, :, :, 13] = (torch.rand(B, Hkv, S, generator=gen) * 2 - 1) * 1e30
+            V[:, :, 13::16, :] = (torch.rand(V[:, :, 13::16, :].shape, generator=gen) * 2 + 1) * 1e-30
+            V[:, :, 14::16, :] = (torch.rand(V[:, :, 14::16, :].shape, generator=gen) * 2 - 1) * 1e30
+        K[:, :, :, 17] = -0.75  # constant groups
+        V[:, :, 3::16, :] = 0.0
+        kv[l] = (K.to(dt).to(DEV), V.to(dt).to(DEV))
+        for lo in range(0, S, 40):
+            cache.append_kv(l, kv[l][0][:, :, lo:lo + 40].contiguous(), kv[l][1][:, :, lo:lo + 40].contiguous())
+    torch.cuda.synchronize()
+    for l in range(L):
+        for hk in range(Hkv):
+            oc = util.oracle_for_stream(cfg, list(range(L)), 0, hk, kv)
+            util.compare_regions(cache, oc, l, 0, hk)
+    cache.close()
+
+
 @pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 6, 7, 8])
 def test_decode_step_head_groupings(G):
     """Every size of query-head group the tensor-core kernel takes, through xq_decode_step (in-kernel append) over
