@@ -59,7 +59,8 @@ def _ncu_traffic(config):
 
 def _config_block(args, w):
     """What both arms print as `config`: the workload by name and its shape."""
-    return {"workload": f"{args.config}: BASELINE.json configs[{args.config[1:]}]",
+    from paper_2510_11236_b200 import workloads
+    return {"workload": f"{args.config}: {workloads.TITLES.get(args.config, 'custom')}",
             **{k: w[k] for k in ("n_layers", "batch", "n_q_heads", "n_kv_heads", "head_dim", "seq", "residual_len",
                                  "group_size", "kq", "vq", "km", "vm")},
             "eta1": args.eta1, "eta2": args.eta2,

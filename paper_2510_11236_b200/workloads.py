@@ -37,6 +37,16 @@ CONFIGS = {
                 group_size=32, kq=48, vq=24, km=0, vm=0, n_outliers=3, outlier_scale=10.0, seed=5, n_splits=0),
 }
 
+# one line per workload for reports
+TITLES = {
+    "c0": "configuration 0: tiny layer pair, 4 heads, head_dim 64, 512 tokens",
+    "c1": "configuration 1: Llama-2-7B-shaped MHA, batch 8, 4k context, 2-bit keys and values",
+    "c2": "configuration 2: Llama-3-8B-shaped GQA, batch 4, 32k context, 2-bit keys, 1-bit values",
+    "c3": "configuration 3: Mistral-7B-shaped GQA, batch 16, 8k context, groups of 64, 2-bit keys and values",
+    "c4": "configuration 4: long context, batch 1, 128k tokens, 64 splits per head",
+    "q14": "Qwen2.5-14B-shaped GQA (48 layers, groups of five heads), batch 4, 16k context",
+}
+
 NOISE_SIGMA = 0.1
 
 
