@@ -20,7 +20,7 @@ identity of the calibration derivation, the 1-bit MSE closed form and brute
 force on tiny groups; packing against the round-trip identity and a bit census;
 attention against brute-force loops, the empty-quantized-region case and the
 uniform-logit case; the gamma-interval enumeration of the weighted merge.
-Parity unpinned by the paper (fixed by this build's readings and then enforced
+Parity unpinned by the paper (fixed by readings of it made here and then enforced
 between the oracle and the CUDA path): the residual-window flush policy, the
 fp16 storage type of scale / zero-point and the bit layout of packed words.
 """
@@ -229,7 +229,7 @@ def merge_codes_gamma1(e0: np.ndarray, e1: np.ndarray, gamma1) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------
-# Packed layouts (this build's choice; the paper does not discuss packing)
+# Packed layouts (a choice made here; the paper does not discuss packing)
 # --------------------------------------------------------------------------
 # Words are little-endian 32-bit.  A byte of a word holds the codes of 8/bits
 # row elements, the four bytes of a word hold four consecutive row elements at
